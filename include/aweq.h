@@ -1,0 +1,245 @@
+/*
+ * aweq.h -- C ABI of the B200 (sm_100a) AWEQ calibration library.
+ *
+ * AWEQ (arXiv 2311.01305, "Post-Training Quantization with Activation-Weight
+ * Equalization for Large Language Models") calibrates one linear layer
+ * y = W x (+ bias) from N calibration inputs x_1..x_N in six steps:
+ *   1. per-channel min / max / mean of the inputs            aweq_stats
+ *   2. per-input-channel range of the weights                aweq_wrange
+ *   3. equalisation factors s (Eq. 10) and diagnostics       aweq_factors
+ *   4. fold s into W and quantise (Eq. 3, Eq. 1-2), pack     aweq_equalize_quantize
+ *   5. statistical bias correction (Eq. 11-15)               aweq_bias_correct
+ *   6. 8-bit quantisation of the equalised inputs (W8A8)     aweq_quant_act
+ * aweq_layer_pass runs all six for one input and the matrices it feeds.
+ *
+ * General rules
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned
+ *     by the caller.  The library allocates no device memory and keeps no
+ *     per-call state; scratch memory is passed in as `ws` (size from
+ *     aweq_workspace_bytes, 256-byte aligned, contents irrelevant on entry).
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) and the call returns without synchronising.
+ *   - The return value is the result of host-side validation and of the
+ *     launches.  When it is not AWEQ_OK nothing was enqueued (validation) or
+ *     the CUDA error is reported (AWEQ_ERR_CUDA); no exception crosses the ABI.
+ *   - Conditions found on the device are counted into *st (may be NULL); the
+ *     caller zeroes it and reads it back after synchronising.
+ *   - Matrices are row-major with the innermost dimension contiguous.
+ *     X is [N x C_in] with row pitch ldx elements, W is [C_out x C_in] with
+ *     row pitch ldw elements ("channel i" of the paper is always the input
+ *     channel, a column of both).  16-bit elements are fp16 or bf16.
+ *     Base pointers of X and W must be 16-byte aligned, ldx / ldw and C_in
+ *     multiples of 8; a violation is an error code, never a fault.
+ *   - Outputs are overwritten completely unless `accumulate` is set.
+ *   - Floating-point decisions that produce integer codes are taken in IEEE
+ *     binary32, round to nearest even, without fused multiply-add:
+ *     v^ = fl(v * scale), Step = fl(fl(hi - lo) / (2^b - 1)),
+ *     inv = fl(1 / Step), Z = -rint(fl(lo * inv)),
+ *     q = clamp(rint(fl(v^ * inv)) + Z, 0, 2^b - 1).
+ *     A constant vector (hi == lo) takes Step = |lo| (1 if lo == 0).
+ */
+#ifndef AWEQ_H
+#define AWEQ_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AWEQ_OK = 0,
+    AWEQ_ERR_NULL = 1,        /* a required pointer is NULL */
+    AWEQ_ERR_SHAPE = 2,       /* a size is <= 0, not a multiple of 8, or too large */
+    AWEQ_ERR_ALIGN = 3,       /* a base pointer or pitch breaks the alignment rule */
+    AWEQ_ERR_DTYPE = 4,
+    AWEQ_ERR_BITS = 5,        /* bit-width outside 2..8 */
+    AWEQ_ERR_GROUP = 6,       /* group size not a power of two in [8, 256] or not dividing C_in */
+    AWEQ_ERR_WORKSPACE = 7,   /* ws is NULL, misaligned or smaller than aweq_workspace_bytes */
+    AWEQ_ERR_CUDA = 8,        /* a CUDA call failed; see aweq_last_cuda_error */
+    AWEQ_ERR_UNSUPPORTED = 9
+} aweq_status;
+
+typedef enum { AWEQ_F16 = 0, AWEQ_BF16 = 1 } aweq_dtype;
+
+/* Granularity of one (Step, Z) pair: the whole tensor; one row (an output
+ * channel of W, a token of X); or a group of `group` consecutive input
+ * channels inside one row of W. */
+typedef enum { AWEQ_PER_TENSOR = 0, AWEQ_PER_ROW = 1, AWEQ_PER_GROUP = 2 } aweq_gran;
+
+/* Device-side condition counters.  nonfinite: channels / vectors whose
+ * statistics were Inf or NaN; zero_range: dead channels (factor forced to 1);
+ * wait_timeout: a bounded wait inside a kernel gave up (results of that call
+ * are invalid). */
+typedef struct {
+    unsigned long long nonfinite;
+    unsigned long long zero_range;
+    unsigned long long wait_timeout;
+    unsigned long long reserved;
+} aweq_dev_status;
+
+typedef enum {
+    AWEQ_OP_STATS = 1,
+    AWEQ_OP_WRANGE = 2,
+    AWEQ_OP_EQUALIZE_QUANTIZE = 4,
+    AWEQ_OP_BIAS_CORRECT = 5,
+    AWEQ_OP_QUANT_ACT = 6
+} aweq_op;
+
+/* Host helpers (no CUDA calls). */
+const char *aweq_strerror(aweq_status code);
+const char *aweq_last_cuda_error(void);          /* text of the last CUDA error seen by this thread */
+int aweq_version(void);
+/* Number of kernels this library has launched in this process (diagnostic). */
+unsigned long long aweq_launch_count(void);
+
+/* Scratch bytes an operation needs for the given shape: rows x cols is
+ * N x C_in for AWEQ_OP_STATS / AWEQ_OP_QUANT_ACT and C_out x C_in for the
+ * weight operations.  Returns 0 when the operation needs none. */
+size_t aweq_workspace_bytes(int op, long long rows, long long cols, int bits, int gran, int group);
+
+/*
+ * Step 1 -- calibration statistics (Section 3.2: the range of channel i is its
+ * maximum minus its minimum over all inputs; Section 3.3, last paragraph: E[x]
+ * is gathered in the same sweep as the factors).
+ *   xmin[j] = min_n X[n,j], xmax[j] = max_n X[n,j]  (exact)
+ *   xmean[j] = (1/N) sum_n X[n,j]  (binary32 partial sums over at most 8 rows,
+ *              folded into binary64; final division in binary64)
+ * X: [N x C_in] 16-bit, read once.  xmin, xmax, xmean: float[C_in], written.
+ * xsum: double[C_in], count: long long[1] -- optional running state; both
+ * required when accumulate != 0, in which case xmin / xmax / xsum / count
+ * hold the result of earlier chunks on entry and the merged result on exit
+ * (calibration data can be streamed in chunks; also the hook for sharding
+ * tokens over devices).  N == 0 is allowed (identity).
+ * ws: aweq_workspace_bytes(AWEQ_OP_STATS, N, C_in, 0, 0, 0).
+ */
+aweq_status aweq_stats(const void *X, aweq_dtype dt, long long N, long long C_in, long long ldx,
+                       float *xmin, float *xmax, float *xmean,
+                       double *xsum, long long *count, int accumulate,
+                       void *ws, size_t ws_bytes, aweq_dev_status *st, void *stream);
+
+/*
+ * Step 2 -- per-input-channel weight range (Section 3.2, same definition
+ * applied to W): wmin[j] = min_o W[o,j], wmax[j] = max_o W[o,j].
+ * accumulate != 0 merges with the values already in wmin / wmax, which gives
+ * matrices that share one input (q/k/v, gate/up) a common range.
+ * ws: aweq_workspace_bytes(AWEQ_OP_WRANGE, C_out, C_in, 0, 0, 0).
+ */
+aweq_status aweq_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ldw,
+                        float *wmin, float *wmax, int accumulate,
+                        void *ws, size_t ws_bytes, aweq_dev_status *st, void *stream);
+
+/*
+ * Step 3 -- equalisation factors (Eq. 10) and the quantities of Eq. 4-8.
+ *   r^X_j = xmax_j - xmin_j, r^W_j = wmax_j - wmin_j
+ *   s_j = sqrt(r^X_j / r^W_j)          (= (1/r^W_j) sqrt(r^X_j r^W_j), Eq. 10)
+ *   rinv_j = 1 / s_j, mu_hat_j = xmean_j * rinv_j  (E[x^] of the equalised input)
+ *   a dead channel (range <= 0 or not finite) gets s_j = 1 and is counted in
+ *   st->zero_range.
+ * All arrays float[C_in]; s, rinv, mu_hat required, pX, pW optional
+ * (p_j = r_j / R with R the tensor range, Eq. 4).
+ * scalars: optional double[8] = { R^X, R^W, R^X^, R^W^ (tensor ranges after
+ * equalisation), objective of Eq. 5 before and after, the max*max product of
+ * Eq. 8 before (s = 1) and after }.  C_in <= 1048576.
+ */
+aweq_status aweq_factors(const float *xmin, const float *xmax, const float *xmean,
+                         const float *wmin, const float *wmax, long long C_in,
+                         float *s, float *rinv, float *mu_hat, float *pX, float *pW, double *scalars,
+                         aweq_dev_status *st, void *stream);
+
+/*
+ * Step 4 -- fold s into W and quantise (Eq. 3: W^ = diag(s) W, so input
+ * channel j of every row is multiplied by s_j; Eq. 1-2 on every row or group).
+ * One pass over W: rescale, range, quantise and pack are fused.
+ * s: float[C_in] or NULL (no equalisation: the round-to-nearest baseline of
+ * Section 4.2).  mu_hat: float[C_in] or NULL; when given with epsmu,
+ *   epsmu[o] = sum_j (Step (q - Z) - W^[o,j]) mu_hat[j]     (eps . E[x^], Eq. 15)
+ * is produced in the same pass (binary32 accumulation, fixed order).
+ * bits in 2..8.  gran: AWEQ_PER_ROW (one pair per output channel),
+ * AWEQ_PER_GROUP (group: power of two in [8, 256] dividing C_in) or
+ * AWEQ_PER_TENSOR.  Per-row mode supports C_in <= 40960.
+ * codes: unsigned char[C_out x C_in*bits/8], the little-endian bit stream of
+ * each row: code i at bits [i*bits, (i+1)*bits) (8-bit: one per byte; 4-bit:
+ * two per byte, low nibble first; 3-bit: eight codes per three bytes).
+ * step: float, zp: int, one per row ([C_out]), per group ([C_out x C_in/group])
+ * or a single pair.  epsmu: float[C_out] or NULL.
+ * ws: aweq_workspace_bytes(AWEQ_OP_EQUALIZE_QUANTIZE, C_out, C_in, bits, gran, group).
+ */
+aweq_status aweq_equalize_quantize(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ldw,
+                                   const float *s, const float *mu_hat,
+                                   int bits, aweq_gran gran, int group,
+                                   unsigned char *codes, float *step, int *zp, float *epsmu,
+                                   void *ws, size_t ws_bytes, aweq_dev_status *st, void *stream);
+
+/*
+ * Step 5 -- bias correction (Eq. 11-15 and the sentence after them: the
+ * expected output error eps E[x] is subtracted from the output, which for a
+ * linear layer is a change of its bias):
+ *   bias_out[o] = bias_in[o] - sum_j eps[o,j] mu_hat[j],  eps = W~ - W^.
+ * Two routes.  Fused: epsmu != NULL is the sum produced by step 4 and the
+ * weight arguments are ignored.  Standalone: epsmu == NULL and the sum is
+ * recomputed from W, s, the packed codes, step, zp and mu_hat.
+ * bias_in: 16-bit [C_out] of type bias_dt, or NULL for a layer without bias
+ * (the correction then creates one).  bias_out: 16-bit [C_out] (may be NULL);
+ * bias_out_f32: float[C_out] (may be NULL); at least one must be given.
+ */
+aweq_status aweq_bias_correct(const float *epsmu,
+                              const void *W, aweq_dtype dt, const float *s, const unsigned char *codes,
+                              const float *step, const int *zp, const float *mu_hat,
+                              long long C_out, long long C_in, long long ldw, int bits, aweq_gran gran, int group,
+                              const void *bias_in, void *bias_out, float *bias_out_f32, aweq_dtype bias_dt,
+                              aweq_dev_status *st, void *stream);
+
+/*
+ * Step 6 -- quantise the equalised inputs X^ = X diag(s)^-1 (Eq. 3) with
+ * Eq. 1-2 (the activation half of the W8A8 setting of Section 4.4).
+ * rinv: float[C_in] (1 / s) or NULL (no equalisation).  bits in 2..8, one code
+ * per byte.  gran: AWEQ_PER_ROW = one (Step, Z) per token, computed from that
+ * row; AWEQ_PER_TENSOR = a static range: tensor_lo_hi is float[2] = { lo, hi }
+ * of X^ (for instance min_j xmin_j rinv_j and max_j xmax_j rinv_j from step 1)
+ * and step / zp receive one pair.  Per-token mode supports C_in <= 40960.
+ * Xq: unsigned char[N x C_in] (dense rows); step: float[N]; zp: int[N].
+ */
+aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long C_in, long long ldx,
+                           const float *rinv, int bits, aweq_gran gran, const float *tensor_lo_hi,
+                           unsigned char *Xq, float *step, int *zp,
+                           aweq_dev_status *st, void *stream);
+
+/*
+ * One calibration pass for one input X and the n_w weight matrices it feeds,
+ * all six steps in order on `stream` (steps 1-2, then 3, then 4-5 per matrix,
+ * then 6 when Xq != NULL).  Per-channel vectors are float[C_in]; the arrays of
+ * pointers and sizes are HOST arrays of length n_w, their elements device
+ * pointers.  bias_in / bias_out / bias_out_f32 may be NULL, as may their
+ * entries (see aweq_bias_correct).  flags: AWEQ_FLAG_* below.
+ * ws must hold aweq_layer_pass_workspace_bytes().
+ */
+#define AWEQ_FLAG_NO_EQUALIZE 1      /* s = 1: plain round-to-nearest */
+#define AWEQ_FLAG_NO_BIAS_CORRECT 2  /* skip step 5 */
+
+typedef struct {
+    /* input */
+    const void *X; aweq_dtype dt; long long N, C_in, ldx;
+    /* weights sharing this input (host arrays of length n_w) */
+    int n_w;
+    const void *const *W; const long long *C_out; const long long *ldw;
+    int bits; aweq_gran gran; int group;
+    const void *const *bias_in; void *const *bias_out; float *const *bias_out_f32;
+    /* per-matrix outputs (host arrays of device pointers) */
+    unsigned char *const *codes; float *const *step; int *const *zp; float *const *epsmu;
+    /* per-channel outputs */
+    float *xmin, *xmax, *xmean, *wmin, *wmax, *s, *rinv, *mu_hat;
+    float *pX, *pW; double *scalars;             /* optional */
+    /* activation quantisation (optional: Xq == NULL skips step 6) */
+    unsigned char *Xq; float *act_step; int *act_zp; int act_bits;
+    int flags;
+} aweq_layer_args;
+
+size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args);
+aweq_status aweq_layer_pass(const aweq_layer_args *args, void *ws, size_t ws_bytes,
+                            aweq_dev_status *st, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AWEQ_H */
