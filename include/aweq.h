@@ -132,7 +132,8 @@ aweq_status aweq_wrange(const void *W, aweq_dtype dt, long long C_out, long long
 /*
  * Step 3 -- equalisation factors (Eq. 10) and the quantities of Eq. 4-8.
  *   r^X_j = xmax_j - xmin_j, r^W_j = wmax_j - wmin_j
- *   s_j = sqrt(r^X_j / r^W_j)          (= (1/r^W_j) sqrt(r^X_j r^W_j), Eq. 10)
+ *   s_j = (1/r^W_j) sqrt(r^X_j r^W_j)   (Eq. 10 evaluated in binary64 and rounded
+ *                                       once to binary32; = sqrt(r^X_j / r^W_j))
  *   rinv_j = 1 / s_j, mu_hat_j = xmean_j * rinv_j  (E[x^] of the equalised input)
  *   a dead channel (range <= 0 or not finite) gets s_j = 1 and is counted in
  *   st->zero_range.

@@ -1,0 +1,312 @@
+// The C ABI: host-side validation, workspace sizing and the composition of the
+// six calibration steps into one layer pass.  No device memory is allocated
+// here and nothing synchronises.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace aweq {
+
+static std::atomic<unsigned long long> g_launches{0};
+static thread_local char g_cuda_error[256] = "";
+
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+aweq_status cuda_failed(cudaError_t e)
+{
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return AWEQ_ERR_CUDA;
+}
+
+static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+static inline size_t round256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+static aweq_status check_matrix(const void *M, aweq_dtype dt, long long rows, long long cols, long long ld,
+                                bool allow_zero_rows)
+{
+    if (!M) return AWEQ_ERR_NULL;
+    if (dt != AWEQ_F16 && dt != AWEQ_BF16) return AWEQ_ERR_DTYPE;
+    if (cols <= 0 || (cols % 8) != 0 || cols > (1ll << 30)) return AWEQ_ERR_SHAPE;
+    if (rows < 0 || (rows == 0 && !allow_zero_rows) || rows > (1ll << 40)) return AWEQ_ERR_SHAPE;
+    if (ld < cols || (ld % 8) != 0) return AWEQ_ERR_ALIGN;
+    if (!aligned(M, 16)) return AWEQ_ERR_ALIGN;
+    return AWEQ_OK;
+}
+
+static aweq_status check_quant(int bits, int gran, int group, long long cols)
+{
+    if (bits < 2 || bits > 8) return AWEQ_ERR_BITS;
+    if (gran != AWEQ_PER_TENSOR && gran != AWEQ_PER_ROW && gran != AWEQ_PER_GROUP) return AWEQ_ERR_UNSUPPORTED;
+    if (gran == AWEQ_PER_GROUP) {
+        if (group < 8 || group > 256 || (group & (group - 1)) != 0 || (cols % group) != 0) return AWEQ_ERR_GROUP;
+    }
+    return AWEQ_OK;
+}
+
+static aweq_status check_ws(void *ws, size_t ws_bytes, size_t need)
+{
+    if (need == 0) return AWEQ_OK;
+    if (!ws || !aligned(ws, 256) || ws_bytes < need) return AWEQ_ERR_WORKSPACE;
+    return AWEQ_OK;
+}
+
+static size_t eq_ws_bytes(long long rows, long long cols, int gran)
+{
+    if (gran != AWEQ_PER_TENSOR) return 0;
+    // per-tensor: column extremes of W (2 x float[cols]) + lo/hi + the column-reduction scratch
+    return round256((size_t)cols * 8) + 256 + colreduce_ws_bytes(rows, cols);
+}
+
+}  // namespace aweq
+
+using namespace aweq;
+
+extern "C" {
+
+const char *aweq_strerror(aweq_status code)
+{
+    switch (code) {
+    case AWEQ_OK: return "ok";
+    case AWEQ_ERR_NULL: return "a required pointer is NULL";
+    case AWEQ_ERR_SHAPE: return "bad shape (sizes must be positive, C_in a multiple of 8 and within the supported range)";
+    case AWEQ_ERR_ALIGN: return "bad alignment (16-byte base pointers, row pitch a multiple of 8 elements and >= C_in)";
+    case AWEQ_ERR_DTYPE: return "unknown 16-bit element type";
+    case AWEQ_ERR_BITS: return "bit-width must be in 2..8";
+    case AWEQ_ERR_GROUP: return "group size must be a power of two in [8, 256] that divides C_in";
+    case AWEQ_ERR_WORKSPACE: return "workspace missing, misaligned (256 bytes) or too small";
+    case AWEQ_ERR_CUDA: return "a CUDA call failed";
+    case AWEQ_ERR_UNSUPPORTED: return "unsupported mode";
+    }
+    return "unknown status";
+}
+
+const char *aweq_last_cuda_error(void) { return g_cuda_error; }
+int aweq_version(void) { return 100; }
+unsigned long long aweq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t aweq_workspace_bytes(int op, long long rows, long long cols, int bits, int gran, int group)
+{
+    (void)bits; (void)group;
+    if (cols <= 0 || rows < 0) return 0;
+    switch (op) {
+    case AWEQ_OP_STATS:
+    case AWEQ_OP_WRANGE: return colreduce_ws_bytes(rows, cols);
+    case AWEQ_OP_EQUALIZE_QUANTIZE: return eq_ws_bytes(rows, cols, gran);
+    default: return 0;
+    }
+}
+
+aweq_status aweq_stats(const void *X, aweq_dtype dt, long long N, long long C_in, long long ldx, float *xmin,
+                       float *xmax, float *xmean, double *xsum, long long *count, int accumulate, void *ws,
+                       size_t ws_bytes, aweq_dev_status *st, void *stream)
+{
+    aweq_status rc = check_matrix(X, dt, N, C_in, ldx, true);
+    if (rc != AWEQ_OK) return rc;
+    if (!xmin || !xmax || !xmean) return AWEQ_ERR_NULL;
+    if (accumulate && (!xsum || !count)) return AWEQ_ERR_NULL;
+    if (!aligned(xmin, 16) || !aligned(xmax, 16) || !aligned(xmean, 4) || (xsum && !aligned(xsum, 8)))
+        return AWEQ_ERR_ALIGN;
+    rc = check_ws(ws, ws_bytes, colreduce_ws_bytes(N, C_in));
+    if (rc != AWEQ_OK) return rc;
+    return run_stats(X, dt, N, C_in, ldx, xmin, xmax, xmean, xsum, count, accumulate, ws, st, (cudaStream_t)stream);
+}
+
+aweq_status aweq_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ldw, float *wmin,
+                        float *wmax, int accumulate, void *ws, size_t ws_bytes, aweq_dev_status *st, void *stream)
+{
+    aweq_status rc = check_matrix(W, dt, C_out, C_in, ldw, false);
+    if (rc != AWEQ_OK) return rc;
+    if (!wmin || !wmax) return AWEQ_ERR_NULL;
+    rc = check_ws(ws, ws_bytes, colreduce_ws_bytes(C_out, C_in));
+    if (rc != AWEQ_OK) return rc;
+    return run_wrange(W, dt, C_out, C_in, ldw, wmin, wmax, accumulate, ws, st, (cudaStream_t)stream);
+}
+
+aweq_status aweq_factors(const float *xmin, const float *xmax, const float *xmean, const float *wmin,
+                         const float *wmax, long long C_in, float *s, float *rinv, float *mu_hat, float *pX,
+                         float *pW, double *scalars, aweq_dev_status *st, void *stream)
+{
+    if (!xmin || !xmax || !xmean || !wmin || !wmax || !s || !rinv || !mu_hat) return AWEQ_ERR_NULL;
+    if (C_in <= 0 || C_in > (1ll << 20)) return AWEQ_ERR_SHAPE;
+    return run_factors(xmin, xmax, xmean, wmin, wmax, C_in, s, rinv, mu_hat, pX, pW, scalars, st,
+                       (cudaStream_t)stream);
+}
+
+aweq_status aweq_equalize_quantize(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ldw,
+                                   const float *s, const float *mu_hat, int bits, aweq_gran gran, int group,
+                                   unsigned char *codes, float *step, int *zp, float *epsmu, void *ws,
+                                   size_t ws_bytes, aweq_dev_status *st, void *stream)
+{
+    aweq_status rc = check_matrix(W, dt, C_out, C_in, ldw, false);
+    if (rc != AWEQ_OK) return rc;
+    rc = check_quant(bits, gran, group, C_in);
+    if (rc != AWEQ_OK) return rc;
+    if (!codes || !step || !zp) return AWEQ_ERR_NULL;
+    if (!aligned(codes, 16) || (s && !aligned(s, 16)) || (mu_hat && !aligned(mu_hat, 16))) return AWEQ_ERR_ALIGN;
+    rc = check_ws(ws, ws_bytes, eq_ws_bytes(C_out, C_in, gran));
+    if (rc != AWEQ_OK) return rc;
+    cudaStream_t cs = (cudaStream_t)stream;
+    if (gran == AWEQ_PER_ROW) {
+        if (!rowquant_supported(C_out, C_in)) return AWEQ_ERR_SHAPE;
+        return run_rowquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, codes, step, zp, epsmu, st, cs);
+    }
+    if (gran == AWEQ_PER_GROUP)
+        return run_warpquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, group, nullptr, codes, step, zp, epsmu,
+                             st, cs);
+    // per tensor: column extremes of W -> extremes of diag(s) W -> static-range quantiser
+    char *base = reinterpret_cast<char *>(ws);
+    float *cmin = reinterpret_cast<float *>(base);
+    float *cmax = cmin + C_in;
+    float *lo_hi = reinterpret_cast<float *>(base + round256((size_t)C_in * 8));
+    void *ws2 = base + round256((size_t)C_in * 8) + 256;
+    rc = run_wrange(W, dt, C_out, C_in, ldw, cmin, cmax, 0, ws2, st, cs);
+    if (rc != AWEQ_OK) return rc;
+    rc = run_scaled_tensor_range(cmin, cmax, s, C_in, lo_hi, cs);
+    if (rc != AWEQ_OK) return rc;
+    return run_warpquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, 0, lo_hi, codes, step, zp, epsmu, st, cs);
+}
+
+aweq_status aweq_bias_correct(const float *epsmu, const void *W, aweq_dtype dt, const float *s,
+                              const unsigned char *codes, const float *step, const int *zp, const float *mu_hat,
+                              long long C_out, long long C_in, long long ldw, int bits, aweq_gran gran, int group,
+                              const void *bias_in, void *bias_out, float *bias_out_f32, aweq_dtype bias_dt,
+                              aweq_dev_status *st, void *stream)
+{
+    (void)st;
+    if (C_out <= 0) return AWEQ_ERR_SHAPE;
+    if (!bias_out && !bias_out_f32) return AWEQ_ERR_NULL;
+    if (bias_dt != AWEQ_F16 && bias_dt != AWEQ_BF16) return AWEQ_ERR_DTYPE;
+    if (epsmu) return run_bias_apply(epsmu, bias_in, bias_out, bias_out_f32, bias_dt, C_out, (cudaStream_t)stream);
+    aweq_status rc = check_matrix(W, dt, C_out, C_in, ldw, false);
+    if (rc != AWEQ_OK) return rc;
+    rc = check_quant(bits, gran, group, C_in);
+    if (rc != AWEQ_OK) return rc;
+    if (!codes || !step || !zp || !mu_hat) return AWEQ_ERR_NULL;
+    return run_bias_gemv(W, dt, C_out, C_in, ldw, s, codes, step, zp, mu_hat, bits, gran, group, bias_in, bias_out,
+                         bias_out_f32, bias_dt, (cudaStream_t)stream);
+}
+
+aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long C_in, long long ldx,
+                           const float *rinv, int bits, aweq_gran gran, const float *tensor_lo_hi,
+                           unsigned char *Xq, float *step, int *zp, aweq_dev_status *st, void *stream)
+{
+    aweq_status rc = check_matrix(X, dt, N, C_in, ldx, false);
+    if (rc != AWEQ_OK) return rc;
+    if (bits < 2 || bits > 8) return AWEQ_ERR_BITS;
+    if (!Xq || !step || !zp) return AWEQ_ERR_NULL;
+    if (!aligned(Xq, 16) || (rinv && !aligned(rinv, 16))) return AWEQ_ERR_ALIGN;
+    cudaStream_t cs = (cudaStream_t)stream;
+    if (gran == AWEQ_PER_ROW) {
+        if (!rowquant_supported(N, C_in)) return AWEQ_ERR_SHAPE;
+        return run_rowquant(X, dt, N, C_in, ldx, rinv, nullptr, bits, false, Xq, step, zp, nullptr, st, cs);
+    }
+    if (gran == AWEQ_PER_TENSOR) {
+        if (!tensor_lo_hi) return AWEQ_ERR_NULL;
+        return run_warpquant(X, dt, N, C_in, ldx, rinv, nullptr, bits, false, 0, tensor_lo_hi, Xq, step, zp, nullptr,
+                             st, cs);
+    }
+    return AWEQ_ERR_UNSUPPORTED;
+}
+
+// ------------------------------------------------------------------ layer pass
+// workspace layout: [column-reduction scratch | scratch of step 4]
+static size_t layer_ws_parts(const aweq_layer_args *a, size_t *col_part)
+{
+    size_t col = colreduce_ws_bytes(a->N, a->C_in);
+    size_t eq = 0;
+    for (int i = 0; i < a->n_w; ++i) {
+        size_t c = colreduce_ws_bytes(a->C_out[i], a->C_in);
+        if (c > col) col = c;
+        size_t e = eq_ws_bytes(a->C_out[i], a->C_in, a->gran);
+        if (e > eq) eq = e;
+    }
+    col = round256(col);
+    if (col_part) *col_part = col;
+    return col + round256(eq);
+}
+
+size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args)
+{
+    if (!args || args->n_w <= 0 || !args->C_out || args->C_in <= 0) return 0;
+    return layer_ws_parts(args, nullptr);
+}
+
+aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes, aweq_dev_status *st, void *stream)
+{
+    if (!a) return AWEQ_ERR_NULL;
+    if (a->n_w <= 0 || !a->W || !a->C_out || !a->ldw || !a->codes || !a->step || !a->zp) return AWEQ_ERR_NULL;
+    if (!a->xmin || !a->xmax || !a->xmean || !a->wmin || !a->wmax || !a->s || !a->rinv || !a->mu_hat)
+        return AWEQ_ERR_NULL;
+    aweq_status rc = check_matrix(a->X, a->dt, a->N, a->C_in, a->ldx, false);
+    if (rc != AWEQ_OK) return rc;
+    rc = check_quant(a->bits, a->gran, a->group, a->C_in);
+    if (rc != AWEQ_OK) return rc;
+    for (int i = 0; i < a->n_w; ++i) {
+        rc = check_matrix(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], false);
+        if (rc != AWEQ_OK) return rc;
+        if (!a->codes[i] || !a->step[i] || !a->zp[i]) return AWEQ_ERR_NULL;
+    }
+    const bool bc = !(a->flags & AWEQ_FLAG_NO_BIAS_CORRECT);
+    if (bc && (!a->epsmu || (!a->bias_out && !a->bias_out_f32))) return AWEQ_ERR_NULL;
+    for (int i = 0; bc && i < a->n_w; ++i) {
+        if (!a->epsmu[i]) return AWEQ_ERR_NULL;
+        if (!(a->bias_out && a->bias_out[i]) && !(a->bias_out_f32 && a->bias_out_f32[i])) return AWEQ_ERR_NULL;
+    }
+    if (a->Xq && (!a->act_step || !a->act_zp)) return AWEQ_ERR_NULL;
+    size_t col_part = 0;
+    const size_t need = layer_ws_parts(a, &col_part);
+    rc = check_ws(ws, ws_bytes, need);
+    if (rc != AWEQ_OK) return rc;
+    char *base = reinterpret_cast<char *>(ws);
+    void *ws_col = base;
+    void *ws_eq = base + col_part;
+    const size_t ws_eq_bytes = need - col_part;
+
+    // steps 1-2
+    rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
+                    col_part, st, stream);
+    if (rc != AWEQ_OK) return rc;
+    for (int i = 0; i < a->n_w; ++i) {
+        rc = aweq_wrange(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], a->wmin, a->wmax, i > 0, ws_col, col_part,
+                         st, stream);
+        if (rc != AWEQ_OK) return rc;
+    }
+    // step 3
+    rc = aweq_factors(a->xmin, a->xmax, a->xmean, a->wmin, a->wmax, a->C_in, a->s, a->rinv, a->mu_hat, a->pX, a->pW,
+                      a->scalars, st, stream);
+    if (rc != AWEQ_OK) return rc;
+    const bool eq = !(a->flags & AWEQ_FLAG_NO_EQUALIZE);
+    // without equalisation the layer sees x itself, so E[x^] = E[x]
+    const float *s_used = eq ? a->s : nullptr;
+    const float *rinv_used = eq ? a->rinv : nullptr;
+    const float *mu_used = eq ? a->mu_hat : a->xmean;
+    // steps 4-5 per matrix
+    for (int i = 0; i < a->n_w; ++i) {
+        float *em = bc ? a->epsmu[i] : nullptr;
+        rc = aweq_equalize_quantize(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], s_used, bc ? mu_used : nullptr,
+                                    a->bits, a->gran, a->group, a->codes[i], a->step[i], a->zp[i], em, ws_eq,
+                                    ws_eq_bytes, st, stream);
+        if (rc != AWEQ_OK) return rc;
+        if (bc) {
+            const void *bin = a->bias_in ? a->bias_in[i] : nullptr;
+            void *bout = a->bias_out ? a->bias_out[i] : nullptr;
+            float *bout32 = a->bias_out_f32 ? a->bias_out_f32[i] : nullptr;
+            rc = aweq_bias_correct(em, nullptr, a->dt, nullptr, nullptr, nullptr, nullptr, nullptr, a->C_out[i],
+                                   a->C_in, a->ldw[i], a->bits, a->gran, a->group, bin, bout, bout32, a->dt, st,
+                                   stream);
+            if (rc != AWEQ_OK) return rc;
+        }
+    }
+    // step 6
+    if (a->Xq) {
+        rc = aweq_quant_act(a->X, a->dt, a->N, a->C_in, a->ldx, rinv_used, a->act_bits ? a->act_bits : 8, AWEQ_PER_ROW,
+                            nullptr, a->Xq, a->act_step, a->act_zp, st, stream);
+        if (rc != AWEQ_OK) return rc;
+    }
+    return AWEQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,335 @@
+// Steps 1 and 2: per-column min / max (/ sum) of a row-major 16-bit matrix.
+//
+// Step 1 (aweq_stats) reduces the calibration inputs X[N x C_in] to per-channel
+// min, max and mean (Section 3.2: channel range = max - min; Section 3.3: E[x]
+// is gathered in the same sweep).  Step 2 (aweq_wrange) reduces W[C_out x C_in]
+// to per-input-channel min and max.  Both are one streaming read of the matrix
+// and are bound by HBM bandwidth.
+//
+// Layout of the work: the columns are cut into slabs of at most 256 16-byte
+// vectors (2048 columns) and the rows into splits; one CTA owns one
+// (slab, split) pair, so a thread owns one vector column for its whole life and
+// keeps that column's eight running minima, maxima and sums in registers.
+// A producer warp streams the CTA's rows through a ring of shared-memory
+// stages with 1-D bulk copies (TMA, completion on mbarriers); eight consumer
+// warps read the stages back conflict-free (consecutive lanes, consecutive
+// 16-byte vectors).  min / max stay in packed 16-bit arithmetic (exact); sums
+// are binary32 over the eight rows of one stage and are folded into binary64
+// after every stage.  Each CTA writes one partial per column; a second small
+// kernel reduces the partials over the splits in a fixed order, so results are
+// bit-reproducible from run to run.
+#include "common.cuh"
+
+namespace aweq {
+
+constexpr int kColThreads = 256;        // consumer threads = vectors per slab
+constexpr int kColRows = 8;             // rows per stage
+constexpr int kColStages = 3;
+constexpr int kColTargetCtas = 2 * kSmCount;
+
+struct ColPlan {
+    int nvec, nslab, slab_w, nsplit;
+    long long rows_per_split;
+};
+
+ColPlan plan_colreduce(long long rows, long long cols)
+{
+    ColPlan p;
+    p.nvec = (int)(cols / 8);
+    p.nslab = (p.nvec + kColThreads - 1) / kColThreads;
+    p.slab_w = (p.nvec + p.nslab - 1) / p.nslab;
+    int nsplit = kColTargetCtas / p.nslab;
+    if (nsplit < 1) nsplit = 1;
+    long long max_split = (rows + kColRows - 1) / kColRows;
+    if (max_split < 1) max_split = 1;
+    if (nsplit > max_split) nsplit = (int)max_split;
+    long long rps = (rows + nsplit - 1) / nsplit;
+    rps = (rps + kColRows - 1) / kColRows * kColRows;
+    if (rps < kColRows) rps = kColRows;
+    p.rows_per_split = rps;
+    p.nsplit = (int)((rows + rps - 1) / rps);
+    if (p.nsplit < 1) p.nsplit = 1;
+    return p;
+}
+
+size_t colreduce_ws_bytes(long long rows, long long cols)
+{
+    ColPlan p = plan_colreduce(rows, cols);
+    // pmin, pmax: float[nsplit][cols]; psum: double[nsplit][cols]
+    return (size_t)p.nsplit * (size_t)cols * 16 + 256;
+}
+
+struct ColSmem {
+    uint64_t full[kColStages];
+    uint64_t empty[kColStages];
+    int abort_flag;
+};
+
+template <class D, bool WITH_SUM>
+__global__ void __launch_bounds__(kColThreads + 32, 2)
+colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, int nvec, int nslab, int slab_w,
+                 long long rows_per_split, long long cols, float *__restrict__ pmin, float *__restrict__ pmax,
+                 double *__restrict__ psum, aweq_dev_status *st)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    ColSmem *sm = reinterpret_cast<ColSmem *>(smem_raw);
+    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw + 128);
+
+    const int slab = blockIdx.x % nslab;
+    const int split = blockIdx.x / nslab;
+    const int v0 = slab * slab_w;
+    const int w = min(slab_w, nvec - v0);                 // vectors in this slab (> 0)
+    const long long r0 = (long long)split * rows_per_split;
+    const long long r1 = min(nrows, r0 + rows_per_split);
+    const int ntiles = r1 > r0 ? (int)((r1 - r0 + kColRows - 1) / kColRows) : 0;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int active_warps = (w + 31) / 32;
+    const size_t stage_vecs = (size_t)kColRows * slab_w;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kColStages; ++s) {
+            mbar_init(&sm->full[s], 1);
+            mbar_init(&sm->empty[s], active_warps);
+        }
+        sm->abort_flag = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+
+    if (warp == kColThreads / 32) {
+        // ---------------- producer warp
+        const bool contiguous = (nslab == 1) && (ld == cols);
+        bool ok = true;
+        for (int t = 0; t < ntiles && ok; ++t) {
+            const int s = t % kColStages;
+            const uint32_t use = t / kColStages;
+            if (use > 0) {
+                ok = mbar_wait(&sm->empty[s], (use - 1) & 1);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+            }
+            const long long row0 = r0 + (long long)t * kColRows;
+            const int rows = (int)min((long long)kColRows, r1 - row0);
+            uint4 *dst = stage_base + (size_t)s * stage_vecs;
+            if (lane == 0) mbar_arrive_expect_tx(&sm->full[s], (uint32_t)rows * w * 16u);
+            __syncwarp();
+            if (contiguous) {
+                if (lane == 0) bulk_g2s(dst, X + row0 * ld, (uint32_t)rows * w * 16u, &sm->full[s]);
+            } else if (lane < rows) {
+                bulk_g2s(dst + (size_t)lane * w, X + (row0 + lane) * ld + (long long)v0 * 8, (uint32_t)w * 16u,
+                         &sm->full[s]);
+            }
+        }
+        if (!ok && lane == 0) {
+            atomicExch(&sm->abort_flag, 1);
+            if (st) atomicAdd(&st->wait_timeout, 1ull);
+        }
+    } else if (warp < active_warps) {
+        // ---------------- consumer warps: thread <-> one vector column
+        const int t_col = threadIdx.x;
+        const bool mine = t_col < w;
+        typename D::T2 mn[4], mx[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            mn[k] = D::from_bits(D::pos_inf2());
+            mx[k] = D::from_bits(D::neg_inf2());
+        }
+        double acc64[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc64[k] = 0.0;
+        bool ok = true;
+        for (int t = 0; t < ntiles; ++t) {
+            const int s = t % kColStages;
+            const uint32_t use = t / kColStages;
+            ok = mbar_wait(&sm->full[s], use & 1);
+            if (!ok || *reinterpret_cast<volatile int *>(&sm->abort_flag)) { ok = false; break; }
+            const long long row0 = r0 + (long long)t * kColRows;
+            const int rows = (int)min((long long)kColRows, r1 - row0);
+            const uint4 *src = stage_base + (size_t)s * stage_vecs + t_col;
+            if (mine) {
+                float acc32[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) acc32[k] = 0.0f;
+                if (rows == kColRows) {
+                    uint4 v[kColRows];
+#pragma unroll
+                    for (int r = 0; r < kColRows; ++r) v[r] = src[(size_t)r * w];
+#pragma unroll
+                    for (int r = 0; r < kColRows; ++r) {
+                        const uint32_t u[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            typename D::T2 h = D::from_bits(u[k]);
+                            mn[k] = __hmin2(mn[k], h);
+                            mx[k] = __hmax2(mx[k], h);
+                            if (WITH_SUM) {
+                                float2 f = D::to_float2(h);
+                                acc32[2 * k] += f.x;
+                                acc32[2 * k + 1] += f.y;
+                            }
+                        }
+                    }
+                } else {
+                    for (int r = 0; r < rows; ++r) {
+                        uint4 vr = src[(size_t)r * w];
+                        const uint32_t u[4] = {vr.x, vr.y, vr.z, vr.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            typename D::T2 h = D::from_bits(u[k]);
+                            mn[k] = __hmin2(mn[k], h);
+                            mx[k] = __hmax2(mx[k], h);
+                            if (WITH_SUM) {
+                                float2 f = D::to_float2(h);
+                                acc32[2 * k] += f.x;
+                                acc32[2 * k + 1] += f.y;
+                            }
+                        }
+                    }
+                }
+                if (WITH_SUM) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc64[k] += (double)acc32[k];
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm->empty[s]);
+        }
+        if (!ok && lane == 0) {
+            atomicExch(&sm->abort_flag, 1);
+            if (st) atomicAdd(&st->wait_timeout, 1ull);
+        }
+        if (mine) {
+            const size_t o = (size_t)split * (size_t)cols + (size_t)(v0 + t_col) * 8;
+            float lo[8], hi[8];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float2 a = D::to_float2(mn[k]), b = D::to_float2(mx[k]);
+                lo[2 * k] = a.x; lo[2 * k + 1] = a.y;
+                hi[2 * k] = b.x; hi[2 * k + 1] = b.y;
+            }
+            float4 *qlo = reinterpret_cast<float4 *>(pmin + o), *qhi = reinterpret_cast<float4 *>(pmax + o);
+            qlo[0] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+            qlo[1] = make_float4(lo[4], lo[5], lo[6], lo[7]);
+            qhi[0] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+            qhi[1] = make_float4(hi[4], hi[5], hi[6], hi[7]);
+            if (WITH_SUM) {
+                double2 *qs = reinterpret_cast<double2 *>(psum + o);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) qs[k] = make_double2(acc64[2 * k], acc64[2 * k + 1]);
+            }
+        }
+    }
+    // Every copy that was issued has been waited for by the consumers unless a
+    // wait timed out; in that case give outstanding copies a bounded chance to
+    // land before the shared memory is released.
+    __syncthreads();
+    if (threadIdx.x == 0 && sm->abort_flag) {
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 1000000ull) { }
+    }
+}
+
+// Reduce the per-split partials in split order; merge with the running state
+// when accumulating.  One thread per column.
+template <bool WITH_SUM>
+__global__ void colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restrict__ pmax,
+                                          const double *__restrict__ psum, int nsplit, long long cols,
+                                          long long nrows, float *omin, float *omax, float *omean, double *osum,
+                                          const long long *count, int accumulate, aweq_dev_status *st)
+{
+    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= cols) return;
+    float lo = INFINITY, hi = -INFINITY;
+    double sum = 0.0;
+    for (int k = 0; k < nsplit; ++k) {
+        lo = fminf(lo, pmin[(size_t)k * cols + j]);
+        hi = fmaxf(hi, pmax[(size_t)k * cols + j]);
+        if (WITH_SUM) sum += psum[(size_t)k * cols + j];
+    }
+    long long total = nrows;
+    if (accumulate) {
+        lo = fminf(lo, omin[j]);
+        hi = fmaxf(hi, omax[j]);
+        if (WITH_SUM) {
+            sum += osum[j];
+            total += count[0];
+        }
+    }
+    omin[j] = lo;
+    omax[j] = hi;
+    if (WITH_SUM) {
+        if (osum) osum[j] = sum;
+        omean[j] = total > 0 ? (float)(sum / (double)total) : 0.0f;
+    }
+    if (st) {
+        bool bad = (nrows > 0 || accumulate) && !(isfinite(lo) && isfinite(hi) && isfinite(sum));
+        if (bad) atomicAdd(&st->nonfinite, 1ull);
+    }
+}
+
+__global__ void bump_count_kernel(long long *count, long long nrows, int accumulate)
+{
+    count[0] = (accumulate ? count[0] : 0) + nrows;
+}
+
+static size_t colreduce_smem_bytes(int slab_w)
+{
+    return 128 + (size_t)kColStages * kColRows * slab_w * 16;
+}
+
+template <class D, bool WITH_SUM>
+static aweq_status launch_colreduce(const void *X, long long rows, long long cols, long long ld, float *omin,
+                                    float *omax, float *omean, double *osum, long long *count, int accumulate,
+                                    void *ws, aweq_dev_status *st, cudaStream_t stream)
+{
+    ColPlan p = plan_colreduce(rows, cols);
+    char *base = reinterpret_cast<char *>(ws);
+    float *pmin = reinterpret_cast<float *>(base);
+    float *pmax = pmin + (size_t)p.nsplit * cols;
+    double *psum = reinterpret_cast<double *>(base + (size_t)p.nsplit * cols * 8);
+    const size_t smem = colreduce_smem_bytes(p.slab_w);
+    auto kern = colreduce_kernel<D, WITH_SUM>;
+    static thread_local bool attr_set = false;
+    if (!attr_set) {
+        AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)colreduce_smem_bytes(kColThreads)));
+        attr_set = true;
+    }
+    int nsplit_eff = rows > 0 ? p.nsplit : 0;
+    if (rows > 0) {
+        kern<<<p.nslab * p.nsplit, kColThreads + 32, smem, stream>>>(
+            reinterpret_cast<const uint16_t *>(X), rows, ld, p.nvec, p.nslab, p.slab_w, p.rows_per_split, cols, pmin,
+            pmax, psum, st);
+        AWEQ_LAUNCH_CHECK();
+    }
+    const int ft = 256;
+    colreduce_finalize_kernel<WITH_SUM><<<(unsigned)((cols + ft - 1) / ft), ft, 0, stream>>>(
+        pmin, pmax, psum, nsplit_eff, cols, rows, omin, omax, omean, osum, count, accumulate, st);
+    AWEQ_LAUNCH_CHECK();
+    if (WITH_SUM && count) {
+        bump_count_kernel<<<1, 1, 0, stream>>>(count, rows, accumulate);
+        AWEQ_LAUNCH_CHECK();
+    }
+    return AWEQ_OK;
+}
+
+aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin, float *xmax,
+                      float *xmean, double *xsum, long long *count, int accumulate, void *ws, aweq_dev_status *st,
+                      cudaStream_t stream)
+{
+    if (dt == AWEQ_F16)
+        return launch_colreduce<F16, true>(X, N, C, ld, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
+    return launch_colreduce<BF16, true>(X, N, C, ld, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
+}
+
+aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld, float *wmin,
+                       float *wmax, int accumulate, void *ws, aweq_dev_status *st, cudaStream_t stream)
+{
+    if (dt == AWEQ_F16)
+        return launch_colreduce<F16, false>(W, C_out, C_in, ld, wmin, wmax, nullptr, nullptr, nullptr, accumulate, ws,
+                                            st, stream);
+    return launch_colreduce<BF16, false>(W, C_out, C_in, ld, wmin, wmax, nullptr, nullptr, nullptr, accumulate, ws, st,
+                                         stream);
+}
+
+}  // namespace aweq

@@ -1,0 +1,206 @@
+// Shared device helpers of the AWEQ kernels (sm_100a only): 16-bit type
+// traits, mbarrier / bulk-copy (TMA) wrappers with bounded waits, warp
+// reductions and the scalar pieces of the Eq. 1-2 quantiser.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/aweq.h"
+
+namespace aweq {
+
+constexpr int kSmCount = 148;              // B200
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a wait longer than 2 s is reported, not spun on
+
+// ------------------------------------------------------------------ host side
+void note_launch();                        // bumps the launch counter
+aweq_status cuda_failed(cudaError_t e);    // records the error text, returns AWEQ_ERR_CUDA
+
+#define AWEQ_CUDA_OK(expr)                                   \
+    do {                                                     \
+        cudaError_t e__ = (expr);                            \
+        if (e__ != cudaSuccess) return ::aweq::cuda_failed(e__); \
+    } while (0)
+
+#define AWEQ_LAUNCH_CHECK()                                  \
+    do {                                                     \
+        ::aweq::note_launch();                               \
+        cudaError_t e__ = cudaGetLastError();                \
+        if (e__ != cudaSuccess) return ::aweq::cuda_failed(e__); \
+    } while (0)
+
+// ------------------------------------------------------------------ 16-bit traits
+struct F16 {
+    using T2 = __half2;
+    static __device__ __forceinline__ T2 from_bits(uint32_t u) { return *reinterpret_cast<T2 *>(&u); }
+    static __device__ __forceinline__ uint32_t pos_inf2() { return 0x7C007C00u; }
+    static __device__ __forceinline__ uint32_t neg_inf2() { return 0xFC00FC00u; }
+    static __device__ __forceinline__ float2 to_float2(T2 v) { return __half22float2(v); }
+    static __device__ __forceinline__ float one(uint16_t b) { return __half2float(__ushort_as_half(b)); }
+    static __device__ __forceinline__ uint16_t encode(float f) { return __half_as_ushort(__float2half_rn(f)); }
+};
+struct BF16 {
+    using T2 = __nv_bfloat162;
+    static __device__ __forceinline__ T2 from_bits(uint32_t u) { return *reinterpret_cast<T2 *>(&u); }
+    static __device__ __forceinline__ uint32_t pos_inf2() { return 0x7F807F80u; }
+    static __device__ __forceinline__ uint32_t neg_inf2() { return 0xFF80FF80u; }
+    static __device__ __forceinline__ float2 to_float2(T2 v)
+    {
+        uint32_t u = *reinterpret_cast<uint32_t *>(&v);    // bf16 is the upper half of a binary32
+        return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+    }
+    static __device__ __forceinline__ float one(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+    static __device__ __forceinline__ uint16_t encode(float f) { return __bfloat16_as_ushort(__float2bfloat16_rn(f)); }
+};
+
+// widen the 8 elements of a 16-byte vector
+template <class D>
+__device__ __forceinline__ void widen8(const uint4 &v, float (&f)[8])
+{
+    float2 a = D::to_float2(D::from_bits(v.x)), b = D::to_float2(D::from_bits(v.y));
+    float2 c = D::to_float2(D::from_bits(v.z)), d = D::to_float2(D::from_bits(v.w));
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y; f[4] = c.x; f[5] = c.y; f[6] = d.x; f[7] = d.y;
+}
+
+// ------------------------------------------------------------------ loads
+__device__ __forceinline__ uint4 ldg_stream(const void *p)   // read-once data: bypass L1 allocation
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float4 ldg_f4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ void load8(const float *p, float (&f)[8])
+{
+    float4 a = ldg_f4(p), b = ldg_f4(p + 4);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+}
+
+// ------------------------------------------------------------------ mbarrier + bulk copy
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for a phase of the barrier; gives up after kWaitLimitNs and returns false.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > kWaitLimitNs) return false;
+    }
+}
+// 1-D bulk copy global -> this CTA's shared memory, completion on an mbarrier.
+// Both addresses 16-byte aligned, bytes a multiple of 16.  No multicast.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// barrier over `threads` threads that also ANDs a predicate (all arrive, all get the same answer)
+__device__ __forceinline__ bool named_bar_and(int id, int threads, bool pred)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %3, 0;\n\t"
+        "bar.red.and.pred p, %1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r) : "r"(id), "r"(threads), "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
+// ------------------------------------------------------------------ warp reductions
+__device__ __forceinline__ float redux_min(float v, uint32_t mask)
+{
+    float r;
+    asm volatile("redux.sync.min.f32 %0, %1, %2;" : "=f"(r) : "f"(v), "r"(mask));
+    return r;
+}
+__device__ __forceinline__ float redux_max(float v, uint32_t mask)
+{
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, %2;" : "=f"(r) : "f"(v), "r"(mask));
+    return r;
+}
+__device__ __forceinline__ float warp_sum(float v)      // fixed butterfly order: reproducible
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ------------------------------------------------------------------ Eq. 1-2, scalar part
+// (Step, 1/Step, Z) of a vector with extremes lo, hi; all IEEE binary32, no FMA.
+struct QParams {
+    float step, inv;
+    int zp;
+    bool fast;      // |Z| small enough for the add-magic rounding path
+};
+__device__ __forceinline__ QParams make_qparams(float lo, float hi, int qmax)
+{
+    QParams p;
+    float st = __fdiv_rn(__fsub_rn(hi, lo), (float)qmax);
+    if (!(st > 0.0f)) st = (lo != 0.0f) ? fabsf(lo) : 1.0f;      // constant vector
+    p.step = st;
+    p.inv = __fdiv_rn(1.0f, st);
+    float z = __fmul_rn(lo, p.inv);
+    int zi;
+    asm("cvt.rni.sat.s32.f32 %0, %1;" : "=r"(zi) : "f"(-z));    // saturating; NaN -> 0
+    p.zp = zi;
+    p.fast = (zi > -(1 << 21)) && (zi < (1 << 21)) && (fabsf(p.inv) <= 3.0e38f) && (fabsf(z) < 4.0e6f);
+    return p;
+}
+// exact reference form of one code: clamp(rint(fl(v*inv)) + Z, 0, qmax) with saturating int32
+__device__ __forceinline__ int code_generic(float v, float inv, int zp, int qmax)
+{
+    int t, q;
+    asm("cvt.rni.sat.s32.f32 %0, %1;" : "=r"(t) : "f"(__fmul_rn(v, inv)));
+    asm("add.sat.s32 %0, %1, %2;" : "=r"(q) : "r"(t), "r"(zp));
+    return min(max(q, 0), qmax);
+}
+constexpr float kMagic = 12582912.0f;            // 1.5 * 2^23: adding it rounds to an integer, ties to even
+constexpr int kMagicBits = 0x4B400000;
+
+}  // namespace aweq

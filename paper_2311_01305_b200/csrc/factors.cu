@@ -1,0 +1,144 @@
+// Step 3: equalisation factors and the diagnostics of Eq. 4-8.
+//
+//   r^X_j = xmax_j - xmin_j, r^W_j = wmax_j - wmin_j            (Section 3.2)
+//   s_j   = (1 / r^W_j) sqrt(r^X_j r^W_j)                        (Eq. 10, binary64, one rounding)
+//   rinv_j = 1 / s_j,  mu_hat_j = xmean_j * rinv_j               (E[x^], Eq. 15)
+//   p^X_j = r^X_j / R^X, p^W_j = r^W_j / R^W                     (Eq. 4)
+//   objective sum_j p^X_j p^W_j before and after equalisation    (Eq. 5)
+//   max_j r^X_j/s_j * max_k s_k r^W_k before and after           (Eq. 8)
+// C_in values: one CTA, fixed reduction order, negligible time.
+#include "common.cuh"
+
+namespace aweq {
+
+constexpr int kFacThreads = 1024;
+
+struct FacRed {
+    float xlo, xhi, wlo, whi, exlo, exhi, ewlo, ewhi, mrx, mrw, merx, merw;
+};
+
+__device__ __forceinline__ void fac_merge(FacRed &a, const FacRed &b)
+{
+    a.xlo = fminf(a.xlo, b.xlo); a.xhi = fmaxf(a.xhi, b.xhi);
+    a.wlo = fminf(a.wlo, b.wlo); a.whi = fmaxf(a.whi, b.whi);
+    a.exlo = fminf(a.exlo, b.exlo); a.exhi = fmaxf(a.exhi, b.exhi);
+    a.ewlo = fminf(a.ewlo, b.ewlo); a.ewhi = fmaxf(a.ewhi, b.ewhi);
+    a.mrx = fmaxf(a.mrx, b.mrx); a.mrw = fmaxf(a.mrw, b.mrw);
+    a.merx = fmaxf(a.merx, b.merx); a.merw = fmaxf(a.merw, b.merw);
+}
+
+__global__ void __launch_bounds__(kFacThreads)
+factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, const float *__restrict__ xmean,
+               const float *__restrict__ wmin, const float *__restrict__ wmax, int C, float *__restrict__ s,
+               float *__restrict__ rinv, float *__restrict__ mu_hat, float *__restrict__ pX, float *__restrict__ pW,
+               double *__restrict__ scalars, aweq_dev_status *st)
+{
+    __shared__ FacRed red[kFacThreads / 32];
+    __shared__ FacRed total;
+    __shared__ double dsum[2][kFacThreads / 32];
+    __shared__ unsigned int dead_count;
+    if (threadIdx.x == 0) dead_count = 0;
+    __syncthreads();
+
+    FacRed a;
+    a.xlo = a.wlo = a.exlo = a.ewlo = INFINITY;
+    a.xhi = a.whi = a.exhi = a.ewhi = -INFINITY;
+    a.mrx = a.mrw = a.merx = a.merw = 0.0f;
+    unsigned int dead = 0;
+    for (int j = threadIdx.x; j < C; j += kFacThreads) {
+        const float lo = xmin[j], hi = xmax[j], wl = wmin[j], wh = wmax[j];
+        const float rx = __fsub_rn(hi, lo), rw = __fsub_rn(wh, wl);
+        float sj = 1.0f;
+        bool ok = isfinite(rx) && isfinite(rw) && rx > 0.0f && rw > 0.0f;
+        if (ok) {
+            // Eq. 10 as printed, in binary64, rounded once to binary32
+            sj = (float)__dmul_rn(__ddiv_rn(1.0, (double)rw), __dsqrt_rn(__dmul_rn((double)rx, (double)rw)));
+            if (!(isfinite(sj) && sj > 0.0f) || !isfinite(__fdiv_rn(1.0f, sj))) {
+                sj = 1.0f;
+                ok = false;
+            }
+        }
+        if (!ok) ++dead;
+        const float ri = __fdiv_rn(1.0f, sj);
+        s[j] = sj;
+        rinv[j] = ri;
+        mu_hat[j] = __fmul_rn(xmean[j], ri);
+        const float exl = __fmul_rn(lo, ri), exh = __fmul_rn(hi, ri);
+        const float ewl = __fmul_rn(wl, sj), ewh = __fmul_rn(wh, sj);
+        a.xlo = fminf(a.xlo, lo); a.xhi = fmaxf(a.xhi, hi);
+        a.wlo = fminf(a.wlo, wl); a.whi = fmaxf(a.whi, wh);
+        a.exlo = fminf(a.exlo, exl); a.exhi = fmaxf(a.exhi, exh);
+        a.ewlo = fminf(a.ewlo, ewl); a.ewhi = fmaxf(a.ewhi, ewh);
+        a.mrx = fmaxf(a.mrx, rx); a.mrw = fmaxf(a.mrw, rw);
+        a.merx = fmaxf(a.merx, exh - exl); a.merw = fmaxf(a.merw, ewh - ewl);
+    }
+    // block reduction of the twelve extremes
+    const uint32_t full = 0xffffffffu;
+    a.xlo = redux_min(a.xlo, full); a.xhi = redux_max(a.xhi, full);
+    a.wlo = redux_min(a.wlo, full); a.whi = redux_max(a.whi, full);
+    a.exlo = redux_min(a.exlo, full); a.exhi = redux_max(a.exhi, full);
+    a.ewlo = redux_min(a.ewlo, full); a.ewhi = redux_max(a.ewhi, full);
+    a.mrx = redux_max(a.mrx, full); a.mrw = redux_max(a.mrw, full);
+    a.merx = redux_max(a.merx, full); a.merw = redux_max(a.merw, full);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = a;
+    if (dead) atomicAdd(&dead_count, dead);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        FacRed t = red[0];
+        for (int k = 1; k < kFacThreads / 32; ++k) fac_merge(t, red[k]);
+        total = t;
+    }
+    __syncthreads();
+    const FacRed t = total;
+    const double RX = (double)t.xhi - (double)t.xlo, RW = (double)t.whi - (double)t.wlo;
+    const double EX = (double)t.exhi - (double)t.exlo, EW = (double)t.ewhi - (double)t.ewlo;
+
+    double o0 = 0.0, o1 = 0.0;
+    for (int j = threadIdx.x; j < C; j += kFacThreads) {
+        const double rx = (double)__fsub_rn(xmax[j], xmin[j]);
+        const double rw = (double)__fsub_rn(wmax[j], wmin[j]);
+        const float sj = s[j], ri = rinv[j];
+        const double erx = (double)__fmul_rn(xmax[j], ri) - (double)__fmul_rn(xmin[j], ri);
+        const double erw = (double)__fmul_rn(wmax[j], sj) - (double)__fmul_rn(wmin[j], sj);
+        if (pX) pX[j] = (float)(rx / RX);
+        if (pW) pW[j] = (float)(rw / RW);
+        o0 += (rx / RX) * (rw / RW);
+        o1 += (erx / EX) * (erw / EW);
+    }
+    if (scalars) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            o0 += __shfl_xor_sync(full, o0, o);
+            o1 += __shfl_xor_sync(full, o1, o);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            dsum[0][threadIdx.x >> 5] = o0;
+            dsum[1][threadIdx.x >> 5] = o1;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double b0 = 0.0, b1 = 0.0;
+            for (int k = 0; k < kFacThreads / 32; ++k) {
+                b0 += dsum[0][k];
+                b1 += dsum[1][k];
+            }
+            scalars[0] = RX; scalars[1] = RW; scalars[2] = EX; scalars[3] = EW;
+            scalars[4] = b0; scalars[5] = b1;
+            scalars[6] = (double)t.mrx * (double)t.mrw;
+            scalars[7] = (double)t.merx * (double)t.merw;
+        }
+    }
+    if (threadIdx.x == 0 && st && dead_count) atomicAdd(&st->zero_range, (unsigned long long)dead_count);
+}
+
+aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean, const float *wmin,
+                        const float *wmax, long long C, float *s, float *rinv, float *mu_hat, float *pX, float *pW,
+                        double *scalars, aweq_dev_status *st, cudaStream_t stream)
+{
+    factors_kernel<<<1, kFacThreads, 0, stream>>>(xmin, xmax, xmean, wmin, wmax, (int)C, s, rinv, mu_hat, pX, pW,
+                                                  scalars, st);
+    AWEQ_LAUNCH_CHECK();
+    return AWEQ_OK;
+}
+
+}  // namespace aweq

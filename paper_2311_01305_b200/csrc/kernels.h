@@ -1,0 +1,37 @@
+// Internal launch functions behind the C ABI (one per kernel family).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "../../include/aweq.h"
+
+namespace aweq {
+
+size_t colreduce_ws_bytes(long long rows, long long cols);
+
+aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin, float *xmax,
+                      float *xmean, double *xsum, long long *count, int accumulate, void *ws, aweq_dev_status *st,
+                      cudaStream_t stream);
+aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld, float *wmin,
+                       float *wmax, int accumulate, void *ws, aweq_dev_status *st, cudaStream_t stream);
+aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean, const float *wmin,
+                        const float *wmax, long long C, float *s, float *rinv, float *mu_hat, float *pX, float *pW,
+                        double *scalars, aweq_dev_status *st, cudaStream_t stream);
+bool rowquant_supported(long long nrows, long long cols);
+aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
+                         const float *scale, const float *mu, int bits, bool weights, unsigned char *out,
+                         float *step, int *zp, float *epsmu, aweq_dev_status *st, cudaStream_t stream);
+aweq_status run_warpquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
+                          const float *scale, const float *mu, int bits, bool weights, int group,
+                          const float *lo_hi, unsigned char *out, float *step, int *zp, float *epsmu,
+                          aweq_dev_status *st, cudaStream_t stream);
+aweq_status run_scaled_tensor_range(const float *cmin, const float *cmax, const float *scale, long long C,
+                                    float *lo_hi, cudaStream_t stream);
+aweq_status run_bias_apply(const float *epsmu, const void *bias_in, void *bias_out, float *bias_out_f32,
+                           aweq_dtype bias_dt, long long C_out, cudaStream_t stream);
+aweq_status run_bias_gemv(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld,
+                          const float *s, const unsigned char *codes, const float *step, const int *zp,
+                          const float *mu_hat, int bits, int gran, int group, const void *bias_in, void *bias_out,
+                          float *bias_out_f32, aweq_dtype bias_dt, cudaStream_t stream);
+
+}  // namespace aweq
