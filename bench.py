@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the AWEQ per-linear-layer calibration pass (arXiv 2311.01305).
+
+    python bench.py --gpus N --steps K --warmup W [--workload NAME] [--bits B]
+    python bench.py --impl reference ...       # the CPU oracle on a bounded sample
+
+One step is one calibration pass over a whole decoder layer of the workload:
+for every distinct layer input, statistics of X, column ranges of the weight
+matrices it feeds, equalisation factors, the fused rescale + quantise + pack of
+every matrix with its bias correction and, for W8A8 workloads, the per-token
+8-bit quantisation of the equalised input.  Inputs are seeded synthetic tensors
+with the shapes and value distributions of the named model layer; they are
+resident in HBM before the timed region and are far larger than L2.
+
+The metric is layer-pass HBM GB/s: algorithmic bytes of the pass divided by its
+device time (CUDA events, max over ranks).  With N > 1 every rank calibrates
+its own token shard of the same layer (weak scaling, no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2311_01305_b200 import synth  # noqa: E402
+
+DEFAULT_WORKLOAD = "llama7b_layer_w4w3_g128"
+NORTH_STAR_PEAK_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def generate(wl: synth.Workload, device, rank: int):
+    X, W = {}, {}
+    for i, inp in enumerate(wl.inputs):
+        X[inp.name] = synth.make_activations(inp, wl.dtype, synth.tensor_seed(wl.seed, rank, i), device)
+    for i, lin in enumerate(wl.linears):
+        W[lin.name] = synth.make_weight(lin, wl.dtype, synth.tensor_seed(wl.seed, 0, 100 + i), device)
+    return X, W
+
+
+def oracle_pass(wl: synth.Workload, bits: int, Xb, Wb):
+    """One layer pass through the CPU oracle on raw-bit arrays (the reference arm
+    and the cpu_baseline leg)."""
+    from oracle import aweq_oracle as orc
+    dt = orc.F16 if wl.dtype == "f16" else orc.BF16
+    gran = orc.PER_ROW if wl.w_gran == "row" else orc.PER_GROUP
+    for inp in wl.inputs:
+        lins = [l for l in wl.linears if l.input == inp.name]
+        xs = orc.stats(Xb[inp.name], dt)
+        wr = None
+        for l in lins:
+            wr = orc.wrange(Wb[l.name], dt, prev=wr)
+        f = orc.factors(xs[0], xs[1], xs[2], wr[0], wr[1])
+        for l in lins:
+            codes, step, zp, delta = orc.equalize_quantize(Wb[l.name], dt, f["s"], f["mu_hat"], bits, gran, wl.group)
+            orc.bias_correct(delta, None, dt)
+        if wl.act_quant:
+            orc.quant_act(Xb[inp.name], dt, f["rinv"], orc.PER_ROW)
+
+
+def cpu_sample(wl_full: synth.Workload, sample_tokens: int):
+    """The same layer with only the first ``sample_tokens`` tokens of every input."""
+    import dataclasses
+    inputs = tuple(dataclasses.replace(i, n_tokens=min(sample_tokens, i.n_tokens)) for i in wl_full.inputs)
+    return dataclasses.replace(wl_full, inputs=inputs)
+
+
+def run_reference(args, wl, bits):
+    from oracle import aweq_oracle as orc
+    from paper_2311_01305_b200 import calibrate
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    swl = cpu_sample(wl, args.cpu_sample_tokens)
+    X, W = generate(swl, "cpu", 0)
+    Xb = {k: synth.raw_bits(v) for k, v in X.items()}
+    Wb = {k: synth.raw_bits(v) for k, v in W.items()}
+    nbytes = calibrate_bytes(swl, bits)
+    for _ in range(args.warmup):
+        oracle_pass(swl, bits, Xb, Wb)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(swl, bits, Xb, Wb)
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = nbytes / dt / 1e9
+    sample = "first %d tokens of every layer input, all weight matrices at full size" % args.cpu_sample_tokens
+    line = {
+        "impl": "reference", "metric": "aweq_layer_pass_hbm_gbs", "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "w_bits": bits, "sample": sample},
+        "tokens_per_s": swl.inputs[0].n_tokens / dt,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": orc.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def calibrate_bytes(wl, bits):
+    from paper_2311_01305_b200 import calibrate
+    return calibrate.algorithmic_bytes(wl, bits)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--bits", type=int, default=0, help="weight bit-width (default: the workload's first)")
+    ap.add_argument("--tokens-scale", type=float, default=1.0, help="shrink the token count (profiling captures)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=2048)
+    args = ap.parse_args()
+
+    wl = synth.workloads(args.tokens_scale)[args.workload]
+    bits = args.bits or wl.w_bits[0]
+    if args.impl == "reference":
+        return run_reference(args, wl, bits)
+
+    from paper_2311_01305_b200 import aweq, calibrate
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the calibration pass has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    X, W = generate(wl, dev, rank)
+    cal = calibrate.LayerCalibrator(wl, bits, X, W, None)
+    nbytes = calibrate.algorithmic_bytes(wl, bits)
+    tokens = wl.inputs[0].n_tokens
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # profiling hooks around step 1 (and step 6) of every library call in the timed region
+    def ev_pair():
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); b.record()              # create the handles
+        return a, b
+    hooks = [[(ev_pair(), ev_pair() if wl.act_quant else None) for _ in cal.passes] for _ in range(args.steps)]
+    torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        cal.run()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.15)
+    n0 = aweq.launch_count()
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record()
+    for k in range(args.steps):
+        for lp, (es, ea) in zip(cal.passes, hooks[k]):
+            lp.set_events(es, ea)
+            lp(cal.ws, cal.status)
+    t_end.record()
+    barrier()
+    launches = aweq.launch_count() - n0
+    clocks = sampler.stop()
+    for lp in cal.passes:
+        lp.set_events(None, None)
+    ms = t_begin.elapsed_time(t_end) / args.steps
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    status = aweq.read_status(cal.status)
+    if status["wait_timeout"]:
+        raise SystemExit("a bounded wait inside a kernel gave up: results invalid")
+
+    # dominant kernel: the statistics sweep (W8A8 workloads: the activation quantiser moves more bytes)
+    stats_ms = [sum(es[0].elapsed_time(es[1]) for es, _ in hooks[k]) for k in range(args.steps)]
+    stats_bytes = sum(2 * i.n_tokens * i.c_in for i in wl.inputs)
+    dom = {"kernel": "colreduce_kernel (aweq_stats)", "bytes": stats_bytes, "ms": statistics.mean(stats_ms),
+           "launches_per_step": len(cal.passes)}
+    if wl.act_quant:
+        act_ms = [sum(ea[0].elapsed_time(ea[1]) for _, ea in hooks[k]) for k in range(args.steps)]
+        act_bytes = sum(3 * i.n_tokens * i.c_in + 8 * i.n_tokens for i in wl.inputs)
+        dom = {"kernel": "rowquant_kernel (aweq_quant_act)", "bytes": act_bytes, "ms": statistics.mean(act_ms),
+               "launches_per_step": len(cal.passes), "stats_gbs": stats_bytes / statistics.mean(stats_ms) / 1e6}
+    peak, peak_kind = measured_peaks()
+    achieved = dom["bytes"] / dom["ms"] / 1e6
+    roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": None,
+                "launch_ms": dom["ms"] / dom["launches_per_step"],
+                "bytes_per_launch": dom["bytes"] / dom["launches_per_step"]}
+    if "stats_gbs" in dom:
+        roofline["stats_gbs"] = dom["stats_gbs"]
+
+    gbs = world * nbytes / ms / 1e6
+    line = {
+        "metric": "aweq_layer_pass_hbm_gbs", "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "w_bits": bits, "w_gran": wl.w_gran, "group": wl.group,
+                   "act_quant": wl.act_quant, "storage": wl.dtype, "tokens_per_gpu": tokens,
+                   "algorithmic_bytes_per_gpu": nbytes, "cache": "inputs (GBs) far larger than the 126 MB L2",
+                   "parallelism": "token shards, one per GPU" if world > 1 else "single GPU"},
+        "tokens_per_s": world * tokens / (ms / 1e3),
+        "pct_of_8000_gbs": 100.0 * gbs / world / NORTH_STAR_PEAK_GBS,
+        "pct_of_measured_copy": 100.0 * gbs / world / peak,
+        "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "device_status": status,
+    }
+
+    # ---------------------------------------------------------------- end to end: host buffers in, results out
+    if not args.no_e2e:
+        hostX = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in X.items()}
+        hostW = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in W.items()}
+        res_names = {l.name: ("codes", "step", "zp", "bias") for l in wl.linears}
+        res_names.update({i.name: ("s",) + (("Xq", "act_step", "act_zp") if wl.act_quant else ()) for i in wl.inputs})
+        host_out = {n: {k: torch.empty(cal.out[n][k].shape, dtype=cal.out[n][k].dtype, pin_memory=True)
+                        for k in ks} for n, ks in res_names.items() if n in cal.out}
+        h2d = sum(v.numel() * v.element_size() for v in list(hostX.values()) + list(hostW.values()))
+        d2h = sum(t.numel() * t.element_size() for d in host_out.values() for t in d.values())
+
+        def e2e_step():
+            for k, v in hostW.items():
+                W[k].copy_(v, non_blocking=True)
+            for lp, inp in zip(cal.passes, [i for i in wl.inputs if i.name in cal.out]):
+                X[inp.name].copy_(hostX[inp.name], non_blocking=True)
+                lp(cal.ws, cal.status)
+            for n, d in host_out.items():
+                for k, t in d.items():
+                    t.copy_(cal.out[n][k], non_blocking=True)
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        ems = a.elapsed_time(b) / args.e2e_steps
+        if dist is not None:
+            t = torch.tensor([ems], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        line["e2e"] = {"value": world * nbytes / ems / 1e6, "unit": "GB/s", "ms_per_step": ems,
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
+        del hostX, hostW, host_out
+
+    # ---------------------------------------------------------------- the oracle beside it (rank 0, 1 GPU)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import aweq_oracle as orc
+        swl = cpu_sample(wl, args.cpu_sample_tokens)
+        Xb = {i.name: synth.raw_bits(X[i.name][:i.n_tokens]) for i in swl.inputs}
+        Wb = {k: synth.raw_bits(v) for k, v in W.items()}
+        t0 = time.perf_counter()
+        oracle_pass(swl, bits, Xb, Wb)
+        dt = time.perf_counter() - t0
+        sbytes = calibrate.algorithmic_bytes(swl, bits)
+        line["cpu_baseline"] = {"value": sbytes / dt / 1e9, "unit": "GB/s", "cores": orc.threads(), "kind": "oracle",
+                                "seconds": dt, "tokens_per_s": swl.inputs[0].n_tokens / dt,
+                                "sample": "first %d tokens of every layer input, all weight matrices at full size"
+                                          % args.cpu_sample_tokens}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

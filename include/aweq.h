@@ -234,6 +234,9 @@ typedef struct {
     /* activation quantisation (optional: Xq == NULL skips step 6) */
     unsigned char *Xq; float *act_step; int *act_zp; int act_bits;
     int flags;
+    /* optional profiling hooks: cudaEvent_t handles (or NULL) recorded on `stream`
+     * immediately before and after step 1 and step 6 */
+    void *ev_stats_begin, *ev_stats_end, *ev_act_begin, *ev_act_end;
 } aweq_layer_args;
 
 size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args);

@@ -49,6 +49,7 @@ class LayerArgs(ctypes.Structure):
         ("xmin", _vp), ("xmax", _vp), ("xmean", _vp), ("wmin", _vp), ("wmax", _vp), ("s", _vp), ("rinv", _vp),
         ("mu_hat", _vp), ("pX", _vp), ("pW", _vp), ("scalars", _vp),
         ("Xq", _vp), ("act_step", _vp), ("act_zp", _vp), ("act_bits", _i), ("flags", _i),
+        ("ev_stats_begin", _vp), ("ev_stats_end", _vp), ("ev_act_begin", _vp), ("ev_act_end", _vp),
     ]
 
 
@@ -221,6 +222,15 @@ class LayerPass:
         a.act_bits, a.flags = act_bits, flags
         self.args = a
         self.ws_bytes = int(_lib.aweq_layer_pass_workspace_bytes(ctypes.byref(a)))
+
+    def set_events(self, stats=None, act=None) -> None:
+        """Profiling hooks: pairs of recorded-once ``torch.cuda.Event(enable_timing=True)``
+        (or None) that the library records around step 1 and step 6."""
+        def h(e):
+            return None if e is None else e.cuda_event
+        self._events = (stats, act)
+        self.args.ev_stats_begin, self.args.ev_stats_end = (h(stats[0]), h(stats[1])) if stats else (None, None)
+        self.args.ev_act_begin, self.args.ev_act_end = (h(act[0]), h(act[1])) if act else (None, None)
 
     def __call__(self, ws: torch.Tensor, st: Optional[torch.Tensor] = None) -> None:
         _check(_lib.aweq_layer_pass(ctypes.byref(self.args), _ptr(ws), ws.numel(), _ptr(st), _stream()))

@@ -265,10 +265,13 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     void *ws_eq = base + col_part;
     const size_t ws_eq_bytes = need - col_part;
 
+    cudaStream_t cs = (cudaStream_t)stream;
     // steps 1-2
+    if (a->ev_stats_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_begin, cs));
     rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
                     col_part, st, stream);
     if (rc != AWEQ_OK) return rc;
+    if (a->ev_stats_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_end, cs));
     for (int i = 0; i < a->n_w; ++i) {
         rc = aweq_wrange(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], a->wmin, a->wmax, i > 0, ws_col, col_part,
                          st, stream);
@@ -302,9 +305,11 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     }
     // step 6
     if (a->Xq) {
+        if (a->ev_act_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_act_begin, cs));
         rc = aweq_quant_act(a->X, a->dt, a->N, a->C_in, a->ldx, rinv_used, a->act_bits ? a->act_bits : 8, AWEQ_PER_ROW,
                             nullptr, a->Xq, a->act_step, a->act_zp, st, stream);
         if (rc != AWEQ_OK) return rc;
+        if (a->ev_act_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_act_end, cs));
     }
     return AWEQ_OK;
 }

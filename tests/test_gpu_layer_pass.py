@@ -1,0 +1,104 @@
+"""The fused layer pass (all six steps through one C-ABI call per input)
+against the oracle chain: the single OPT-125M-shaped W8A8 linear at full size,
+matrices that share one input, and the AWE / BC switches of the paper's
+ablation (Table 4)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import aweq_oracle as orc
+from paper_2311_01305_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def make_workload_tensors(wl, device="cpu", layer=0, offset=None):
+    X, W = {}, {}
+    for i, inp in enumerate(wl.inputs):
+        off = None if offset is None else torch.linspace(-offset, offset, inp.c_in)
+        X[inp.name] = synth.make_activations(inp, wl.dtype, synth.tensor_seed(wl.seed, layer, i), device,
+                                             channel_offset=off)
+    for i, lin in enumerate(wl.linears):
+        W[lin.name] = synth.make_weight(lin, wl.dtype, synth.tensor_seed(wl.seed, layer, 100 + i), device)
+    return X, W
+
+
+def compare_layer(wl, bits, Xc, Wc, bias_c=None, flags=0):
+    from paper_2311_01305_b200 import aweq, calibrate
+    Xd = {k: v.to(DEV) for k, v in Xc.items()}
+    Wd = {k: v.to(DEV) for k, v in Wc.items()}
+    bd = None if bias_c is None else {k: v.to(DEV) for k, v in bias_c.items()}
+    cal = calibrate.LayerCalibrator(wl, bits, Xd, Wd, bd, flags=flags)
+    n0 = aweq.launch_count()
+    cal.run()
+    torch.cuda.synchronize()
+    assert aweq.launch_count() > n0
+    assert aweq.read_status(cal.status) == {"nonfinite": 0, "zero_range": 0, "wait_timeout": 0}
+    gran = orc.PER_ROW if wl.w_gran == "row" else orc.PER_GROUP
+    eq = not (flags & aweq.FLAG_NO_EQUALIZE)
+    bc = not (flags & aweq.FLAG_NO_BIAS_CORRECT)
+    for inp in wl.inputs:
+        lins = [l for l in wl.linears if l.input == inp.name]
+        ref = util.oracle_layer(Xc[inp.name], [Wc[l.name] for l in lins], bits, gran, wl.group,
+                                None if bias_c is None else [bias_c.get(l.name) for l in lins],
+                                act_quant=wl.act_quant, equalize=eq, bias_correct=bc)
+        o = {k: v.cpu().numpy() for k, v in cal.out[inp.name].items()}
+        util.assert_same_values(o["xmin"], ref["stats"][0])
+        util.assert_same_values(o["xmax"], ref["stats"][1])
+        mean_abs = np.abs(Xc[inp.name].double().numpy()).mean(axis=0)
+        assert np.all(np.abs(o["xmean"].astype(np.float64) - ref["stats"][2]) <= util.mean_tolerance(ref["stats"][2], mean_abs))
+        util.assert_same_values(o["wmin"], ref["wrange"][0])
+        util.assert_same_values(o["wmax"], ref["wrange"][1])
+        f = ref["factors"]
+        # Eq. 10 is evaluated in binary64 on both sides: identical factors
+        util.assert_same_values(o["s"], f["s"], "s")
+        util.assert_same_values(o["rinv"], f["rinv"], "rinv")
+        assert np.allclose(o["mu_hat"], f["mu_hat"], rtol=1e-6, atol=1e-9 * mean_abs.max())
+        assert np.allclose(o["pX"], f["pX"], rtol=1e-6) and np.allclose(o["pW"], f["pW"], rtol=1e-6)
+        assert np.allclose(o["scalars"], f["scalars"], rtol=1e-6)
+        for l, r in zip(lins, ref["linears"]):
+            lo = {k: v.cpu() for k, v in cal.out[l.name].items()}
+            util.assert_same_values(lo["zp"].numpy(), r["zp"], l.name + " zp")
+            util.assert_same_values(lo["step"].numpy(), r["step"], l.name + " step")
+            util.assert_same_values(lo["codes"].numpy(), r["codes"], l.name + " codes")
+            if bc:
+                assert np.allclose(lo["bias_f32"].numpy(), r["bias_f32"], rtol=0, atol=1e-5)
+                got = orc.decode16(util.bits(lo["bias"]), util.odt(lo["bias"]))
+                assert np.all(np.abs(got - orc.decode16(r["bias_16"], util.odt(lo["bias"]))) <= 1e-3)
+        if wl.act_quant:
+            util.assert_same_values(o["act_zp"], ref["act"][2], "act zp")
+            util.assert_same_values(o["act_step"], ref["act"][1], "act step")
+            util.assert_same_values(o["Xq"], ref["act"][0], "act codes")
+    return cal
+
+
+def test_opt125m_single_linear_w8a8_full_size():
+    wl = synth.workloads()["opt125m_linear_w8a8"]
+    Xc, Wc = make_workload_tensors(wl)
+    bias = {"linear": torch.zeros(768, dtype=torch.float16)}
+    compare_layer(wl, 8, Xc, Wc, bias)
+
+
+def test_opt125m_single_linear_with_channel_offsets_makes_a_bias():
+    wl = synth.workloads()["opt125m_linear_w8a8"]
+    Xc, Wc = make_workload_tensors(wl, offset=3.0)
+    cal = compare_layer(wl, 8, Xc, Wc, None)
+    assert float(cal.out["linear"]["bias_f32"].abs().max()) > 1e-4
+
+
+@pytest.mark.parametrize("name,bits", [("opt125m_model_w8a8", 8), ("llama7b_layer_w4w3_g128", 4),
+                                       ("llama7b_layer_w4w3_g128", 3), ("llama13b_layer_w8a8", 8)])
+def test_decoder_layer_shapes_with_shared_inputs_few_tokens(name, bits):
+    wl = synth.workloads(n_tokens_scale=1.0 / 1024)[name]       # 256 tokens, full channel counts
+    Xc, Wc = make_workload_tensors(wl, offset=1.0)
+    compare_layer(wl, bits, Xc, Wc, None)
+
+
+def test_ablation_switches():
+    from paper_2311_01305_b200 import aweq
+    wl = synth.workloads(n_tokens_scale=1.0 / 8)["opt125m_linear_w8a8"]
+    Xc, Wc = make_workload_tensors(wl, offset=2.0)
+    for flags in (aweq.FLAG_NO_EQUALIZE, aweq.FLAG_NO_BIAS_CORRECT, aweq.FLAG_NO_EQUALIZE | aweq.FLAG_NO_BIAS_CORRECT):
+        compare_layer(wl, 8, Xc, Wc, None, flags=flags)

@@ -347,7 +347,7 @@ def test_quant_act_per_token(N, C_in, dtype):
 
 
 def test_quant_act_row_pitch_and_low_bits():
-    big = util.rand16((500, 1100), torch.float16, seed=9, offset=1.0).to(DEV)
+    big = util.rand16((500, 1104), torch.float16, seed=9, offset=1.0).to(DEV)
     X = big[:, 8:8 + 1024]
     rinv = (torch.rand(1024, generator=torch.Generator().manual_seed(1)) + 0.5).numpy()
     for bits in (8, 4):

@@ -61,3 +61,31 @@ def assert_same_values(a, b, what=""):
     bad = ~((a == b) | (np.isnan(a.astype(np.float64)) & np.isnan(b.astype(np.float64))))
     assert not bad.any(), "%s: %d mismatches, first at %s: %s vs %s" % (
         what, int(bad.sum()), np.argwhere(bad)[0], a[bad][0], b[bad][0])
+
+
+def oracle_layer(Xc, Wcs, bits, gran, group, biases=None, act_quant=True, equalize=True, bias_correct=True):
+    """The six steps through the CPU oracle for one input and the matrices it feeds."""
+    dt = odt(Xc)
+    xs = orc.stats(bits_of(Xc), dt)
+    wr = None
+    for Wc in Wcs:
+        wr = orc.wrange(bits_of(Wc), dt, prev=wr)
+    f = orc.factors(xs[0], xs[1], xs[2], wr[0], wr[1])
+    s = f["s"] if equalize else None
+    rinv = f["rinv"] if equalize else None
+    mu = f["mu_hat"] if equalize else xs[2]
+    res = {"stats": xs, "wrange": wr, "factors": f, "linears": []}
+    for i, Wc in enumerate(Wcs):
+        codes, step, zp, delta = orc.equalize_quantize(bits_of(Wc), dt, s, mu if bias_correct else None, bits, gran, group)
+        lin = {"codes": codes, "step": step, "zp": zp, "delta": delta}
+        if bias_correct:
+            b = None if biases is None or biases[i] is None else bits_of(biases[i])
+            lin["bias_f32"], lin["bias_16"] = orc.bias_correct(delta, b, dt)
+        res["linears"].append(lin)
+    if act_quant:
+        res["act"] = orc.quant_act(bits_of(Xc), dt, rinv, orc.PER_ROW)
+    return res
+
+
+def bits_of(t):
+    return bits(t)
