@@ -312,7 +312,8 @@ def test_bias_correct_both_routes(bits, gran, group, dtype):
             ref16 = o_16 if with_bias else orc.bias_correct(o_delta, None, util.odt(bias_c))[1]
             assert np.allclose(b32.cpu().numpy(), ref32, rtol=0, atol=1e-5)
             got16 = orc.decode16(util.bits(b16), util.odt(bias_c))
-            assert np.all(np.abs(got16 - orc.decode16(ref16, util.odt(bias_c))) <= 1e-3)
+            want16 = orc.decode16(ref16, util.odt(bias_c))
+            assert np.all(np.abs(got16 - want16) <= util.bias16_tolerance(want16, util.odt(bias_c)))
 
 
 # ------------------------------------------------------------------ step 6

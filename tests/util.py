@@ -89,3 +89,14 @@ def oracle_layer(Xc, Wcs, bits, gran, group, biases=None, act_quant=True, equali
 
 def bits_of(t):
     return bits(t)
+
+
+def bias16_tolerance(ref, dtype_tag):
+    """1e-3 absolute (the stated bound for fp16 biases), but never tighter than one
+    unit in the last place of the 16-bit format at that magnitude: a binary32 value
+    that sits next to a rounding tie may legitimately round to the neighbouring
+    16-bit value (bf16 has 8 significant bits: one ulp is 2e-3 already at 0.25)."""
+    mant = 10 if dtype_tag == orc.F16 else 7
+    a = np.maximum(np.abs(np.asarray(ref, dtype=np.float64)), 2.0 ** -14)
+    ulp = 2.0 ** (np.floor(np.log2(a)) - mant)
+    return np.maximum(1e-3, ulp)
