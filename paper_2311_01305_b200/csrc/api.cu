@@ -135,10 +135,11 @@ aweq_status aweq_factors(const float *xmin, const float *xmax, const float *xmea
                        (cudaStream_t)stream);
 }
 
-aweq_status aweq_equalize_quantize(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ldw,
-                                   const float *s, const float *mu_hat, int bits, aweq_gran gran, int group,
-                                   unsigned char *codes, float *step, int *zp, float *epsmu, void *ws,
-                                   size_t ws_bytes, aweq_dev_status *st, void *stream)
+static aweq_status equalize_quantize_impl(const void *W, aweq_dtype dt, long long C_out, long long C_in,
+                                          long long ldw, const float *s, const float *mu_hat, int bits,
+                                          aweq_gran gran, int group, unsigned char *codes, float *step, int *zp,
+                                          float *epsmu, const BiasIO &bias, void *ws, size_t ws_bytes,
+                                          aweq_dev_status *st, void *stream)
 {
     aweq_status rc = check_matrix(W, dt, C_out, C_in, ldw, false);
     if (rc != AWEQ_OK) return rc;
@@ -151,11 +152,11 @@ aweq_status aweq_equalize_quantize(const void *W, aweq_dtype dt, long long C_out
     cudaStream_t cs = (cudaStream_t)stream;
     if (gran == AWEQ_PER_ROW) {
         if (!rowquant_supported(C_out, C_in)) return AWEQ_ERR_SHAPE;
-        return run_rowquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, codes, step, zp, epsmu, st, cs);
+        return run_rowquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, codes, step, zp, epsmu, bias, st, cs);
     }
     if (gran == AWEQ_PER_GROUP)
         return run_warpquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, group, nullptr, codes, step, zp, epsmu,
-                             st, cs);
+                             bias, st, cs);
     // per tensor: column extremes of W -> extremes of diag(s) W -> static-range quantiser
     char *base = reinterpret_cast<char *>(ws);
     float *cmin = reinterpret_cast<float *>(base);
@@ -166,7 +167,18 @@ aweq_status aweq_equalize_quantize(const void *W, aweq_dtype dt, long long C_out
     if (rc != AWEQ_OK) return rc;
     rc = run_scaled_tensor_range(cmin, cmax, s, C_in, lo_hi, cs);
     if (rc != AWEQ_OK) return rc;
-    return run_warpquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, 0, lo_hi, codes, step, zp, epsmu, st, cs);
+    return run_warpquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, 0, lo_hi, codes, step, zp, epsmu, bias, st,
+                         cs);
+}
+
+aweq_status aweq_equalize_quantize(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ldw,
+                                   const float *s, const float *mu_hat, int bits, aweq_gran gran, int group,
+                                   unsigned char *codes, float *step, int *zp, float *epsmu, void *ws,
+                                   size_t ws_bytes, aweq_dev_status *st, void *stream)
+{
+    const BiasIO none = {nullptr, nullptr, nullptr, 0};
+    return equalize_quantize_impl(W, dt, C_out, C_in, ldw, s, mu_hat, bits, gran, group, codes, step, zp, epsmu, none,
+                                  ws, ws_bytes, st, stream);
 }
 
 aweq_status aweq_bias_correct(const float *epsmu, const void *W, aweq_dtype dt, const float *s,
@@ -201,12 +213,14 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
     cudaStream_t cs = (cudaStream_t)stream;
     if (gran == AWEQ_PER_ROW) {
         if (!rowquant_supported(N, C_in)) return AWEQ_ERR_SHAPE;
-        return run_rowquant(X, dt, N, C_in, ldx, rinv, nullptr, bits, false, Xq, step, zp, nullptr, st, cs);
+        const BiasIO none = {nullptr, nullptr, nullptr, 0};
+        return run_rowquant(X, dt, N, C_in, ldx, rinv, nullptr, bits, false, Xq, step, zp, nullptr, none, st, cs);
     }
     if (gran == AWEQ_PER_TENSOR) {
         if (!tensor_lo_hi) return AWEQ_ERR_NULL;
+        const BiasIO none = {nullptr, nullptr, nullptr, 0};
         return run_warpquant(X, dt, N, C_in, ldx, rinv, nullptr, bits, false, 0, tensor_lo_hi, Xq, step, zp, nullptr,
-                             st, cs);
+                             none, st, cs);
     }
     return AWEQ_ERR_UNSUPPORTED;
 }
@@ -286,22 +300,19 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     const float *s_used = eq ? a->s : nullptr;
     const float *rinv_used = eq ? a->rinv : nullptr;
     const float *mu_used = eq ? a->mu_hat : a->xmean;
-    // steps 4-5 per matrix
+    // steps 4-5 per matrix: the corrected bias is written by the quantiser itself
     for (int i = 0; i < a->n_w; ++i) {
         float *em = bc ? a->epsmu[i] : nullptr;
-        rc = aweq_equalize_quantize(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], s_used, bc ? mu_used : nullptr,
-                                    a->bits, a->gran, a->group, a->codes[i], a->step[i], a->zp[i], em, ws_eq,
+        BiasIO bias = {nullptr, nullptr, nullptr, a->dt == AWEQ_BF16};
+        if (bc) {
+            bias.in = reinterpret_cast<const uint16_t *>(a->bias_in ? a->bias_in[i] : nullptr);
+            bias.out = reinterpret_cast<uint16_t *>(a->bias_out ? a->bias_out[i] : nullptr);
+            bias.out_f32 = a->bias_out_f32 ? a->bias_out_f32[i] : nullptr;
+        }
+        rc = equalize_quantize_impl(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], s_used, bc ? mu_used : nullptr,
+                                    a->bits, a->gran, a->group, a->codes[i], a->step[i], a->zp[i], em, bias, ws_eq,
                                     ws_eq_bytes, st, stream);
         if (rc != AWEQ_OK) return rc;
-        if (bc) {
-            const void *bin = a->bias_in ? a->bias_in[i] : nullptr;
-            void *bout = a->bias_out ? a->bias_out[i] : nullptr;
-            float *bout32 = a->bias_out_f32 ? a->bias_out_f32[i] : nullptr;
-            rc = aweq_bias_correct(em, nullptr, a->dt, nullptr, nullptr, nullptr, nullptr, nullptr, a->C_out[i],
-                                   a->C_in, a->ldw[i], a->bits, a->gran, a->group, bin, bout, bout32, a->dt, st,
-                                   stream);
-            if (rc != AWEQ_OK) return rc;
-        }
     }
     // step 6
     if (a->Xq) {

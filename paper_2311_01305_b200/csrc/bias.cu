@@ -7,17 +7,6 @@
 
 namespace aweq {
 
-// bias'[o] = bias[o] - delta, written as binary32 and / or in the 16-bit bias type
-__device__ __forceinline__ void write_bias(long long o, float delta, const uint16_t *bias_in, uint16_t *bias_out,
-                                           float *bias_out_f32, int bias_bf16)
-{
-    float b = 0.0f;
-    if (bias_in) b = bias_bf16 ? BF16::one(bias_in[o]) : F16::one(bias_in[o]);
-    const float c = __fsub_rn(b, delta);
-    if (bias_out_f32) bias_out_f32[o] = c;
-    if (bias_out) bias_out[o] = bias_bf16 ? BF16::encode(c) : F16::encode(c);
-}
-
 __global__ void bias_apply_kernel(const float *__restrict__ epsmu, const uint16_t *__restrict__ bias_in,
                                   uint16_t *__restrict__ bias_out, float *__restrict__ bias_out_f32, int bias_bf16,
                                   long long C_out)

@@ -7,25 +7,41 @@
 // and are bound by HBM bandwidth.
 //
 // Layout of the work: the columns are cut into slabs of at most 256 16-byte
-// vectors (2048 columns) and the rows into splits; one CTA owns one
+// vectors (2048 columns) and the rows into splits; one CTA per SM owns one
 // (slab, split) pair, so a thread owns one vector column for its whole life and
 // keeps that column's eight running minima, maxima and sums in registers.
-// A producer warp streams the CTA's rows through a ring of shared-memory
-// stages with 1-D bulk copies (TMA, completion on mbarriers); eight consumer
-// warps read the stages back conflict-free (consecutive lanes, consecutive
-// 16-byte vectors).  min / max stay in packed 16-bit arithmetic (exact); sums
-// are binary32 over the eight rows of one stage and are folded into binary64
-// after every stage.  Each CTA writes one partial per column; a second small
+// A producer warp streams the CTA's rows through two shared-memory stages of
+// 24 rows each (up to 96 KB per stage) with 1-D bulk copies (TMA, completion on
+// mbarriers); eight consumer warps read the stages back conflict-free
+// (consecutive lanes, consecutive 16-byte vectors).  Of the geometries timed
+// on B200 (2-6 stages of 8-24 rows, one or two CTAs per SM) this one was the
+// fastest on both the 4096- and the 11008-column inputs.  min / max stay in packed 16-bit arithmetic (exact); sums
+// are binary32 over eight rows at a time (one mixed-precision add per element)
+// and are then added without rounding loss into a (hi, lo) pair of binary32
+// values per column, which is widened to binary64 once at the end.  Each CTA writes one partial per column; a second small
 // kernel reduces the partials over the splits in a fixed order, so results are
 // bit-reproducible from run to run.
 #include "common.cuh"
 
 namespace aweq {
 
-constexpr int kColThreads = 256;        // consumer threads = vectors per slab
-constexpr int kColRows = 8;             // rows per stage
-constexpr int kColStages = 3;
-constexpr int kColTargetCtas = 2 * kSmCount;
+#ifndef AWEQ_COL_THREADS
+#define AWEQ_COL_THREADS 256
+#endif
+#ifndef AWEQ_COL_ROWS
+#define AWEQ_COL_ROWS 24
+#endif
+#ifndef AWEQ_COL_STAGES
+#define AWEQ_COL_STAGES 2
+#endif
+#ifndef AWEQ_COL_CTAS_PER_SM
+#define AWEQ_COL_CTAS_PER_SM 1
+#endif
+constexpr int kColThreads = AWEQ_COL_THREADS;   // consumer threads = vectors per slab
+constexpr int kColRows = AWEQ_COL_ROWS;         // rows per stage
+constexpr int kColStages = AWEQ_COL_STAGES;
+constexpr int kColCtasPerSm = AWEQ_COL_CTAS_PER_SM;
+constexpr int kColTargetCtas = kColCtasPerSm * kSmCount;
 
 struct ColPlan {
     int nvec, nslab, slab_w, nsplit;
@@ -54,9 +70,61 @@ ColPlan plan_colreduce(long long rows, long long cols)
 
 size_t colreduce_ws_bytes(long long rows, long long cols)
 {
-    ColPlan p = plan_colreduce(rows, cols);
-    // pmin, pmax: float[nsplit][cols]; psum: double[nsplit][cols]
-    return (size_t)p.nsplit * (size_t)cols * 16 + 256;
+    // pmin, pmax: float[nsplit][cols]; psum: double[nsplit][cols].  Sized for the
+    // largest number of row splits any row count can get, so that a buffer sized
+    // for N rows also serves every call with fewer rows (streamed chunks).
+    (void)rows;
+    const int nvec = (int)(cols / 8);
+    const int nslab = (nvec + kColThreads - 1) / kColThreads;
+    int max_split = kColTargetCtas / (nslab > 0 ? nslab : 1);
+    if (max_split < 1) max_split = 1;
+    return (size_t)max_split * (size_t)cols * 16 + 256;
+}
+
+constexpr int kFlushRows = 8;           // rows summed in binary32 before the error-free fold
+static_assert(kColRows % kFlushRows == 0, "stage rows must be a multiple of the flush period");
+
+// acc += widen(16-bit value): one mixed-precision add per element (exact widening,
+// one binary32 rounding), no separate conversion
+template <class D>
+__device__ __forceinline__ void add_pair(float &a0, float &a1, uint32_t u);
+template <>
+__device__ __forceinline__ void add_pair<F16>(float &a0, float &a1, uint32_t u)
+{
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\t"
+        "add.rn.f32.f16 %0, l, %0;\n\tadd.rn.f32.f16 %1, h, %1;\n\t}"
+        : "+f"(a0), "+f"(a1) : "r"(u));
+}
+template <>
+__device__ __forceinline__ void add_pair<BF16>(float &a0, float &a1, uint32_t u)
+{
+    asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\t"
+        "add.rn.f32.bf16 %0, l, %0;\n\tadd.rn.f32.bf16 %1, h, %1;\n\t}"
+        : "+f"(a0), "+f"(a1) : "r"(u));
+}
+
+template <class D, bool WITH_SUM>
+__device__ __forceinline__ void accumulate_vec(const uint4 &v, typename D::T2 (&mn)[4], typename D::T2 (&mx)[4],
+                                               float (&acc)[8])
+{
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        typename D::T2 h = D::from_bits(u[k]);
+        mn[k] = __hmin2(mn[k], h);
+        mx[k] = __hmax2(mx[k], h);
+        if (WITH_SUM) add_pair<D>(acc[2 * k], acc[2 * k + 1], u[k]);
+    }
+}
+
+// (hi, lo) += a without losing the rounding error of hi + a (Knuth's two-sum)
+__device__ __forceinline__ void two_sum_into(float &hi, float &lo, float a)
+{
+    const float s = __fadd_rn(hi, a);
+    const float bb = __fsub_rn(s, hi);
+    const float e = __fadd_rn(__fsub_rn(hi, __fsub_rn(s, bb)), __fsub_rn(a, bb));
+    lo = __fadd_rn(lo, e);
+    hi = s;
 }
 
 struct ColSmem {
@@ -66,7 +134,7 @@ struct ColSmem {
 };
 
 template <class D, bool WITH_SUM>
-__global__ void __launch_bounds__(kColThreads + 32, 2)
+__global__ void __launch_bounds__(kColThreads + 32, kColCtasPerSm)
 colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, int nvec, int nslab, int slab_w,
                  long long rows_per_split, long long cols, float *__restrict__ pmin, float *__restrict__ pmax,
                  double *__restrict__ psum, aweq_dev_status *st)
@@ -134,9 +202,9 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
             mn[k] = D::from_bits(D::pos_inf2());
             mx[k] = D::from_bits(D::neg_inf2());
         }
-        double acc64[8];
+        float sum_hi[8], sum_lo[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) acc64[k] = 0.0;
+        for (int k = 0; k < 8; ++k) sum_hi[k] = sum_lo[k] = 0.0f;
         bool ok = true;
         for (int t = 0; t < ntiles; ++t) {
             const int s = t % kColStages;
@@ -147,48 +215,27 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
             const int rows = (int)min((long long)kColRows, r1 - row0);
             const uint4 *src = stage_base + (size_t)s * stage_vecs + t_col;
             if (mine) {
-                float acc32[8];
+                // groups of kFlushRows rows: binary32 partial sums, then an error-free
+                // addition into the (hi, lo) running sum
+                for (int rb = 0; rb < rows; rb += kFlushRows) {
+                    float acc32[8];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) acc32[k] = 0.0f;
-                if (rows == kColRows) {
-                    uint4 v[kColRows];
+                    for (int k = 0; k < 8; ++k) acc32[k] = 0.0f;
+                    if (rows - rb >= kFlushRows) {
+                        uint4 v[kFlushRows];
 #pragma unroll
-                    for (int r = 0; r < kColRows; ++r) v[r] = src[(size_t)r * w];
+                        for (int r = 0; r < kFlushRows; ++r) v[r] = src[(size_t)(rb + r) * w];
 #pragma unroll
-                    for (int r = 0; r < kColRows; ++r) {
-                        const uint32_t u[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            typename D::T2 h = D::from_bits(u[k]);
-                            mn[k] = __hmin2(mn[k], h);
-                            mx[k] = __hmax2(mx[k], h);
-                            if (WITH_SUM) {
-                                float2 f = D::to_float2(h);
-                                acc32[2 * k] += f.x;
-                                acc32[2 * k + 1] += f.y;
-                            }
-                        }
+                        for (int r = 0; r < kFlushRows; ++r)
+                            accumulate_vec<D, WITH_SUM>(v[r], mn, mx, acc32);
+                    } else {
+                        for (int r = rb; r < rows; ++r)
+                            accumulate_vec<D, WITH_SUM>(src[(size_t)r * w], mn, mx, acc32);
                     }
-                } else {
-                    for (int r = 0; r < rows; ++r) {
-                        uint4 vr = src[(size_t)r * w];
-                        const uint32_t u[4] = {vr.x, vr.y, vr.z, vr.w};
+                    if (WITH_SUM) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            typename D::T2 h = D::from_bits(u[k]);
-                            mn[k] = __hmin2(mn[k], h);
-                            mx[k] = __hmax2(mx[k], h);
-                            if (WITH_SUM) {
-                                float2 f = D::to_float2(h);
-                                acc32[2 * k] += f.x;
-                                acc32[2 * k + 1] += f.y;
-                            }
-                        }
+                        for (int k = 0; k < 8; ++k) two_sum_into(sum_hi[k], sum_lo[k], acc32[k]);
                     }
-                }
-                if (WITH_SUM) {
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) acc64[k] += (double)acc32[k];
                 }
             }
             __syncwarp();
@@ -215,7 +262,9 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
             if (WITH_SUM) {
                 double2 *qs = reinterpret_cast<double2 *>(psum + o);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) qs[k] = make_double2(acc64[2 * k], acc64[2 * k + 1]);
+                for (int k = 0; k < 4; ++k)
+                    qs[k] = make_double2((double)sum_hi[2 * k] + (double)sum_lo[2 * k],
+                                         (double)sum_hi[2 * k + 1] + (double)sum_lo[2 * k + 1]);
             }
         }
     }
@@ -229,22 +278,41 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
     }
 }
 
-// Reduce the per-split partials in split order; merge with the running state
-// when accumulating.  One thread per column.
+// Reduce the per-split partials in a fixed order; merge with the running state
+// when accumulating.  A block handles 32 columns with 8 threads each: thread
+// (c, k) folds splits k, k+8, ... and the eight partial results of a column are
+// then combined in order of k, so the result does not depend on timing.
+constexpr int kFinCols = 32, kFinLanes = 8;
+
 template <bool WITH_SUM>
-__global__ void colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restrict__ pmax,
-                                          const double *__restrict__ psum, int nsplit, long long cols,
-                                          long long nrows, float *omin, float *omax, float *omean, double *osum,
-                                          const long long *count, int accumulate, aweq_dev_status *st)
+__global__ void __launch_bounds__(kFinCols * kFinLanes)
+colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restrict__ pmax,
+                          const double *__restrict__ psum, int nsplit, long long cols, long long nrows, float *omin,
+                          float *omax, float *omean, double *osum, const long long *count, int accumulate,
+                          aweq_dev_status *st)
 {
-    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= cols) return;
+    __shared__ float slo[kFinLanes][kFinCols], shi[kFinLanes][kFinCols];
+    __shared__ double ssum[kFinLanes][kFinCols];
+    const int c = threadIdx.x % kFinCols, k0 = threadIdx.x / kFinCols;
+    const long long j = (long long)blockIdx.x * kFinCols + c;
     float lo = INFINITY, hi = -INFINITY;
     double sum = 0.0;
-    for (int k = 0; k < nsplit; ++k) {
-        lo = fminf(lo, pmin[(size_t)k * cols + j]);
-        hi = fmaxf(hi, pmax[(size_t)k * cols + j]);
-        if (WITH_SUM) sum += psum[(size_t)k * cols + j];
+    if (j < cols) {
+        for (int k = k0; k < nsplit; k += kFinLanes) {
+            lo = fminf(lo, pmin[(size_t)k * cols + j]);
+            hi = fmaxf(hi, pmax[(size_t)k * cols + j]);
+            if (WITH_SUM) sum += psum[(size_t)k * cols + j];
+        }
+    }
+    slo[k0][c] = lo;
+    shi[k0][c] = hi;
+    if (WITH_SUM) ssum[k0][c] = sum;
+    __syncthreads();
+    if (k0 != 0 || j >= cols) return;
+    for (int k = 1; k < kFinLanes; ++k) {
+        lo = fminf(lo, slo[k][c]);
+        hi = fmaxf(hi, shi[k][c]);
+        if (WITH_SUM) sum += ssum[k][c];
     }
     long long total = nrows;
     if (accumulate) {
@@ -302,8 +370,7 @@ static aweq_status launch_colreduce(const void *X, long long rows, long long col
             pmax, psum, st);
         AWEQ_LAUNCH_CHECK();
     }
-    const int ft = 256;
-    colreduce_finalize_kernel<WITH_SUM><<<(unsigned)((cols + ft - 1) / ft), ft, 0, stream>>>(
+    colreduce_finalize_kernel<WITH_SUM><<<(unsigned)((cols + kFinCols - 1) / kFinCols), kFinCols * kFinLanes, 0, stream>>>(
         pmin, pmax, psum, nsplit_eff, cols, rows, omin, omax, omean, osum, count, accumulate, st);
     AWEQ_LAUNCH_CHECK();
     if (WITH_SUM && count) {

@@ -171,6 +171,25 @@ __device__ __forceinline__ float warp_sum(float v)      // fixed butterfly order
     return v;
 }
 
+// ------------------------------------------------------------------ Eq. 15, last step
+struct BiasIO {
+    const uint16_t *in;      // 16-bit bias of the layer, or NULL (no bias)
+    uint16_t *out;           // corrected bias, 16-bit (may be NULL)
+    float *out_f32;          // corrected bias, binary32 (may be NULL)
+    int bf16;                // 16-bit type of in / out
+};
+// bias'[o] = bias[o] - delta, written as binary32 and / or in the 16-bit bias type
+__device__ __forceinline__ void write_bias(long long o, float delta, const uint16_t *bias_in, uint16_t *bias_out,
+                                           float *bias_out_f32, int bias_bf16)
+{
+    float b = 0.0f;
+    if (bias_in) b = bias_bf16 ? BF16::one(bias_in[o]) : F16::one(bias_in[o]);
+    const float c = __fsub_rn(b, delta);
+    if (bias_out_f32) bias_out_f32[o] = c;
+    if (bias_out) bias_out[o] = bias_bf16 ? BF16::encode(c) : F16::encode(c);
+}
+
+
 // ------------------------------------------------------------------ Eq. 1-2, scalar part
 // (Step, 1/Step, Z) of a vector with extremes lo, hi; all IEEE binary32, no FMA.
 struct QParams {

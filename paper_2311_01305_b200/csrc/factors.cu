@@ -27,6 +27,55 @@ __device__ __forceinline__ void fac_merge(FacRed &a, const FacRed &b)
     a.merx = fmaxf(a.merx, b.merx); a.merw = fmaxf(a.merw, b.merw);
 }
 
+struct FacOut {
+    float s, rinv, mu;
+};
+
+// one channel of pass 1: the factor, its reciprocal, E[x^], and the running extremes
+__device__ __forceinline__ FacOut fac_channel(float lo, float hi, float mean, float wl, float wh, FacRed &a,
+                                              unsigned int &dead)
+{
+    const float rx = __fsub_rn(hi, lo), rw = __fsub_rn(wh, wl);
+    float sj = 1.0f;
+    bool ok = isfinite(rx) && isfinite(rw) && rx > 0.0f && rw > 0.0f;
+    if (ok) {
+        // Eq. 10 as printed, in binary64, rounded once to binary32
+        sj = (float)__dmul_rn(__ddiv_rn(1.0, (double)rw), __dsqrt_rn(__dmul_rn((double)rx, (double)rw)));
+        if (!(isfinite(sj) && sj > 0.0f) || !isfinite(__fdiv_rn(1.0f, sj))) {
+            sj = 1.0f;
+            ok = false;
+        }
+    }
+    if (!ok) ++dead;
+    const float ri = __fdiv_rn(1.0f, sj);
+    const float exl = __fmul_rn(lo, ri), exh = __fmul_rn(hi, ri);
+    const float ewl = __fmul_rn(wl, sj), ewh = __fmul_rn(wh, sj);
+    a.xlo = fminf(a.xlo, lo); a.xhi = fmaxf(a.xhi, hi);
+    a.wlo = fminf(a.wlo, wl); a.whi = fmaxf(a.whi, wh);
+    a.exlo = fminf(a.exlo, exl); a.exhi = fmaxf(a.exhi, exh);
+    a.ewlo = fminf(a.ewlo, ewl); a.ewhi = fmaxf(a.ewhi, ewh);
+    a.mrx = fmaxf(a.mrx, rx); a.mrw = fmaxf(a.mrw, rw);
+    a.merx = fmaxf(a.merx, exh - exl); a.merw = fmaxf(a.merw, ewh - ewl);
+    FacOut o;
+    o.s = sj; o.rinv = ri; o.mu = __fmul_rn(mean, ri);
+    return o;
+}
+
+// one channel of pass 2: p^X, p^W and the two objective terms (reciprocals of the tensor ranges given)
+__device__ __forceinline__ void fac_precision(float lo, float hi, float wl, float wh, float sj, float ri, double iRX,
+                                              double iRW, double iEX, double iEW, float &px, float &pw, double &o0,
+                                              double &o1)
+{
+    const double rx = (double)__fsub_rn(hi, lo), rw = (double)__fsub_rn(wh, wl);
+    const double erx = (double)__fmul_rn(hi, ri) - (double)__fmul_rn(lo, ri);
+    const double erw = (double)__fmul_rn(wh, sj) - (double)__fmul_rn(wl, sj);
+    const double a = rx * iRX, b = rw * iRW;
+    px = (float)a;
+    pw = (float)b;
+    o0 += a * b;
+    o1 += (erx * iEX) * (erw * iEW);
+}
+
 __global__ void __launch_bounds__(kFacThreads)
 factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, const float *__restrict__ xmean,
                const float *__restrict__ wmin, const float *__restrict__ wmax, int C, float *__restrict__ s,
@@ -40,37 +89,35 @@ factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, c
     if (threadIdx.x == 0) dead_count = 0;
     __syncthreads();
 
+    // four channels per thread and step (128-bit loads) when the arrays allow it
+    const bool vec4 = ((reinterpret_cast<uintptr_t>(xmin) | reinterpret_cast<uintptr_t>(xmax) |
+                        reinterpret_cast<uintptr_t>(xmean) | reinterpret_cast<uintptr_t>(wmin) |
+                        reinterpret_cast<uintptr_t>(wmax) | reinterpret_cast<uintptr_t>(s) |
+                        reinterpret_cast<uintptr_t>(rinv) | reinterpret_cast<uintptr_t>(mu_hat) |
+                        reinterpret_cast<uintptr_t>(pX) | reinterpret_cast<uintptr_t>(pW)) & 15) == 0;
+    const int nquad = vec4 ? C / 4 : 0;
+
     FacRed a;
     a.xlo = a.wlo = a.exlo = a.ewlo = INFINITY;
     a.xhi = a.whi = a.exhi = a.ewhi = -INFINITY;
     a.mrx = a.mrw = a.merx = a.merw = 0.0f;
     unsigned int dead = 0;
-    for (int j = threadIdx.x; j < C; j += kFacThreads) {
-        const float lo = xmin[j], hi = xmax[j], wl = wmin[j], wh = wmax[j];
-        const float rx = __fsub_rn(hi, lo), rw = __fsub_rn(wh, wl);
-        float sj = 1.0f;
-        bool ok = isfinite(rx) && isfinite(rw) && rx > 0.0f && rw > 0.0f;
-        if (ok) {
-            // Eq. 10 as printed, in binary64, rounded once to binary32
-            sj = (float)__dmul_rn(__ddiv_rn(1.0, (double)rw), __dsqrt_rn(__dmul_rn((double)rx, (double)rw)));
-            if (!(isfinite(sj) && sj > 0.0f) || !isfinite(__fdiv_rn(1.0f, sj))) {
-                sj = 1.0f;
-                ok = false;
-            }
-        }
-        if (!ok) ++dead;
-        const float ri = __fdiv_rn(1.0f, sj);
-        s[j] = sj;
-        rinv[j] = ri;
-        mu_hat[j] = __fmul_rn(xmean[j], ri);
-        const float exl = __fmul_rn(lo, ri), exh = __fmul_rn(hi, ri);
-        const float ewl = __fmul_rn(wl, sj), ewh = __fmul_rn(wh, sj);
-        a.xlo = fminf(a.xlo, lo); a.xhi = fmaxf(a.xhi, hi);
-        a.wlo = fminf(a.wlo, wl); a.whi = fmaxf(a.whi, wh);
-        a.exlo = fminf(a.exlo, exl); a.exhi = fmaxf(a.exhi, exh);
-        a.ewlo = fminf(a.ewlo, ewl); a.ewhi = fmaxf(a.ewhi, ewh);
-        a.mrx = fmaxf(a.mrx, rx); a.mrw = fmaxf(a.mrw, rw);
-        a.merx = fmaxf(a.merx, exh - exl); a.merw = fmaxf(a.merw, ewh - ewl);
+    for (int q = threadIdx.x; q < nquad; q += kFacThreads) {
+        const float4 lo = ldg_f4(xmin + 4 * q), hi = ldg_f4(xmax + 4 * q), me = ldg_f4(xmean + 4 * q);
+        const float4 wl = ldg_f4(wmin + 4 * q), wh = ldg_f4(wmax + 4 * q);
+        const FacOut o0 = fac_channel(lo.x, hi.x, me.x, wl.x, wh.x, a, dead);
+        const FacOut o1 = fac_channel(lo.y, hi.y, me.y, wl.y, wh.y, a, dead);
+        const FacOut o2 = fac_channel(lo.z, hi.z, me.z, wl.z, wh.z, a, dead);
+        const FacOut o3 = fac_channel(lo.w, hi.w, me.w, wl.w, wh.w, a, dead);
+        *reinterpret_cast<float4 *>(s + 4 * q) = make_float4(o0.s, o1.s, o2.s, o3.s);
+        *reinterpret_cast<float4 *>(rinv + 4 * q) = make_float4(o0.rinv, o1.rinv, o2.rinv, o3.rinv);
+        *reinterpret_cast<float4 *>(mu_hat + 4 * q) = make_float4(o0.mu, o1.mu, o2.mu, o3.mu);
+    }
+    for (int j = 4 * nquad + threadIdx.x; j < C; j += kFacThreads) {
+        const FacOut o = fac_channel(xmin[j], xmax[j], xmean[j], wmin[j], wmax[j], a, dead);
+        s[j] = o.s;
+        rinv[j] = o.rinv;
+        mu_hat[j] = o.mu;
     }
     // block reduction of the twelve extremes
     const uint32_t full = 0xffffffffu;
@@ -87,23 +134,33 @@ factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, c
         FacRed t = red[0];
         for (int k = 1; k < kFacThreads / 32; ++k) fac_merge(t, red[k]);
         total = t;
+        if (st && dead_count) atomicAdd(&st->zero_range, (unsigned long long)dead_count);
     }
+    if (!pX && !pW && !scalars) return;
     __syncthreads();
     const FacRed t = total;
     const double RX = (double)t.xhi - (double)t.xlo, RW = (double)t.whi - (double)t.wlo;
     const double EX = (double)t.exhi - (double)t.exlo, EW = (double)t.ewhi - (double)t.ewlo;
+    const double iRX = 1.0 / RX, iRW = 1.0 / RW, iEX = 1.0 / EX, iEW = 1.0 / EW;
 
     double o0 = 0.0, o1 = 0.0;
-    for (int j = threadIdx.x; j < C; j += kFacThreads) {
-        const double rx = (double)__fsub_rn(xmax[j], xmin[j]);
-        const double rw = (double)__fsub_rn(wmax[j], wmin[j]);
-        const float sj = s[j], ri = rinv[j];
-        const double erx = (double)__fmul_rn(xmax[j], ri) - (double)__fmul_rn(xmin[j], ri);
-        const double erw = (double)__fmul_rn(wmax[j], sj) - (double)__fmul_rn(wmin[j], sj);
-        if (pX) pX[j] = (float)(rx / RX);
-        if (pW) pW[j] = (float)(rw / RW);
-        o0 += (rx / RX) * (rw / RW);
-        o1 += (erx / EX) * (erw / EW);
+    for (int q = threadIdx.x; q < nquad; q += kFacThreads) {
+        const float4 lo = ldg_f4(xmin + 4 * q), hi = ldg_f4(xmax + 4 * q);
+        const float4 wl = ldg_f4(wmin + 4 * q), wh = ldg_f4(wmax + 4 * q);
+        const float4 sj = *reinterpret_cast<const float4 *>(s + 4 * q), ri = *reinterpret_cast<const float4 *>(rinv + 4 * q);
+        float4 px, pw;
+        fac_precision(lo.x, hi.x, wl.x, wh.x, sj.x, ri.x, iRX, iRW, iEX, iEW, px.x, pw.x, o0, o1);
+        fac_precision(lo.y, hi.y, wl.y, wh.y, sj.y, ri.y, iRX, iRW, iEX, iEW, px.y, pw.y, o0, o1);
+        fac_precision(lo.z, hi.z, wl.z, wh.z, sj.z, ri.z, iRX, iRW, iEX, iEW, px.z, pw.z, o0, o1);
+        fac_precision(lo.w, hi.w, wl.w, wh.w, sj.w, ri.w, iRX, iRW, iEX, iEW, px.w, pw.w, o0, o1);
+        if (pX) *reinterpret_cast<float4 *>(pX + 4 * q) = px;
+        if (pW) *reinterpret_cast<float4 *>(pW + 4 * q) = pw;
+    }
+    for (int j = 4 * nquad + threadIdx.x; j < C; j += kFacThreads) {
+        float px, pw;
+        fac_precision(xmin[j], xmax[j], wmin[j], wmax[j], s[j], rinv[j], iRX, iRW, iEX, iEW, px, pw, o0, o1);
+        if (pX) pX[j] = px;
+        if (pW) pW[j] = pw;
     }
     if (scalars) {
 #pragma unroll
@@ -128,7 +185,6 @@ factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, c
             scalars[7] = (double)t.merx * (double)t.merw;
         }
     }
-    if (threadIdx.x == 0 && st && dead_count) atomicAdd(&st->zero_range, (unsigned long long)dead_count);
 }
 
 aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean, const float *wmin,

@@ -4,6 +4,7 @@
 #include <stddef.h>
 
 #include "../../include/aweq.h"
+#include "common.cuh"
 
 namespace aweq {
 
@@ -20,11 +21,12 @@ aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean
 bool rowquant_supported(long long nrows, long long cols);
 aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
                          const float *scale, const float *mu, int bits, bool weights, unsigned char *out,
-                         float *step, int *zp, float *epsmu, aweq_dev_status *st, cudaStream_t stream);
+                         float *step, int *zp, float *epsmu, const BiasIO &bias, aweq_dev_status *st,
+                         cudaStream_t stream);
 aweq_status run_warpquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
                           const float *scale, const float *mu, int bits, bool weights, int group,
                           const float *lo_hi, unsigned char *out, float *step, int *zp, float *epsmu,
-                          aweq_dev_status *st, cudaStream_t stream);
+                          const BiasIO &bias, aweq_dev_status *st, cudaStream_t stream);
 aweq_status run_scaled_tensor_range(const float *cmin, const float *cmax, const float *scale, long long C,
                                     float *lo_hi, cudaStream_t stream);
 aweq_status run_bias_apply(const float *epsmu, const void *bias_in, void *bias_out, float *bias_out_f32,

@@ -38,6 +38,7 @@ struct RowQuantParams {
     float *step;
     int *zp;
     float *epsmu;
+    BiasIO bias;             // when out / out_f32 is set, the corrected bias is written with epsmu
     int bits;
     int team;             // threads per row (multiple of 32, divides NT)
     int rows_per_stage;
@@ -269,9 +270,13 @@ rowquant_kernel(const RowQuantParams p)
                             float tot = 0.0f;
                             for (int w2 = 0; w2 < wpt; ++w2) tot += sm->rsum[parity][tw0 + w2];
                             p.epsmu[row] = tot;
+                            if (p.bias.out || p.bias.out_f32)
+                                write_bias(row, tot, p.bias.in, p.bias.out, p.bias.out_f32, p.bias.bf16);
                         }
                     } else if (lane == 0) {
                         p.epsmu[row] = eacc;
+                        if (p.bias.out || p.bias.out_f32)
+                            write_bias(row, eacc, p.bias.in, p.bias.out, p.bias.out_f32, p.bias.bf16);
                     }
                 }
                 parity ^= 1;
@@ -378,7 +383,8 @@ bool rowquant_supported(long long nrows, long long cols)
 // weights == true: packed bit stream + optional eps.mu sums; false: one byte per code
 aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
                          const float *scale, const float *mu, int bits, bool weights, unsigned char *out,
-                         float *step, int *zp, float *epsmu, aweq_dev_status *st, cudaStream_t stream)
+                         float *step, int *zp, float *epsmu, const BiasIO &bias, aweq_dev_status *st,
+                         cudaStream_t stream)
 {
     RowQuantPlan pl;
     if (!plan_rowquant(nrows, cols, &pl)) return AWEQ_ERR_SHAPE;
@@ -387,7 +393,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     p.nrows = nrows; p.ld = ld; p.nvec = (int)(cols / 8);
     p.scale = scale; p.mu = mu; p.out = out;
     p.out_pitch = weights ? cols * bits / 8 : cols;
-    p.step = step; p.zp = zp; p.epsmu = epsmu; p.bits = bits;
+    p.step = step; p.zp = zp; p.epsmu = epsmu; p.bits = bits; p.bias = bias;
     p.team = pl.team; p.rows_per_stage = pl.rows_per_stage; p.stages = pl.stages; p.ntiles = pl.ntiles;
     p.st = st;
     const bool has_mu = weights && mu && epsmu;
