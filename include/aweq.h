@@ -57,7 +57,8 @@ typedef enum {
     AWEQ_ERR_GROUP = 6,       /* group size not a power of two in [8, 256] or not dividing C_in */
     AWEQ_ERR_WORKSPACE = 7,   /* ws is NULL, misaligned or smaller than aweq_workspace_bytes */
     AWEQ_ERR_CUDA = 8,        /* a CUDA call failed; see aweq_last_cuda_error */
-    AWEQ_ERR_UNSUPPORTED = 9
+    AWEQ_ERR_UNSUPPORTED = 9,
+    AWEQ_ERR_LIMIT = 10       /* size beyond the built-in scratch of aweq_stats_static */
 } aweq_status;
 
 typedef enum { AWEQ_F16 = 0, AWEQ_BF16 = 1 } aweq_dtype;
@@ -117,6 +118,29 @@ aweq_status aweq_stats(const void *X, aweq_dtype dt, long long N, long long C_in
                        float *xmin, float *xmax, float *xmean,
                        double *xsum, long long *count, int accumulate,
                        void *ws, size_t ws_bytes, aweq_dev_status *st, void *stream);
+
+/*
+ * Step 1 for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of aweq_stats, same kernels, same
+ * results.)  Some callers have no way to provide `ws`: code running inside a
+ * framework whose allocator they must not touch, plug-ins that are handed
+ * tensors but no allocation service, or a latency-critical section where a
+ * cudaMalloc (which synchronises the device) is not acceptable.  For them the
+ * scratch is a fixed array inside the library image: about 4.6 MiB of device
+ * memory on every GPU that loads the library, held until the process exits.
+ * Limits: C_in <= 16384 (a multiple of 8); N >= 1; no running state (no
+ * accumulate).  Anything larger returns AWEQ_ERR_LIMIT and enqueues nothing.
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  The call
+ * allocates and frees nothing.  All calls on a device share the one array, and
+ * it keeps what the last call left there: nothing in it has to be cleared,
+ * because each call writes every partial it later reads, but two calls whose
+ * kernels may overlap on the GPU (different streams, no ordering between them)
+ * would overwrite each other's partials -- order such calls yourself.
+ * Other arguments and results as for aweq_stats.
+ */
+aweq_status aweq_stats_static(const void *X, aweq_dtype dt, long long N, long long C_in, long long ldx,
+                              float *xmin, float *xmax, float *xmean, aweq_dev_status *st, void *stream);
 
 /*
  * Step 2 -- per-input-channel weight range (Section 3.2, same definition

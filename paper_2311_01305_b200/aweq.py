@@ -61,6 +61,8 @@ _lib.aweq_launch_count.restype = ctypes.c_ulonglong
 _lib.aweq_workspace_bytes.restype = _sz
 _lib.aweq_workspace_bytes.argtypes = [_i, _ll, _ll, _i, _i, _i]
 _lib.aweq_stats.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _vp, _vp, _vp, _i, _vp, _sz, _vp, _vp]
+_lib.aweq_stats_static.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _vp, _vp, _vp]
+_lib.aweq_stats_static.restype = _i
 _lib.aweq_wrange.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _i, _vp, _sz, _vp, _vp]
 _lib.aweq_factors.argtypes = [_vp, _vp, _vp, _vp, _vp, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.aweq_equalize_quantize.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz,
@@ -152,6 +154,13 @@ def aweq_stats(X, xmin, xmax, xmean, xsum=None, count=None, accumulate=False, ws
     _check(_lib.aweq_stats(_ptr(X), dtype_tag(X), n, X.shape[1], _ld(X), _ptr(xmin), _ptr(xmax), _ptr(xmean),
                            _ptr(xsum), _ptr(count), int(accumulate), _ptr(ws), 0 if ws is None else ws.numel(),
                            _ptr(st), _stream()))
+
+
+def aweq_stats_static(X, xmin, xmax, xmean, st=None):
+    """Step 1 with the library's built-in scratch: for callers that cannot allocate
+    device memory (no ``ws`` argument; C_in <= 16384).  Same results as aweq_stats."""
+    _check(_lib.aweq_stats_static(_ptr(X), dtype_tag(X), X.shape[0], X.shape[1], _ld(X), _ptr(xmin), _ptr(xmax),
+                                  _ptr(xmean), _ptr(st), _stream()))
 
 
 def aweq_wrange(W, wmin, wmax, accumulate=False, ws=None, st=None):

@@ -79,6 +79,7 @@ const char *aweq_strerror(aweq_status code)
     case AWEQ_ERR_WORKSPACE: return "workspace missing, misaligned (256 bytes) or too small";
     case AWEQ_ERR_CUDA: return "a CUDA call failed";
     case AWEQ_ERR_UNSUPPORTED: return "unsupported mode";
+    case AWEQ_ERR_LIMIT: return "size beyond the built-in scratch of aweq_stats_static (C_in <= 16384)";
     }
     return "unknown status";
 }

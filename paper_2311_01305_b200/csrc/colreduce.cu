@@ -21,6 +21,8 @@
 // values per column, which is widened to binary64 once at the end.  Each CTA writes one partial per column; a second small
 // kernel reduces the partials over the splits in a fixed order, so results are
 // bit-reproducible from run to run.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace aweq {
@@ -400,3 +402,58 @@ aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long 
 }
 
 }  // namespace aweq
+
+// ------------------------------------------------------------------ statistics without caller scratch
+// Scratch for aweq_stats_static: the per-split partials of one call.  It lives in
+// the library image, so every GPU that loads the library holds these bytes until
+// the process exits.  The partials need (row splits) x C_in x 16 bytes and the
+// number of row splits is at most 148 / ceil(C_in / 2048), so 148 x 2048 x 16
+// bytes cover every supported width.
+namespace aweq {
+constexpr size_t kStaticScratchBytes = (size_t)kColTargetCtas * kColThreads * 8 * 16 + 256;
+constexpr long long kStaticMaxCin = 16384;
+constexpr int kMaxDevices = 64;
+}  // namespace aweq
+static __device__ __align__(256) unsigned char g_stats_static_scratch[aweq::kStaticScratchBytes];
+
+namespace aweq {
+// Device address of the scratch array on the current device.  The array's name is
+// only a host-side handle in host code; the address a kernel can use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static aweq_status static_scratch_address(void **out)
+{
+    static std::mutex lock;
+    static void *address[kMaxDevices] = {};
+    int dev = -1;
+    AWEQ_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return AWEQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> guard(lock);
+    if (!address[dev]) {
+        void *p = nullptr;
+        AWEQ_CUDA_OK(cudaGetSymbolAddress(&p, g_stats_static_scratch));
+        address[dev] = p;
+    }
+    *out = address[dev];
+    return AWEQ_OK;
+}
+}  // namespace aweq
+
+extern "C" aweq_status aweq_stats_static(const void *X, aweq_dtype dt, long long N, long long C_in, long long ldx,
+                                         float *xmin, float *xmax, float *xmean, aweq_dev_status *st, void *stream)
+{
+    using namespace aweq;
+    if (!X || !xmin || !xmax || !xmean) return AWEQ_ERR_NULL;
+    if (dt != AWEQ_F16 && dt != AWEQ_BF16) return AWEQ_ERR_DTYPE;
+    if (C_in <= 0 || (C_in % 8) != 0 || N <= 0 || N > (1ll << 40)) return AWEQ_ERR_SHAPE;
+    if (C_in > kStaticMaxCin || colreduce_ws_bytes(N, C_in) > kStaticScratchBytes) return AWEQ_ERR_LIMIT;
+    if (ldx < C_in || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0) return AWEQ_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(xmin) & 15) != 0 || (reinterpret_cast<uintptr_t>(xmax) & 15) != 0)
+        return AWEQ_ERR_ALIGN;
+    void *scratch = nullptr;
+    aweq_status rc = static_scratch_address(&scratch);
+    if (rc != AWEQ_OK) return rc;
+    // every partial the reduction reads is written by this call first, so the
+    // contents left by an earlier call need no clearing
+    return run_stats(X, dt, N, C_in, ldx, xmin, xmax, xmean, nullptr, nullptr, 0, scratch, st, (cudaStream_t)stream);
+}
+
