@@ -58,12 +58,12 @@ ColPlan plan_colreduce(long long rows, long long cols)
     p.slab_w = (p.nvec + p.nslab - 1) / p.nslab;
     int nsplit = kColTargetCtas / p.nslab;
     if (nsplit < 1) nsplit = 1;
-    long long max_split = (rows + kColRows - 1) / kColRows;
+    long long max_split = (rows + 7) / 8;
     if (max_split < 1) max_split = 1;
     if (nsplit > max_split) nsplit = (int)max_split;
     long long rps = (rows + nsplit - 1) / nsplit;
-    rps = (rps + kColRows - 1) / kColRows * kColRows;
-    if (rps < kColRows) rps = kColRows;
+    rps = (rps + 7) / 8 * 8;            // whole eight-row groups; the last stage of a split may be partial
+    if (rps < 8) rps = 8;
     p.rows_per_split = rps;
     p.nsplit = (int)((rows + rps - 1) / rps);
     if (p.nsplit < 1) p.nsplit = 1;

@@ -203,12 +203,14 @@ __device__ __forceinline__ QParams make_qparams(float lo, float hi, int qmax)
     float st = __fdiv_rn(__fsub_rn(hi, lo), (float)qmax);
     if (!(st > 0.0f)) st = (lo != 0.0f) ? fabsf(lo) : 1.0f;      // constant vector
     p.step = st;
-    p.inv = __fdiv_rn(1.0f, st);
-    float z = __fmul_rn(lo, p.inv);
+    p.inv = __frcp_rn(st);                                       // correctly rounded 1 / Step
+    const float z = __fmul_rn(lo, p.inv);
     int zi;
     asm("cvt.rni.sat.s32.f32 %0, %1;" : "=r"(zi) : "f"(-z));    // saturating; NaN -> 0
     p.zp = zi;
-    p.fast = (zi > -(1 << 21)) && (zi < (1 << 21)) && (fabsf(p.inv) <= 3.0e38f) && (fabsf(z) < 4.0e6f);
+    // |lo / Step| < 4e6 keeps every clamped value below 2^22, where adding 1.5 * 2^23 rounds
+    // exactly like rint; an infinite 1 / Step makes z infinite or NaN and fails the test
+    p.fast = fabsf(z) < 4.0e6f;
     return p;
 }
 // exact reference form of one code: clamp(rint(fl(v*inv)) + Z, 0, qmax) with saturating int32

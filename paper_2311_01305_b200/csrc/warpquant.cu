@@ -38,6 +38,7 @@ struct WarpQuantParams {
     BiasIO bias;             // when out / out_f32 is set, the corrected bias is written with epsmu
     int bits;
     int lanes_per_group;        // group / 8 (group mode)
+    int log2_lanes;             // log2 of it
     int ngroups;                // groups per row (group mode)
     const float *lo_hi;         // static mode: device float[2]
     aweq_dev_status *st;
@@ -51,11 +52,10 @@ constexpr int kQNoClamp = 2;    // the upper clamp cannot fire
 
 __device__ __forceinline__ int qflags(const QParams &q, float hi, int qmax)
 {
-    int f = q.fast ? kQFast : 0;
     int top;
     asm("cvt.rni.sat.s32.f32 %0, %1;" : "=r"(top) : "f"(__fmul_rn(hi, q.inv)));
-    if (q.fast && (long long)top + (long long)q.zp <= (long long)qmax) f |= kQNoClamp;
-    return f;
+    // with q.fast both terms are below 2^22 in magnitude: no overflow
+    return q.fast ? (kQFast | ((top + q.zp <= qmax) ? kQNoClamp : 0)) : 0;
 }
 
 // store the codes u[i] + K of one vector; BITS == 0 means "runtime bits"
@@ -137,7 +137,9 @@ warpquant_kernel(const WarpQuantParams p)
     for (long long row = warp0; row < p.nrows; row += nwarps) {
         const uint16_t *xrow = p.X + row * p.ld;
         unsigned char *orow = p.out + row * p.out_pitch;
-        float2 eacc = make_float2(0.0f, 0.0f);
+        float *step_row = STATIC ? p.step : p.step + row * p.ngroups;
+        int *zp_row = STATIC ? p.zp : p.zp + row * p.ngroups;
+        float2 eneg = make_float2(0.0f, 0.0f);                 // minus the running eps . mu sum
         uint4 nxt = lane < p.nvec ? ldg_stream(xrow + (size_t)lane * 8) : make_uint4(0, 0, 0, 0);
         for (int it = 0; it < nsteps; ++it) {
             const int idx = it * 32 + lane;
@@ -181,9 +183,8 @@ warpquant_kernel(const WarpQuantParams p)
                 q = make_qparams(a, b, qmax);
                 fl = qflags(q, b, qmax);
                 if (active && (lane & (L - 1)) == 0) {
-                    const long long g = row * p.ngroups + idx / L;
-                    p.step[g] = q.step;
-                    p.zp[g] = q.zp;
+                    step_row[idx >> p.log2_lanes] = q.step;
+                    zp_row[idx >> p.log2_lanes] = q.zp;
                 }
             }
             const bool all_lean = __all_sync(0xffffffffu, !active || fl == (kQFast | kQNoClamp));
@@ -192,7 +193,7 @@ warpquant_kernel(const WarpQuantParams p)
             if (all_lean) {
                 K = (uint32_t)(q.zp - kMagicBits);
                 const float2 inv2 = make_float2(q.inv, q.inv);
-                const float2 step2 = make_float2(q.step, q.step);
+                const float2 nstep2 = make_float2(-q.step, -q.step);
                 const float hic = (float)(qmax - q.zp), loc = (float)(-q.zp);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
@@ -210,8 +211,8 @@ warpquant_kernel(const WarpQuantParams p)
                     u[2 * k + 1] = __float_as_uint(uf.y);
                     if (MU) {
                         const float2 rq = __fadd2_rn(uf, nmagic2);                 // q - Z, exact
-                        const float2 eps = __ffma2_rn(step2, rq, make_float2(-w2[k].x, -w2[k].y));
-                        eacc = __ffma2_rn(eps, make_float2(mu8[2 * k], mu8[2 * k + 1]), eacc);
+                        const float2 neps = __ffma2_rn(nstep2, rq, w2[k]);         // -(Step (q - Z) - w^)
+                        eneg = __ffma2_rn(neps, make_float2(mu8[2 * k], mu8[2 * k + 1]), eneg);
                     }
                 }
             } else {
@@ -223,15 +224,15 @@ warpquant_kernel(const WarpQuantParams p)
                     u[2 * k + 1] = (uint32_t)c1;
                     if (MU) {
                         const float r0 = (float)((long long)c0 - (long long)q.zp), r1 = (float)((long long)c1 - (long long)q.zp);
-                        eacc.x = __fmaf_rn(__fmaf_rn(q.step, r0, -w2[k].x), mu8[2 * k], eacc.x);
-                        eacc.y = __fmaf_rn(__fmaf_rn(q.step, r1, -w2[k].y), mu8[2 * k + 1], eacc.y);
+                        eneg.x = __fmaf_rn(__fmaf_rn(-q.step, r0, w2[k].x), mu8[2 * k], eneg.x);
+                        eneg.y = __fmaf_rn(__fmaf_rn(-q.step, r1, w2[k].y), mu8[2 * k + 1], eneg.y);
                     }
                 }
             }
             store_vec<BITS, BYTES_OUT>(orow, idx, u, K, bits, active, quad3, lane);
         }
         if (MU) {
-            const float tot = warp_sum(__fadd_rn(eacc.x, eacc.y));
+            const float tot = -warp_sum(__fadd_rn(eneg.x, eneg.y));
             if (lane == 0) {
                 p.epsmu[row] = tot;
                 if (p.bias.out || p.bias.out_f32) write_bias(row, tot, p.bias.in, p.bias.out, p.bias.out_f32, p.bias.bf16);
@@ -313,6 +314,8 @@ aweq_status run_warpquant(const void *X, aweq_dtype dt, long long nrows, long lo
     p.out_pitch = weights ? cols * bits / 8 : cols;
     p.step = step; p.zp = zp; p.epsmu = epsmu; p.bits = bits; p.bias = bias;
     p.lanes_per_group = group > 0 ? group / 8 : 32;
+    p.log2_lanes = 0;
+    while ((1 << p.log2_lanes) < p.lanes_per_group) ++p.log2_lanes;
     p.ngroups = group > 0 ? (int)(cols / group) : 1;
     p.lo_hi = lo_hi; p.st = st;
     const bool has_mu = weights && mu && epsmu;
