@@ -221,6 +221,18 @@ __device__ __forceinline__ int code_generic(float v, float inv, int zp, int qmax
     asm("add.sat.s32 %0, %1, %2;" : "=r"(q) : "r"(t), "r"(zp));
     return min(max(q, 0), qmax);
 }
+// flags travelling with a (Step, inv, Z) triple
+constexpr int kQFast = 1;       // add-constant rounding is valid
+constexpr int kQNoClamp = 2;    // the upper clamp cannot fire
+
+__device__ __forceinline__ int qflags(const QParams &q, float hi, int qmax)
+{
+    int top;
+    asm("cvt.rni.sat.s32.f32 %0, %1;" : "=r"(top) : "f"(__fmul_rn(hi, q.inv)));
+    // with q.fast both terms are below 2^22 in magnitude: no overflow
+    return q.fast ? (kQFast | ((top + q.zp <= qmax) ? kQNoClamp : 0)) : 0;
+}
+
 constexpr float kMagic = 12582912.0f;            // 1.5 * 2^23: adding it rounds to an integer, ties to even
 constexpr int kMagicBits = 0x4B400000;
 

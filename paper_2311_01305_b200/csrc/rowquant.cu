@@ -14,12 +14,13 @@
 // and Z are then computed redundantly by every thread and the codes are formed
 // from the registers and stored with coalesced 8-byte (or b-byte) stores.
 //
-// Rounding uses the add-magic trick (adding 1.5 * 2^23 in binary32 rounds to an
-// integer, ties to even), with the upper clamp applied before rounding; both
-// commute with the reference order clamp(rint(t) + Z) because the bounds are
-// integers.  The lower clamp cannot fire when Step and Z come from the same
-// vector (t >= fl(lo * inv) implies rint(t) >= -Z).  Rows whose zero-point is
-// too large for that trick take the literal cvt.rni path.
+// Rounding adds 1.5 * 2^23 in binary32 (rounds to an integer, ties to even, like
+// rint).  The lower clamp of Eq. 1 cannot fire when Step and Z come from the
+// same vector (t >= fl(lo * inv) implies rint(t) >= -Z); the upper clamp can only
+// fire when rint(hi * inv) + Z exceeds 2^b - 1, which is decided once per row.
+// Rows where it does, and rows whose zero-point is too large for the rounding
+// trick, take the literal cvt.rni path.  Multiplies, the rounding add and the
+// eps . E[x^] terms use the packed binary32 instructions of sm_100.
 #include "common.cuh"
 
 namespace aweq {
@@ -162,6 +163,23 @@ rowquant_kernel(const RowQuantParams p)
         const int tw0 = tm * wpt;                     // first warp of my team
         int parity = 0;
         bool ok = true;
+        // a thread keeps the same columns for every row: their scale factors live in registers
+        constexpr bool SC_REGS = SCALE && V <= 4;
+        float2 sc[SC_REGS ? V : 1][4];
+        if (SC_REGS) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                const int idx = tt + v * T;
+                if (idx < p.nvec) {
+                    const float4 s0 = ldg_f4(p.scale + (size_t)idx * 8), s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
+                    sc[v][0] = make_float2(s0.x, s0.y); sc[v][1] = make_float2(s0.z, s0.w);
+                    sc[v][2] = make_float2(s1.x, s1.y); sc[v][3] = make_float2(s1.z, s1.w);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) sc[v][k] = make_float2(1.0f, 1.0f);
+                }
+            }
+        }
         for (long long k = 0; k < my_tiles; ++k) {
             const int s = (int)(k % S);
             const uint32_t use = (uint32_t)(k / S);
@@ -174,25 +192,33 @@ rowquant_kernel(const RowQuantParams p)
             const uint4 *tile = stage_base + (size_t)s * stage_vecs;
             for (int r = tm; r < rows; r += teams) {
                 const uint4 *rowp = tile + (size_t)r * p.nvec;
-                float xh[V][8];
+                float2 xh[V][4];
                 float lo = INFINITY, hi = -INFINITY;
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     const int idx = tt + v * T;
                     if (idx < p.nvec) {
                         const uint4 raw = rowp[idx];
-                        widen8<D>(raw, xh[v]);
+                        xh[v][0] = D::to_float2(D::from_bits(raw.x));
+                        xh[v][1] = D::to_float2(D::from_bits(raw.y));
+                        xh[v][2] = D::to_float2(D::from_bits(raw.z));
+                        xh[v][3] = D::to_float2(D::from_bits(raw.w));
                         if (SCALE) {
-                            float sc[8];
-                            load8(p.scale + (size_t)idx * 8, sc);
+                            if (SC_REGS) {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) xh[v][e] = __fmul_rn(xh[v][e], sc[e]);
+                                for (int k = 0; k < 4; ++k) xh[v][k] = __fmul2_rn(xh[v][k], sc[v][k]);
+                            } else {
+                                const float4 s0 = ldg_f4(p.scale + (size_t)idx * 8), s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
+                                xh[v][0] = __fmul2_rn(xh[v][0], make_float2(s0.x, s0.y));
+                                xh[v][1] = __fmul2_rn(xh[v][1], make_float2(s0.z, s0.w));
+                                xh[v][2] = __fmul2_rn(xh[v][2], make_float2(s1.x, s1.y));
+                                xh[v][3] = __fmul2_rn(xh[v][3], make_float2(s1.z, s1.w));
+                            }
                         }
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            lo = fminf(lo, xh[v][e]);
-                            hi = fmaxf(hi, xh[v][e]);
-                        }
+                        lo = fminf(fminf(lo, xh[v][0].x), xh[v][0].y); hi = fmaxf(fmaxf(hi, xh[v][0].x), xh[v][0].y);
+                        lo = fminf(fminf(lo, xh[v][1].x), xh[v][1].y); hi = fmaxf(fmaxf(hi, xh[v][1].x), xh[v][1].y);
+                        lo = fminf(fminf(lo, xh[v][2].x), xh[v][2].y); hi = fmaxf(fmaxf(hi, xh[v][2].x), xh[v][2].y);
+                        lo = fminf(fminf(lo, xh[v][3].x), xh[v][3].y); hi = fmaxf(fmaxf(hi, xh[v][3].x), xh[v][3].y);
                     }
                 }
                 lo = redux_min(lo, 0xffffffffu);
@@ -207,6 +233,7 @@ rowquant_kernel(const RowQuantParams p)
                     }
                 }
                 const QParams q = make_qparams(lo, hi, qmax);
+                const int fl = qflags(q, hi, qmax);
                 const long long row = row0 + r;
                 if (tt == 0) {
                     p.step[row] = q.step;
@@ -214,10 +241,13 @@ rowquant_kernel(const RowQuantParams p)
                 }
                 unsigned char *orow = p.out + row * p.out_pitch;
                 const int vec_bytes = BYTES_OUT ? 8 : p.bits;
-                float eacc = 0.0f;
-                if (q.fast) {
-                    const float hic = (float)(qmax - q.zp);
+                float2 eneg = make_float2(0.0f, 0.0f);            // minus the eps . mu partial sum
+                if (fl == (kQFast | kQNoClamp)) {
+                    // lean path: no clamp can fire in this row; packed multiply and rounding add
                     const uint32_t K = (uint32_t)(q.zp - kMagicBits);
+                    const float2 inv2 = make_float2(q.inv, q.inv), nstep2 = make_float2(-q.step, -q.step);
+                    const float2 magic2 = make_float2(kMagic, kMagic), nmagic2 = make_float2(-kMagic, -kMagic);
+                    const float2 one2 = make_float2(1.0f, 1.0f);
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
                         const int idx = tt + v * T;
@@ -226,14 +256,17 @@ rowquant_kernel(const RowQuantParams p)
                             float mu8[8];
                             if (MU) load8(p.mu + (size_t)idx * 8, mu8);
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const float t = fminf(__fmul_rn(xh[v][e], q.inv), hic);
-                                const float uf = __fadd_rn(t, kMagic);
-                                u[e] = __float_as_uint(uf);
+                            for (int k = 0; k < 4; ++k) {
+                                const float2 t = __fmul2_rn(xh[v][k], inv2);
+                                // t * 1 + magic as one FMA: equal to t + magic, and it cannot be
+                                // contracted with the multiply above (which would change ties)
+                                const float2 uf = __ffma2_rn(t, one2, magic2);
+                                u[2 * k] = __float_as_uint(uf.x);
+                                u[2 * k + 1] = __float_as_uint(uf.y);
                                 if (MU) {
-                                    const float rq = __fsub_rn(uf, kMagic);          // q - Z, exact
-                                    const float eps = __fmaf_rn(q.step, rq, -xh[v][e]);
-                                    eacc = __fmaf_rn(eps, mu8[e], eacc);
+                                    const float2 rq = __fadd2_rn(uf, nmagic2);              // q - Z, exact
+                                    const float2 neps = __ffma2_rn(nstep2, rq, xh[v][k]);   // -(Step (q - Z) - v^)
+                                    eneg = __ffma2_rn(neps, make_float2(mu8[2 * k], mu8[2 * k + 1]), eneg);
                                 }
                             }
                             store_codes(orow + (size_t)idx * vec_bytes, u, K, p.bits, BYTES_OUT);
@@ -248,13 +281,16 @@ rowquant_kernel(const RowQuantParams p)
                             float mu8[8];
                             if (MU) load8(p.mu + (size_t)idx * 8, mu8);
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const int c = code_generic(xh[v][e], q.inv, q.zp, qmax);
-                                u[e] = (uint32_t)c;
+                            for (int k = 0; k < 4; ++k) {
+                                const int c0 = code_generic(xh[v][k].x, q.inv, q.zp, qmax);
+                                const int c1 = code_generic(xh[v][k].y, q.inv, q.zp, qmax);
+                                u[2 * k] = (uint32_t)c0;
+                                u[2 * k + 1] = (uint32_t)c1;
                                 if (MU) {
-                                    const float rq = (float)((long long)c - (long long)q.zp);
-                                    const float eps = __fmaf_rn(q.step, rq, -xh[v][e]);
-                                    eacc = __fmaf_rn(eps, mu8[e], eacc);
+                                    const float r0 = (float)((long long)c0 - (long long)q.zp);
+                                    const float r1 = (float)((long long)c1 - (long long)q.zp);
+                                    eneg.x = __fmaf_rn(__fmaf_rn(-q.step, r0, xh[v][k].x), mu8[2 * k], eneg.x);
+                                    eneg.y = __fmaf_rn(__fmaf_rn(-q.step, r1, xh[v][k].y), mu8[2 * k + 1], eneg.y);
                                 }
                             }
                             store_codes(orow + (size_t)idx * vec_bytes, u, 0u, p.bits, BYTES_OUT);
@@ -262,7 +298,7 @@ rowquant_kernel(const RowQuantParams p)
                     }
                 }
                 if (MU) {
-                    eacc = warp_sum(eacc);
+                    const float eacc = -warp_sum(__fadd_rn(eneg.x, eneg.y));
                     if (wpt > 1) {
                         if (lane == 0) sm->rsum[parity][warp] = eacc;
                         named_bar_sync(1 + tm, T);

@@ -46,18 +46,6 @@ struct WarpQuantParams {
 
 constexpr int kWqWarps = 8;
 
-// flags travelling with a (Step, inv, Z) triple
-constexpr int kQFast = 1;       // add-constant rounding is valid
-constexpr int kQNoClamp = 2;    // the upper clamp cannot fire
-
-__device__ __forceinline__ int qflags(const QParams &q, float hi, int qmax)
-{
-    int top;
-    asm("cvt.rni.sat.s32.f32 %0, %1;" : "=r"(top) : "f"(__fmul_rn(hi, q.inv)));
-    // with q.fast both terms are below 2^22 in magnitude: no overflow
-    return q.fast ? (kQFast | ((top + q.zp <= qmax) ? kQNoClamp : 0)) : 0;
-}
-
 // store the codes u[i] + K of one vector; BITS == 0 means "runtime bits"
 template <int BITS, bool BYTES_OUT>
 __device__ __forceinline__ void store_vec(unsigned char *orow, int idx, const uint32_t (&u)[8], uint32_t K, int bits,
