@@ -1,358 +1,38 @@
-// Row-wise Eq. 1-2 quantiser with a per-column scale: the kernel behind
-// step 4 in per-output-channel mode (W^ = diag(s) W, Eq. 3, quantised per row)
-// and step 6 in per-token mode (X^ = X diag(s)^-1 quantised per token).
-//
-// Every row needs its own minimum and maximum before a single code can be
-// produced, so a row must be looked at twice while HBM should see it once.
-// The kernel keeps the scaled row on chip: persistent CTAs pull tiles of whole
-// rows through a ring of shared-memory stages with 1-D bulk copies (TMA,
-// completion on mbarriers, one dedicated producer warp); a team of T threads
-// owns one row of the stage at a time, each thread holding V 16-byte vectors of
-// the row, already multiplied by the column scale, in registers.  The row
-// extremes are reduced with redux.sync inside a warp and through a few words of
-// shared memory plus a named barrier across the warps of a team; Step, 1/Step
-// and Z are then computed redundantly by every thread and the codes are formed
-// from the registers and stored with coalesced 8-byte (or b-byte) stores.
-//
-// Rounding adds 1.5 * 2^23 in binary32 (rounds to an integer, ties to even, like
-// rint).  The lower clamp of Eq. 1 cannot fire when Step and Z come from the
-// same vector (t >= fl(lo * inv) implies rint(t) >= -Z); the upper clamp can only
-// fire when rint(hi * inv) + Z exceeds 2^b - 1, which is decided once per row.
-// Rows where it does, and rows whose zero-point is too large for the rounding
-// trick, take the literal cvt.rni path.  Multiplies, the rounding add and the
-// eps . E[x^] terms use the packed binary32 instructions of sm_100.
-#include "common.cuh"
+// Host side of the row quantiser: how a row is split over threads, how many rows
+// form a stage, and the dispatch to the fp16 / bf16 instantiations.
+#include "rowquant_impl.cuh"
 
 namespace aweq {
 
-constexpr int kRqStagesMax = 4;
-constexpr int kRqMaxV = 10;
-
-struct RowQuantParams {
-    const uint16_t *X;
-    long long nrows, ld;
-    int nvec;
-    const float *scale;
-    const float *mu;
-    unsigned char *out;
-    long long out_pitch;
-    float *step;
-    int *zp;
-    float *epsmu;
-    BiasIO bias;             // when out / out_f32 is set, the corrected bias is written with epsmu
-    int bits;
-    int team;             // threads per row (multiple of 32, divides NT)
-    int rows_per_stage;
-    int stages;
-    long long ntiles;
-    aweq_dev_status *st;
-};
-
-struct RqSmem {
-    uint64_t full[kRqStagesMax];
-    uint64_t empty[kRqStagesMax];
-    int abort_flag;
-    int pad[15];
-    float2 red[2][16];
-    float rsum[2][16];
-};
-constexpr int kRqHeader = 512;
-static_assert(sizeof(RqSmem) <= kRqHeader, "header");
-
-// pack eight values u[i] + K (each in [0, 2^b)) into the little-endian bit stream
-__device__ __forceinline__ void store_codes(unsigned char *dst, const uint32_t (&u)[8], uint32_t K, int bits, bool bytes_out)
+// Everything that happens once per row (exchange of the extremes, Step, 1/Step, Z) is
+// repeated by every warp of the row's team, and a thread's last vector may be padding, so
+// the cost of a row is about (T / 32) * (V * c_vec + c_row) issue slots.  Pick the team
+// size that minimises it with V <= kRqMaxV.
+static void pick_team(int nvec, int *T_out, int *V_out)
 {
-    if (bytes_out || bits == 8) {
-        const uint32_t kp = K * 0x01010101u;
-        uint2 w;
-        w.x = u[0] + (u[1] << 8) + (u[2] << 16) + (u[3] << 24) + kp;
-        w.y = u[4] + (u[5] << 8) + (u[6] << 16) + (u[7] << 24) + kp;
-        *reinterpret_cast<uint2 *>(dst) = w;
-    } else if (bits <= 4) {
-        uint32_t w = 0, m = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            w += u[i] << (i * bits);
-            m += 1u << (i * bits);
-        }
-        w += K * m;
-        if (bits == 4) {
-            *reinterpret_cast<uint32_t *>(dst) = w;
-        } else if (bits == 2) {
-            *reinterpret_cast<uint16_t *>(dst) = (uint16_t)w;
-        } else {
-            dst[0] = (unsigned char)w;
-            dst[1] = (unsigned char)(w >> 8);
-            dst[2] = (unsigned char)(w >> 16);
-        }
-    } else {
-        unsigned long long w = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) w |= (unsigned long long)((u[i] + K) & ((1u << bits) - 1)) << (i * bits);
-        for (int k = 0; k < bits; ++k) dst[k] = (unsigned char)(w >> (8 * k));
+    double best = 1e30;
+    int bestT = 0, bestV = 0;
+    for (int T = 32; T <= 512; T *= 2) {
+        const int V = (nvec + T - 1) / T;
+        if (V > kRqMaxV) continue;
+        const double c_vec = V <= kRqScaleRegsMaxV ? 55.0 : 59.0;
+        const double cost = (T / 32) * (V * c_vec + 90.0);
+        if (cost < best) { best = cost; bestT = T; bestV = V; }
     }
+    *T_out = bestT;
+    *V_out = bestV;
 }
-
-template <class D, int V, int NT, bool SCALE, bool MU, bool BYTES_OUT>
-__global__ void __launch_bounds__(NT + 32, (NT <= 256 && V <= 4) ? 2 : 1)
-rowquant_kernel(const RowQuantParams p)
-{
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    RqSmem *sm = reinterpret_cast<RqSmem *>(smem_raw);
-    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw + kRqHeader);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int T = p.team;
-    const int teams = NT / T;
-    const int R = p.rows_per_stage;
-    const int S = p.stages;
-    const size_t stage_vecs = (size_t)R * p.nvec;
-    const int qmax = (1 << p.bits) - 1;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(&sm->full[s], 1);
-            mbar_init(&sm->empty[s], NT / 32);
-        }
-        sm->abort_flag = 0;
-        mbar_init_fence();
-    }
-    __syncthreads();
-
-    // tiles of R rows, dealt round-robin to the persistent CTAs
-    const long long my_tiles = p.ntiles > blockIdx.x ? (p.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-
-    if (warp == NT / 32) {
-        // ---------------- producer warp
-        const bool contiguous = p.ld == (long long)p.nvec * 8;
-        bool ok = true;
-        for (long long k = 0; k < my_tiles && ok; ++k) {
-            const int s = (int)(k % S);
-            const uint32_t use = (uint32_t)(k / S);
-            if (use > 0) {
-                ok = mbar_wait(&sm->empty[s], (use - 1) & 1);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-            }
-            const long long row0 = (blockIdx.x + k * gridDim.x) * (long long)R;
-            const int rows = (int)min((long long)R, p.nrows - row0);
-            const uint32_t row_bytes = (uint32_t)p.nvec * 16u;
-            uint4 *dst = stage_base + (size_t)s * stage_vecs;
-            if (lane == 0) mbar_arrive_expect_tx(&sm->full[s], (uint32_t)rows * row_bytes);
-            __syncwarp();
-            if (contiguous) {
-                // one copy per <= 64 KB chunk of the contiguous tile
-                const uint32_t total = (uint32_t)rows * row_bytes;
-                const uint32_t chunk = 32768u;
-                const char *src = reinterpret_cast<const char *>(p.X + row0 * p.ld);
-                for (uint32_t off = lane * chunk; off < total; off += 32u * chunk)
-                    bulk_g2s(reinterpret_cast<char *>(dst) + off, src + off, min(chunk, total - off), &sm->full[s]);
-            } else {
-                for (int r = lane; r < rows; r += 32)
-                    bulk_g2s(dst + (size_t)r * p.nvec, p.X + (row0 + r) * p.ld, row_bytes, &sm->full[s]);
-            }
-        }
-        if (!ok && lane == 0) {
-            atomicExch(&sm->abort_flag, 1);
-            if (p.st) atomicAdd(&p.st->wait_timeout, 1ull);
-        }
-    } else {
-        // ---------------- consumer teams
-        const int tm = threadIdx.x / T, tt = threadIdx.x % T;
-        const int wpt = T / 32;                       // warps per team
-        const int tw0 = tm * wpt;                     // first warp of my team
-        int parity = 0;
-        bool ok = true;
-        // a thread keeps the same columns for every row: their scale factors live in registers
-        constexpr bool SC_REGS = SCALE && V <= 4;
-        float2 sc[SC_REGS ? V : 1][4];
-        if (SC_REGS) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int idx = tt + v * T;
-                if (idx < p.nvec) {
-                    const float4 s0 = ldg_f4(p.scale + (size_t)idx * 8), s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
-                    sc[v][0] = make_float2(s0.x, s0.y); sc[v][1] = make_float2(s0.z, s0.w);
-                    sc[v][2] = make_float2(s1.x, s1.y); sc[v][3] = make_float2(s1.z, s1.w);
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) sc[v][k] = make_float2(1.0f, 1.0f);
-                }
-            }
-        }
-        for (long long k = 0; k < my_tiles; ++k) {
-            const int s = (int)(k % S);
-            const uint32_t use = (uint32_t)(k / S);
-            ok = mbar_wait(&sm->full[s], use & 1) && !*reinterpret_cast<volatile int *>(&sm->abort_flag);
-            // the whole team leaves together, or a later team barrier would miss a warp
-            ok = wpt > 1 ? named_bar_and(1 + tm, T, ok) : __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            const long long row0 = (blockIdx.x + k * gridDim.x) * (long long)R;
-            const int rows = (int)min((long long)R, p.nrows - row0);
-            const uint4 *tile = stage_base + (size_t)s * stage_vecs;
-            for (int r = tm; r < rows; r += teams) {
-                const uint4 *rowp = tile + (size_t)r * p.nvec;
-                float2 xh[V][4];
-                float lo = INFINITY, hi = -INFINITY;
-#pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    const int idx = tt + v * T;
-                    if (idx < p.nvec) {
-                        const uint4 raw = rowp[idx];
-                        xh[v][0] = D::to_float2(D::from_bits(raw.x));
-                        xh[v][1] = D::to_float2(D::from_bits(raw.y));
-                        xh[v][2] = D::to_float2(D::from_bits(raw.z));
-                        xh[v][3] = D::to_float2(D::from_bits(raw.w));
-                        if (SCALE) {
-                            if (SC_REGS) {
-#pragma unroll
-                                for (int k = 0; k < 4; ++k) xh[v][k] = __fmul2_rn(xh[v][k], sc[v][k]);
-                            } else {
-                                const float4 s0 = ldg_f4(p.scale + (size_t)idx * 8), s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
-                                xh[v][0] = __fmul2_rn(xh[v][0], make_float2(s0.x, s0.y));
-                                xh[v][1] = __fmul2_rn(xh[v][1], make_float2(s0.z, s0.w));
-                                xh[v][2] = __fmul2_rn(xh[v][2], make_float2(s1.x, s1.y));
-                                xh[v][3] = __fmul2_rn(xh[v][3], make_float2(s1.z, s1.w));
-                            }
-                        }
-                        lo = fminf(fminf(lo, xh[v][0].x), xh[v][0].y); hi = fmaxf(fmaxf(hi, xh[v][0].x), xh[v][0].y);
-                        lo = fminf(fminf(lo, xh[v][1].x), xh[v][1].y); hi = fmaxf(fmaxf(hi, xh[v][1].x), xh[v][1].y);
-                        lo = fminf(fminf(lo, xh[v][2].x), xh[v][2].y); hi = fmaxf(fmaxf(hi, xh[v][2].x), xh[v][2].y);
-                        lo = fminf(fminf(lo, xh[v][3].x), xh[v][3].y); hi = fmaxf(fmaxf(hi, xh[v][3].x), xh[v][3].y);
-                    }
-                }
-                lo = redux_min(lo, 0xffffffffu);
-                hi = redux_max(hi, 0xffffffffu);
-                if (wpt > 1) {
-                    if (lane == 0) sm->red[parity][warp] = make_float2(lo, hi);
-                    named_bar_sync(1 + tm, T);
-                    for (int w2 = 0; w2 < wpt; ++w2) {
-                        const float2 o = sm->red[parity][tw0 + w2];
-                        lo = fminf(lo, o.x);
-                        hi = fmaxf(hi, o.y);
-                    }
-                }
-                const QParams q = make_qparams(lo, hi, qmax);
-                const int fl = qflags(q, hi, qmax);
-                const long long row = row0 + r;
-                if (tt == 0) {
-                    p.step[row] = q.step;
-                    p.zp[row] = q.zp;
-                }
-                unsigned char *orow = p.out + row * p.out_pitch;
-                const int vec_bytes = BYTES_OUT ? 8 : p.bits;
-                float2 eneg = make_float2(0.0f, 0.0f);            // minus the eps . mu partial sum
-                if (fl == (kQFast | kQNoClamp)) {
-                    // lean path: no clamp can fire in this row; packed multiply and rounding add
-                    const uint32_t K = (uint32_t)(q.zp - kMagicBits);
-                    const float2 inv2 = make_float2(q.inv, q.inv), nstep2 = make_float2(-q.step, -q.step);
-                    const float2 magic2 = make_float2(kMagic, kMagic), nmagic2 = make_float2(-kMagic, -kMagic);
-                    const float2 one2 = make_float2(1.0f, 1.0f);
-#pragma unroll
-                    for (int v = 0; v < V; ++v) {
-                        const int idx = tt + v * T;
-                        if (idx < p.nvec) {
-                            uint32_t u[8];
-                            float mu8[8];
-                            if (MU) load8(p.mu + (size_t)idx * 8, mu8);
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                const float2 t = __fmul2_rn(xh[v][k], inv2);
-                                // t * 1 + magic as one FMA: equal to t + magic, and it cannot be
-                                // contracted with the multiply above (which would change ties)
-                                const float2 uf = __ffma2_rn(t, one2, magic2);
-                                u[2 * k] = __float_as_uint(uf.x);
-                                u[2 * k + 1] = __float_as_uint(uf.y);
-                                if (MU) {
-                                    const float2 rq = __fadd2_rn(uf, nmagic2);              // q - Z, exact
-                                    const float2 neps = __ffma2_rn(nstep2, rq, xh[v][k]);   // -(Step (q - Z) - v^)
-                                    eneg = __ffma2_rn(neps, make_float2(mu8[2 * k], mu8[2 * k + 1]), eneg);
-                                }
-                            }
-                            store_codes(orow + (size_t)idx * vec_bytes, u, K, p.bits, BYTES_OUT);
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int v = 0; v < V; ++v) {
-                        const int idx = tt + v * T;
-                        if (idx < p.nvec) {
-                            uint32_t u[8];
-                            float mu8[8];
-                            if (MU) load8(p.mu + (size_t)idx * 8, mu8);
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                const int c0 = code_generic(xh[v][k].x, q.inv, q.zp, qmax);
-                                const int c1 = code_generic(xh[v][k].y, q.inv, q.zp, qmax);
-                                u[2 * k] = (uint32_t)c0;
-                                u[2 * k + 1] = (uint32_t)c1;
-                                if (MU) {
-                                    const float r0 = (float)((long long)c0 - (long long)q.zp);
-                                    const float r1 = (float)((long long)c1 - (long long)q.zp);
-                                    eneg.x = __fmaf_rn(__fmaf_rn(-q.step, r0, xh[v][k].x), mu8[2 * k], eneg.x);
-                                    eneg.y = __fmaf_rn(__fmaf_rn(-q.step, r1, xh[v][k].y), mu8[2 * k + 1], eneg.y);
-                                }
-                            }
-                            store_codes(orow + (size_t)idx * vec_bytes, u, 0u, p.bits, BYTES_OUT);
-                        }
-                    }
-                }
-                if (MU) {
-                    const float eacc = -warp_sum(__fadd_rn(eneg.x, eneg.y));
-                    if (wpt > 1) {
-                        if (lane == 0) sm->rsum[parity][warp] = eacc;
-                        named_bar_sync(1 + tm, T);
-                        if (tt == 0) {
-                            float tot = 0.0f;
-                            for (int w2 = 0; w2 < wpt; ++w2) tot += sm->rsum[parity][tw0 + w2];
-                            p.epsmu[row] = tot;
-                            if (p.bias.out || p.bias.out_f32)
-                                write_bias(row, tot, p.bias.in, p.bias.out, p.bias.out_f32, p.bias.bf16);
-                        }
-                    } else if (lane == 0) {
-                        p.epsmu[row] = eacc;
-                        if (p.bias.out || p.bias.out_f32)
-                            write_bias(row, eacc, p.bias.in, p.bias.out, p.bias.out_f32, p.bias.bf16);
-                    }
-                }
-                parity ^= 1;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm->empty[s]);
-        }
-        if (!ok && lane == 0) {
-            atomicExch(&sm->abort_flag, 1);
-            if (p.st) atomicAdd(&p.st->wait_timeout, 1ull);
-        }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0 && sm->abort_flag) {
-        const unsigned long long t0 = global_ns();
-        while (global_ns() - t0 < 1000000ull) { }
-    }
-}
-
-// ------------------------------------------------------------------ host side
-struct RowQuantPlan {
-    int V, NT, team, rows_per_stage, stages, grid;
-    size_t smem;
-    long long ntiles;
-};
 
 bool plan_rowquant(long long nrows, long long cols, RowQuantPlan *out)
 {
     const int nvec = (int)(cols / 8);
-    // smallest team (fewest cross-warp exchanges) whose threads hold at most 4
-    // vectors each; wide rows use all 512 threads and up to kRqMaxV vectors
-    int T = 32;
-    while (T < 512 && (nvec + T - 1) / T > 4) T *= 2;
-    int V = (nvec + T - 1) / T;
-    if (V > kRqMaxV) return false;
-    // a tighter fit with the same team when the row does not fill it
+    int T = 0, V = 0;
+    pick_team(nvec, &T, &V);
+    if (T == 0) return false;
     RowQuantPlan p;
     p.team = T;
     p.V = V;
-    p.NT = (T == 512 || V > 4) ? 512 : 256;
+    p.NT = T == 512 ? 512 : 256;
     const int teams = p.NT / T;
     const size_t row_bytes = (size_t)nvec * 16;
     const size_t budget = (p.NT == 512 ? 200 * 1024 : 100 * 1024) - kRqHeader;
@@ -367,7 +47,7 @@ bool plan_rowquant(long long nrows, long long cols, RowQuantPlan *out)
         R = (R + 1) / 2;
         S = (int)(budget / ((size_t)R * row_bytes));
     }
-    if (S < 1) return false;
+    if (S < 2) return false;          // the ring needs two stages
     if (S > kRqStagesMax) S = kRqStagesMax;
     p.rows_per_stage = R;
     p.stages = S;
@@ -380,34 +60,6 @@ bool plan_rowquant(long long nrows, long long cols, RowQuantPlan *out)
     p.grid = (int)g;
     *out = p;
     return true;
-}
-
-template <class D, int V, int NT, bool SCALE, bool MU, bool BYTES_OUT>
-static aweq_status launch_one(const RowQuantParams &p, const RowQuantPlan &pl, cudaStream_t stream)
-{
-    auto kern = rowquant_kernel<D, V, NT, SCALE, MU, BYTES_OUT>;
-    AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-    kern<<<pl.grid, NT + 32, pl.smem, stream>>>(p);
-    AWEQ_LAUNCH_CHECK();
-    return AWEQ_OK;
-}
-
-template <class D, bool SCALE, bool MU, bool BYTES_OUT>
-static aweq_status launch_v(const RowQuantParams &p, const RowQuantPlan &pl, cudaStream_t stream)
-{
-#define AWEQ_RQ_CASE(v)                                                                          \
-    case v:                                                                                      \
-        return pl.NT == 512 ? launch_one<D, v, 512, SCALE, MU, BYTES_OUT>(p, pl, stream)         \
-                            : launch_one<D, v, 256, SCALE, MU, BYTES_OUT>(p, pl, stream);
-    switch (pl.V) {
-        AWEQ_RQ_CASE(1) AWEQ_RQ_CASE(2) AWEQ_RQ_CASE(3) AWEQ_RQ_CASE(4)
-    case 5: return launch_one<D, 5, 512, SCALE, MU, BYTES_OUT>(p, pl, stream);
-    case 6: return launch_one<D, 6, 512, SCALE, MU, BYTES_OUT>(p, pl, stream);
-    case 7: case 8: return launch_one<D, 8, 512, SCALE, MU, BYTES_OUT>(p, pl, stream);
-    case 9: case 10: return launch_one<D, 10, 512, SCALE, MU, BYTES_OUT>(p, pl, stream);
-    }
-#undef AWEQ_RQ_CASE
-    return AWEQ_ERR_UNSUPPORTED;
 }
 
 bool rowquant_supported(long long nrows, long long cols)
@@ -432,18 +84,8 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     p.step = step; p.zp = zp; p.epsmu = epsmu; p.bits = bits; p.bias = bias;
     p.team = pl.team; p.rows_per_stage = pl.rows_per_stage; p.stages = pl.stages; p.ntiles = pl.ntiles;
     p.st = st;
-    const bool has_mu = weights && mu && epsmu;
-    const bool has_scale = scale != nullptr;
-#define AWEQ_RQ_GO(DT)                                                                           \
-    if (!weights) return has_scale ? launch_v<DT, true, false, true>(p, pl, stream)              \
-                                   : launch_v<DT, false, false, true>(p, pl, stream);            \
-    if (has_mu) return has_scale ? launch_v<DT, true, true, false>(p, pl, stream)                \
-                                 : launch_v<DT, false, true, false>(p, pl, stream);              \
-    return has_scale ? launch_v<DT, true, false, false>(p, pl, stream)                           \
-                     : launch_v<DT, false, false, false>(p, pl, stream);
-    if (dt == AWEQ_F16) { AWEQ_RQ_GO(F16) }
-    AWEQ_RQ_GO(BF16)
-#undef AWEQ_RQ_GO
+    const int mode = !weights ? 0 : ((mu && epsmu) ? 1 : 2);
+    return dt == AWEQ_F16 ? rq_launch_f16(p, pl, mode, stream) : rq_launch_bf16(p, pl, mode, stream);
 }
 
 }  // namespace aweq
