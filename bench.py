@@ -203,7 +203,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     X, W = generate(wl, dev, rank)
-    cal = calibrate.LayerCalibrator(wl, bits, X, W, None)
+    cal = calibrate.ShardedLayerCalibrator(wl, bits, X, W, None) if world > 1 else calibrate.LayerCalibrator(wl, bits, X, W, None)
     nbytes = calibrate.algorithmic_bytes(wl, bits)
     tokens = wl.inputs[0].n_tokens
 
@@ -231,15 +231,22 @@ def main():
     barrier()
     t_begin.record()
     for k in range(args.steps):
-        for lp, (es, ea) in zip(cal.passes, hooks[k]):
-            lp.set_events(es, ea)
-            lp(cal.ws, cal.status)
+        if world > 1:
+            names = [i.name for i in wl.inputs if i.name in cal.out]
+            cal.events = {n: h for n, h in zip(names, hooks[k])}
+            cal.run()                       # statistics merged over the ranks inside the step
+        else:
+            for lp, (es, ea) in zip(cal.passes, hooks[k]):
+                lp.set_events(es, ea)
+                lp(cal.ws, cal.status)
     t_end.record()
     barrier()
     launches = aweq.launch_count() - n0
     clocks = sampler.stop()
     for lp in cal.passes:
         lp.set_events(None, None)
+    if world > 1:
+        cal.events = None
     ms = t_begin.elapsed_time(t_end) / args.steps
     if dist is not None:
         t = torch.tensor([ms], device=dev)

@@ -13,6 +13,7 @@ from __future__ import annotations
 from typing import Dict, List, Optional
 
 import torch
+import torch.distributed as dist
 
 from . import aweq, synth
 
@@ -90,3 +91,77 @@ class LayerCalibrator:
         """One calibration pass of the whole layer: one library call per input."""
         for lp in self.passes:
             lp(self.ws, self.status)
+
+
+def allreduce_stats(xmin: torch.Tensor, xmax: torch.Tensor, xsum: torch.Tensor, count: torch.Tensor, group=None) -> None:
+    """The one exchange of a token-sharded calibration pass: per-channel minima, maxima,
+    binary64 sums and the token count of all ranks are merged in place (min / max / sum /
+    sum).  Works on any backend (NCCL on GPUs, gloo on CPU tensors)."""
+    dist.all_reduce(xmin, op=dist.ReduceOp.MIN, group=group)
+    dist.all_reduce(xmax, op=dist.ReduceOp.MAX, group=group)
+    dist.all_reduce(xsum, op=dist.ReduceOp.SUM, group=group)
+    dist.all_reduce(count, op=dist.ReduceOp.SUM, group=group)
+
+
+class ShardedLayerCalibrator(LayerCalibrator):
+    """Token-sharded pass: every rank holds its own N tokens of each layer input and a
+    replica of the weights.  Step 1 runs on the local shard, the statistics are merged
+    with ``allreduce_stats`` (3 C_in values per channel plus one count), the mean is
+    re-formed from the merged sums by the library (an empty ``aweq_stats`` call in
+    accumulate mode), steps 2-5 run replicated and step 6 on the local shard."""
+
+    def __init__(self, wl, bits, X, W, bias=None, flags=0, group=None):
+        super().__init__(wl, bits, X, W, bias, flags, diagnostics=True)
+        self.group = group
+        self.events = None          # optional {input name: (stats pair, act pair)} of torch.cuda.Event to record
+        self._X, self._W, self._bias, self._flags = X, W, bias, flags
+        dev = self.ws.device
+        for inp in wl.inputs:
+            if inp.name in self.out:
+                o = self.out[inp.name]
+                o["xsum"] = torch.empty(inp.c_in, dtype=torch.float64, device=dev)
+                o["count"] = torch.zeros(1, dtype=torch.int64, device=dev)
+
+    def run(self) -> None:
+        wl, bits = self.wl, self.bits
+        gran = aweq.PER_ROW if wl.w_gran == "row" else aweq.PER_GROUP
+        dt = aweq.F16 if wl.dtype == "f16" else aweq.BF16
+        eq = not (self._flags & aweq.FLAG_NO_EQUALIZE)
+        bc = not (self._flags & aweq.FLAG_NO_BIAS_CORRECT)
+        for inp in wl.inputs:
+            lins = [l for l in wl.linears if l.input == inp.name]
+            if not lins:
+                continue
+            x, o = self._X[inp.name], self.out[inp.name]
+            ev = self.events.get(inp.name) if self.events else None
+            if ev:
+                ev[0][0].record()
+            aweq.aweq_stats(x, o["xmin"], o["xmax"], o["xmean"], xsum=o["xsum"], count=o["count"], ws=self.ws,
+                            st=self.status)
+            if ev:
+                ev[0][1].record()
+            allreduce_stats(o["xmin"], o["xmax"], o["xsum"], o["count"], self.group)
+            aweq.aweq_stats(x, o["xmin"], o["xmax"], o["xmean"], xsum=o["xsum"], count=o["count"], accumulate=True,
+                            ws=self.ws, st=self.status, N=0)
+            for i, l in enumerate(lins):
+                aweq.aweq_wrange(self._W[l.name], o["wmin"], o["wmax"], accumulate=i > 0, ws=self.ws, st=self.status)
+            aweq.aweq_factors(o["xmin"], o["xmax"], o["xmean"], o["wmin"], o["wmax"], o["s"], o["rinv"], o["mu_hat"],
+                              o.get("pX"), o.get("pW"), o.get("scalars"), st=self.status)
+            s = o["s"] if eq else None
+            mu = o["mu_hat"] if eq else o["xmean"]
+            for l in lins:
+                lo = self.out[l.name]
+                aweq.aweq_equalize_quantize(self._W[l.name], s, mu if bc else None, bits, gran, wl.group, lo["codes"],
+                                            lo["step"], lo["zp"], lo["epsmu"] if bc else None, ws=self.ws,
+                                            st=self.status)
+                if bc:
+                    b_in = None if self._bias is None else self._bias.get(l.name)
+                    aweq.aweq_bias_correct(lo["epsmu"], None, None, None, None, None, None, bits, gran, wl.group,
+                                           b_in, lo["bias"], lo["bias_f32"], dt)
+            if wl.act_quant:
+                if ev:
+                    ev[1][0].record()
+                aweq.aweq_quant_act(x, o["rinv"] if eq else None, 8, aweq.PER_ROW, None, o["Xq"], o["act_step"],
+                                    o["act_zp"], st=self.status)
+                if ev:
+                    ev[1][1].record()

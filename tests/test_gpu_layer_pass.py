@@ -103,3 +103,29 @@ def test_ablation_switches():
     Xc, Wc = make_workload_tensors(wl, offset=2.0)
     for flags in (aweq.FLAG_NO_EQUALIZE, aweq.FLAG_NO_BIAS_CORRECT, aweq.FLAG_NO_EQUALIZE | aweq.FLAG_NO_BIAS_CORRECT):
         compare_layer(wl, 8, Xc, Wc, None, flags=flags)
+
+
+def test_sharded_path_with_one_rank_equals_fused_layer_pass():
+    """The token-sharded route (separate calls, statistics merged by an all-reduce and
+    re-formed by an empty accumulate call) on a one-rank NCCL group gives exactly what the
+    fused layer pass gives."""
+    import socket
+    import torch.distributed as dist
+    from paper_2311_01305_b200 import calibrate
+    wl = synth.workloads(n_tokens_scale=1.0 / 256)["opt125m_model_w8a8"]
+    Xc, Wc = make_workload_tensors(wl, offset=1.0)
+    Xd = {k: v.to(DEV) for k, v in Xc.items()}
+    Wd = {k: v.to(DEV) for k, v in Wc.items()}
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % port, rank=0, world_size=1,
+                            device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        a = calibrate.LayerCalibrator(wl, 8, Xd, Wd, None)
+        b = calibrate.ShardedLayerCalibrator(wl, 8, Xd, Wd, None)
+        a.run(); b.run()
+        torch.cuda.synchronize()
+    finally:
+        dist.destroy_process_group()
+    for name, outs in a.out.items():
+        for k, v in outs.items():
+            assert torch.equal(v, b.out[name][k]), (name, k)
