@@ -8,7 +8,8 @@
 // rows through a ring of shared-memory stages with 1-D bulk copies (TMA,
 // completion on mbarriers; warp 0 issues the copies between its own rows, so
 // that a CTA is 8 or 16 warps and the register file divides evenly over the
-// four schedulers).  A team of T threads owns one row of the stage at a time,
+// four schedulers).  A stage is released as soon as its rows are in registers,
+// so its refill overlaps the rest of the work on those rows.  A team of T threads owns one row of the stage at a time,
 // each thread holding V 16-byte vectors of the row, already multiplied by the
 // column scale, in registers; T is chosen small (few warps per row, V up to
 // 10) because everything that happens once per row -- the exchange of the
@@ -107,19 +108,29 @@ __device__ __forceinline__ void store_codes(unsigned char *dst, const uint32_t (
     }
 }
 
-// warp 0: start the copy of tile `t` of this CTA into its stage (waits, bounded, for the
-// stage to be released by every warp when it has been used before).  Returns false on a
-// timed-out wait.
-__device__ __forceinline__ bool rq_issue_tile(const RowQuantParams &p, RqSmem *sm, uint4 *stage_base, long long t,
-                                              int S, int R, size_t stage_vecs, int lane)
+// warp 0: is the stage of tile `t` free again (released by every warp after its previous
+// use)?  Blocking (bounded) or a single test.  *timed_out is set when a blocking wait gave up.
+__device__ __forceinline__ bool rq_stage_free(RqSmem *sm, long long t, int S, bool block, bool *timed_out)
 {
     const int s = (int)(t % S);
     const uint32_t use = (uint32_t)(t / S);
-    if (use > 0) {
-        bool ok = mbar_wait(&sm->empty[s], (use - 1) & 1);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) return false;
+    if (use == 0) return true;
+    bool ready;
+    if (block) {
+        ready = mbar_wait(&sm->empty[s], (use - 1) & 1);
+        ready = __all_sync(0xffffffffu, ready);
+        if (!ready) *timed_out = true;
+    } else {
+        ready = __all_sync(0xffffffffu, mbar_try_wait(&sm->empty[s], (use - 1) & 1));
     }
+    return ready;
+}
+
+// warp 0: start the copy of tile `t` of this CTA into its (free) stage.
+__device__ __forceinline__ void rq_issue_tile(const RowQuantParams &p, RqSmem *sm, uint4 *stage_base, long long t,
+                                              int S, int R, size_t stage_vecs, int lane)
+{
+    const int s = (int)(t % S);
     const long long row0 = (blockIdx.x + t * gridDim.x) * (long long)R;
     const int rows = (int)min((long long)R, p.nrows - row0);
     const uint32_t row_bytes = (uint32_t)p.nvec * 16u;
@@ -137,7 +148,6 @@ __device__ __forceinline__ bool rq_issue_tile(const RowQuantParams &p, RqSmem *s
         for (int r = lane; r < rows; r += 32)
             bulk_g2s(dst + (size_t)r * p.nvec, p.X + (row0 + r) * p.ld, row_bytes, &sm->full[s]);
     }
-    return true;
 }
 
 template <class D, int V, int NT, bool MU, bool BYTES_OUT>
@@ -169,10 +179,23 @@ rowquant_kernel(const RowQuantParams p)
     // tiles of R rows, dealt round-robin to the persistent CTAs
     const long long my_tiles = p.ntiles > blockIdx.x ? (p.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
+    // A stage is needed only until its rows sit in registers, so it is released right after
+    // the first pass and refilled while Step / Z are formed and the codes are written: up to
+    // S tiles are in flight.  warp 0 refills whenever it sees a free stage (single tests
+    // after each phase, a bounded wait only when the next tile has not been requested yet).
     bool ok = true;
+    long long next_issue = 0;                   // warp 0: first tile not yet requested
     if (warp == 0) {
-        for (long long t = 0; t < S - 1 && t < my_tiles && ok; ++t)
-            ok = rq_issue_tile(p, sm, stage_base, t, S, R, stage_vecs, lane);
+        for (; next_issue < S && next_issue < my_tiles; ++next_issue)
+            rq_issue_tile(p, sm, stage_base, next_issue, S, R, stage_vecs, lane);
+    }
+#define AWEQ_RQ_TRY_REFILL()                                                                   \
+    if (warp == 0 && next_issue < my_tiles) {                                                  \
+        bool dummy = false;                                                                    \
+        if (rq_stage_free(sm, next_issue, S, false, &dummy)) {                                 \
+            rq_issue_tile(p, sm, stage_base, next_issue, S, R, stage_vecs, lane);              \
+            ++next_issue;                                                                      \
+        }                                                                                      \
     }
     {
         const int tm = threadIdx.x / T, tt = threadIdx.x % T;
@@ -198,9 +221,14 @@ rowquant_kernel(const RowQuantParams p)
             }
         }
         for (long long k = 0; k < my_tiles; ++k) {
-            // keep S - 1 tiles in flight: the stage of tile k - 1 is refilled with tile k + S - 1
-            if (warp == 0 && ok && k + S - 1 < my_tiles)
-                ok = rq_issue_tile(p, sm, stage_base, k + S - 1, S, R, stage_vecs, lane);
+            if (warp == 0 && next_issue <= k) {              // cannot happen with S >= 2; kept as a guard
+                bool timed_out = false;
+                if (rq_stage_free(sm, next_issue, S, true, &timed_out)) {
+                    rq_issue_tile(p, sm, stage_base, next_issue, S, R, stage_vecs, lane);
+                    ++next_issue;
+                }
+                if (timed_out) ok = false;
+            }
             const int s = (int)(k % S);
             const uint32_t use = (uint32_t)(k / S);
             ok = ok && mbar_wait(&sm->full[s], use & 1) && !*reinterpret_cast<volatile int *>(&sm->abort_flag);
@@ -210,10 +238,15 @@ rowquant_kernel(const RowQuantParams p)
             const long long row0 = (blockIdx.x + k * gridDim.x) * (long long)R;
             const int rows = (int)min((long long)R, p.nrows - row0);
             const uint4 *tile = stage_base + (size_t)s * stage_vecs;
+            if (tm >= rows) {                                 // no row for this team in a short last tile
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->empty[s]);
+            }
             for (int r = tm; r < rows; r += teams) {
                 const uint4 *rowp = tile + (size_t)r * p.nvec;
                 float2 xh[V][4];
                 float lo = INFINITY, hi = -INFINITY;
+                float lo1 = INFINITY, hi1 = -INFINITY, lo2 = INFINITY, hi2 = -INFINITY, lo3 = INFINITY, hi3 = -INFINITY;
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     const int idx = tt + v * T;
@@ -234,12 +267,19 @@ rowquant_kernel(const RowQuantParams p)
                             xh[v][2] = __fmul2_rn(xh[v][2], make_float2(s1.x, s1.y));
                             xh[v][3] = __fmul2_rn(xh[v][3], make_float2(s1.z, s1.w));
                         }
+                        // four independent running extremes: no long dependent chain
                         lo = fminf(fminf(lo, xh[v][0].x), xh[v][0].y); hi = fmaxf(fmaxf(hi, xh[v][0].x), xh[v][0].y);
-                        lo = fminf(fminf(lo, xh[v][1].x), xh[v][1].y); hi = fmaxf(fmaxf(hi, xh[v][1].x), xh[v][1].y);
-                        lo = fminf(fminf(lo, xh[v][2].x), xh[v][2].y); hi = fmaxf(fmaxf(hi, xh[v][2].x), xh[v][2].y);
-                        lo = fminf(fminf(lo, xh[v][3].x), xh[v][3].y); hi = fmaxf(fmaxf(hi, xh[v][3].x), xh[v][3].y);
+                        lo1 = fminf(fminf(lo1, xh[v][1].x), xh[v][1].y); hi1 = fmaxf(fmaxf(hi1, xh[v][1].x), xh[v][1].y);
+                        lo2 = fminf(fminf(lo2, xh[v][2].x), xh[v][2].y); hi2 = fmaxf(fmaxf(hi2, xh[v][2].x), xh[v][2].y);
+                        lo3 = fminf(fminf(lo3, xh[v][3].x), xh[v][3].y); hi3 = fmaxf(fmaxf(hi3, xh[v][3].x), xh[v][3].y);
                     }
                 }
+                if (r + teams >= rows) {                      // my last row of the tile is in registers
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm->empty[s]);
+                }
+                lo = fminf(fminf(lo, lo1), fminf(lo2, lo3));
+                hi = fmaxf(fmaxf(hi, hi1), fmaxf(hi2, hi3));
                 lo = redux_min(lo, 0xffffffffu);
                 hi = redux_max(hi, 0xffffffffu);
                 if (wpt > 1) {
@@ -250,6 +290,7 @@ rowquant_kernel(const RowQuantParams p)
                     lo = redux_min(o.x, 0xffffffffu);
                     hi = redux_max(o.y, 0xffffffffu);
                 }
+                AWEQ_RQ_TRY_REFILL()
                 const QParams q = make_qparams(lo, hi, qmax);
                 const int fl = qflags(q, hi, qmax);
                 const long long row = row0 + r;
@@ -334,10 +375,10 @@ rowquant_kernel(const RowQuantParams p)
                     }
                 }
                 parity ^= 1;
+                AWEQ_RQ_TRY_REFILL()
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm->empty[s]);
         }
+#undef AWEQ_RQ_TRY_REFILL
         if (!ok && lane == 0) {
             atomicExch(&sm->abort_flag, 1);
             if (p.st) atomicAdd(&p.st->wait_timeout, 1ull);
