@@ -121,7 +121,7 @@ __device__ __forceinline__ bool rq_stage_free(RqSmem *sm, long long t, int S, bo
         ready = __all_sync(0xffffffffu, ready);
         if (!ready) *timed_out = true;
     } else {
-        ready = __all_sync(0xffffffffu, mbar_try_wait(&sm->empty[s], (use - 1) & 1));
+        ready = __all_sync(0xffffffffu, mbar_test(&sm->empty[s], (use - 1) & 1));
     }
     return ready;
 }
