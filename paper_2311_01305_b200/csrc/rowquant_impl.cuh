@@ -183,14 +183,19 @@ rowquant_kernel(const RowQuantParams p)
     // the first pass and refilled while Step / Z are formed and the codes are written: up to
     // S tiles are in flight.  warp 0 refills whenever it sees a free stage (single tests
     // after each phase, a bounded wait only when the next tile has not been requested yet).
+    // That pays when one row fills a stage and the whole CTA works on it (the widest rows: one
+    // tile in flight is then too little); with several rows per stage the stage is released
+    // at the end of the tile and refilled at the top of the next one.
+    const bool early = teams == 1;
     bool ok = true;
     long long next_issue = 0;                   // warp 0: first tile not yet requested
     if (warp == 0) {
-        for (; next_issue < S && next_issue < my_tiles; ++next_issue)
+        const int ahead = early ? S : S - 1;
+        for (; next_issue < ahead && next_issue < my_tiles; ++next_issue)
             rq_issue_tile(p, sm, stage_base, next_issue, S, R, stage_vecs, lane);
     }
 #define AWEQ_RQ_TRY_REFILL()                                                                   \
-    if (warp == 0 && next_issue < my_tiles) {                                                  \
+    if (early && warp == 0 && next_issue < my_tiles) {                                         \
         bool dummy = false;                                                                    \
         if (rq_stage_free(sm, next_issue, S, false, &dummy)) {                                 \
             rq_issue_tile(p, sm, stage_base, next_issue, S, R, stage_vecs, lane);              \
@@ -221,7 +226,8 @@ rowquant_kernel(const RowQuantParams p)
             }
         }
         for (long long k = 0; k < my_tiles; ++k) {
-            if (warp == 0 && next_issue <= k) {              // cannot happen with S >= 2; kept as a guard
+            if (warp == 0 && next_issue < my_tiles && (!early || next_issue <= k)) {
+                // late mode: tile k + S - 1 goes into the stage tile k - 1 used; early mode: only a guard
                 bool timed_out = false;
                 if (rq_stage_free(sm, next_issue, S, true, &timed_out)) {
                     rq_issue_tile(p, sm, stage_base, next_issue, S, R, stage_vecs, lane);
@@ -238,7 +244,7 @@ rowquant_kernel(const RowQuantParams p)
             const long long row0 = (blockIdx.x + k * gridDim.x) * (long long)R;
             const int rows = (int)min((long long)R, p.nrows - row0);
             const uint4 *tile = stage_base + (size_t)s * stage_vecs;
-            if (tm >= rows) {                                 // no row for this team in a short last tile
+            if (early && tm >= rows) {                        // no row for this team in a short last tile
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm->empty[s]);
             }
@@ -274,7 +280,7 @@ rowquant_kernel(const RowQuantParams p)
                         lo3 = fminf(fminf(lo3, xh[v][3].x), xh[v][3].y); hi3 = fmaxf(fmaxf(hi3, xh[v][3].x), xh[v][3].y);
                     }
                 }
-                if (r + teams >= rows) {                      // my last row of the tile is in registers
+                if (early && r + teams >= rows) {             // my last row of the tile is in registers
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm->empty[s]);
                 }
@@ -376,6 +382,10 @@ rowquant_kernel(const RowQuantParams p)
                 }
                 parity ^= 1;
                 AWEQ_RQ_TRY_REFILL()
+            }
+            if (!early) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->empty[s]);
             }
         }
 #undef AWEQ_RQ_TRY_REFILL
