@@ -185,8 +185,9 @@ rowquant_kernel(const RowQuantParams p)
     // after each phase, a bounded wait only when the next tile has not been requested yet).
     // That pays when one row fills a stage and the whole CTA works on it (the widest rows: one
     // tile in flight is then too little); with several rows per stage the stage is released
-    // at the end of the tile and refilled at the top of the next one.
-    const bool early = teams == 1;
+    // at the end of the tile and refilled at the top of the next one (measured: releasing early
+    // costs 5-9 % there).
+    constexpr bool early = NT == 512;           // the 512-thread shape is only used with one team
     bool ok = true;
     long long next_issue = 0;                   // warp 0: first tile not yet requested
     if (warp == 0) {
@@ -252,7 +253,6 @@ rowquant_kernel(const RowQuantParams p)
                 const uint4 *rowp = tile + (size_t)r * p.nvec;
                 float2 xh[V][4];
                 float lo = INFINITY, hi = -INFINITY;
-                float lo1 = INFINITY, hi1 = -INFINITY, lo2 = INFINITY, hi2 = -INFINITY, lo3 = INFINITY, hi3 = -INFINITY;
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     const int idx = tt + v * T;
@@ -273,19 +273,16 @@ rowquant_kernel(const RowQuantParams p)
                             xh[v][2] = __fmul2_rn(xh[v][2], make_float2(s1.x, s1.y));
                             xh[v][3] = __fmul2_rn(xh[v][3], make_float2(s1.z, s1.w));
                         }
-                        // four independent running extremes: no long dependent chain
                         lo = fminf(fminf(lo, xh[v][0].x), xh[v][0].y); hi = fmaxf(fmaxf(hi, xh[v][0].x), xh[v][0].y);
-                        lo1 = fminf(fminf(lo1, xh[v][1].x), xh[v][1].y); hi1 = fmaxf(fmaxf(hi1, xh[v][1].x), xh[v][1].y);
-                        lo2 = fminf(fminf(lo2, xh[v][2].x), xh[v][2].y); hi2 = fmaxf(fmaxf(hi2, xh[v][2].x), xh[v][2].y);
-                        lo3 = fminf(fminf(lo3, xh[v][3].x), xh[v][3].y); hi3 = fmaxf(fmaxf(hi3, xh[v][3].x), xh[v][3].y);
+                        lo = fminf(fminf(lo, xh[v][1].x), xh[v][1].y); hi = fmaxf(fmaxf(hi, xh[v][1].x), xh[v][1].y);
+                        lo = fminf(fminf(lo, xh[v][2].x), xh[v][2].y); hi = fmaxf(fmaxf(hi, xh[v][2].x), xh[v][2].y);
+                        lo = fminf(fminf(lo, xh[v][3].x), xh[v][3].y); hi = fmaxf(fmaxf(hi, xh[v][3].x), xh[v][3].y);
                     }
                 }
                 if (early && r + teams >= rows) {             // my last row of the tile is in registers
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm->empty[s]);
                 }
-                lo = fminf(fminf(lo, lo1), fminf(lo2, lo3));
-                hi = fmaxf(fmaxf(hi, hi1), fmaxf(hi2, hi3));
                 lo = redux_min(lo, 0xffffffffu);
                 hi = redux_max(hi, 0xffffffffu);
                 if (wpt > 1) {
