@@ -359,12 +359,9 @@ static aweq_status launch_colreduce(const void *X, long long rows, long long col
     double *psum = reinterpret_cast<double *>(base + (size_t)p.nsplit * cols * 8);
     const size_t smem = colreduce_smem_bytes(p.slab_w);
     auto kern = colreduce_kernel<D, WITH_SUM>;
-    static thread_local bool attr_set = false;
-    if (!attr_set) {
-        AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)colreduce_smem_bytes(kColThreads)));
-        attr_set = true;
-    }
+    // set on every launch: the attribute belongs to the current device, which may change between calls
+    AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)colreduce_smem_bytes(kColThreads)));
     int nsplit_eff = rows > 0 ? p.nsplit : 0;
     if (rows > 0) {
         kern<<<p.nslab * p.nsplit, kColThreads + 32, smem, stream>>>(
