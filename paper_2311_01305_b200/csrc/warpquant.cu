@@ -6,8 +6,8 @@
 //
 // A group of g columns is g/8 adjacent lanes of a warp, each holding one
 // 16-byte vector, so the group extremes are a single redux.sync over a lane
-// sub-mask and nothing has to be staged.  One warp walks one row, two vectors
-// per lane (512 columns, one 32-byte load) per step with the next step's load already in flight;
+// sub-mask and nothing has to be staged.  One warp walks one row, one vector
+// per lane (256 columns) per step with the next step's load already in flight;
 // many such warps per SM hide each other's latency (the kernel is bound by
 // instruction issue, so every per-element instruction counts).
 // The per-element work uses the packed binary32
@@ -95,74 +95,8 @@ __device__ __forceinline__ void store_vec(unsigned char *orow, int idx, const ui
     }
 }
 
-// 32-byte read-once load (two consecutive vectors of one lane)
-__device__ __forceinline__ void ldg_stream32(const void *p, uint4 &a, uint4 &b)
-{
-    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p));
-}
-
-// The codes u[h][i] + K of the VPL vectors of a lane, stored as one access where the layout
-// allows it (VPL == 2: 16 codes = 16 / 8 / 6 bytes for 8 / 4 / 3 bits).
-template <int BITS, bool BYTES_OUT, int VPL>
-__device__ __forceinline__ void store_lane(unsigned char *orow, int idxl, const uint32_t (&u)[VPL][8], uint32_t K,
-                                           int bits, bool active, bool quad3, bool pair3, int lane)
-{
-    if (VPL == 1) {
-        store_vec<BITS, BYTES_OUT>(orow, idxl, u[0], K, bits, active, quad3, lane);
-        return;
-    }
-    const int b = BITS ? BITS : bits;
-    if (BYTES_OUT || b == 8) {
-        const uint32_t kp = K * 0x01010101u;
-        uint4 w;
-        w.x = u[0][0] + (u[0][1] << 8) + (u[0][2] << 16) + (u[0][3] << 24) + kp;
-        w.y = u[0][4] + (u[0][5] << 8) + (u[0][6] << 16) + (u[0][7] << 24) + kp;
-        w.z = u[VPL - 1][0] + (u[VPL - 1][1] << 8) + (u[VPL - 1][2] << 16) + (u[VPL - 1][3] << 24) + kp;
-        w.w = u[VPL - 1][4] + (u[VPL - 1][5] << 8) + (u[VPL - 1][6] << 16) + (u[VPL - 1][7] << 24) + kp;
-        if (active) *reinterpret_cast<uint4 *>(orow + (size_t)idxl * 16) = w;
-    } else if (b == 4) {
-        uint2 w;
-        w.x = K * 0x11111111u;
-        w.y = w.x;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            w.x += u[0][e] << (4 * e);
-            w.y += u[VPL - 1][e] << (4 * e);
-        }
-        if (active) *reinterpret_cast<uint2 *>(orow + (size_t)idxl * 8) = w;
-    } else if (b == 3 && pair3) {
-        // 48 bits per lane; two lanes hold three 32-bit words (all lanes take part in the shuffle)
-        uint32_t wa = K * 0x249249u, wb = wa;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            wa += u[0][e] << (3 * e);
-            wb += u[VPL - 1][e] << (3 * e);
-        }
-        wa &= 0x00FFFFFFu;
-        wb &= 0x00FFFFFFu;
-        const uint32_t lo32 = wa | (wb << 24), hi16 = wb >> 8;
-        const uint32_t nlo = __shfl_down_sync(0xffffffffu, lo32, 1);       // the odd lane's low word
-        uint32_t *dst = reinterpret_cast<uint32_t *>(orow + (size_t)(idxl >> 1) * 12);
-        if (active) {
-            if ((lane & 1) == 0) {
-                dst[0] = lo32;
-                dst[1] = hi16 | (nlo << 16);
-            } else {
-                dst[2] = (lo32 >> 16) | (hi16 << 16);
-            }
-        }
-    } else {
-#pragma unroll
-        for (int h = 0; h < VPL; ++h) store_vec<BITS, BYTES_OUT>(orow, idxl * VPL + h, u[h], K, bits, active, false, lane);
-    }
-}
-
-// VPL: 16-byte vectors per lane and step.  Two when the group holds at least 16 columns and
-// the row an even number of vectors: the per-group work (Step, 1/Step, Z, their stores) is
-// then spread over 16 elements per lane instead of 8.
-template <class D, int BITS, bool STATIC, bool MU, bool BYTES_OUT, int VPL>
-__global__ void __launch_bounds__(kWqWarps * 32, VPL == 1 ? 4 : 3)
+template <class D, int BITS, bool STATIC, bool MU, bool BYTES_OUT>
+__global__ void __launch_bounds__(kWqWarps * 32, 4)
 warpquant_kernel(const WarpQuantParams p)
 {
     const int lane = threadIdx.x & 31;
@@ -170,13 +104,10 @@ warpquant_kernel(const WarpQuantParams p)
     const long long nwarps = (long long)gridDim.x * kWqWarps;
     const int bits = BITS ? BITS : p.bits;
     const int qmax = (1 << bits) - 1;
-    const int L = VPL == 1 ? p.lanes_per_group : max(p.lanes_per_group / VPL, 1);   // lanes per group
-    const int log2L = VPL == 1 ? p.log2_lanes : max(p.log2_lanes - 1, 0);
+    const int L = p.lanes_per_group;
     const uint32_t gmask = (STATIC || L >= 32) ? 0xffffffffu : (((1u << L) - 1u) << (lane & ~(L - 1)));
-    const int nlv = p.nvec / VPL;                        // lane-vectors per row
-    const int nsteps = (nlv + 31) / 32;
-    const bool quad3 = !BYTES_OUT && bits == 3 && VPL == 1 && (p.nvec % 4 == 0);
-    const bool pair3 = !BYTES_OUT && bits == 3 && VPL == 2 && (p.nvec % 4 == 0);
+    const int nsteps = (p.nvec + 31) / 32;
+    const bool quad3 = !BYTES_OUT && bits == 3 && (p.nvec % 4 == 0);
     const float2 magic2 = make_float2(kMagic, kMagic), nmagic2 = make_float2(-kMagic, -kMagic);
     const float2 one2 = make_float2(1.0f, 1.0f);
 
@@ -197,47 +128,30 @@ warpquant_kernel(const WarpQuantParams p)
         float *step_row = STATIC ? p.step : p.step + row * p.ngroups;
         int *zp_row = STATIC ? p.zp : p.zp + row * p.ngroups;
         float2 eneg = make_float2(0.0f, 0.0f);                 // minus the running eps . mu sum
-        uint4 nxt[VPL];
-#pragma unroll
-        for (int h = 0; h < VPL; ++h) nxt[h] = make_uint4(0, 0, 0, 0);
-        if (lane < nlv) {
-            if (VPL == 2) ldg_stream32(xrow + (size_t)lane * 16, nxt[0], nxt[VPL - 1]);
-            else nxt[0] = ldg_stream(xrow + (size_t)lane * 8);
-        }
+        uint4 nxt = lane < p.nvec ? ldg_stream(xrow + (size_t)lane * 8) : make_uint4(0, 0, 0, 0);
         for (int it = 0; it < nsteps; ++it) {
-            const int idxl = it * 32 + lane;                   // lane-vector index
-            const bool active = idxl < nlv;
-            float2 w2[VPL][4];
+            const int idx = it * 32 + lane;
+            const bool active = idx < p.nvec;
+            float w[8];
+            widen8<D>(nxt, w);
+            nxt = idx + 32 < p.nvec ? ldg_stream(xrow + (size_t)(idx + 32) * 8) : make_uint4(0, 0, 0, 0);
+            float2 w2[4];
+            if (p.scale && active) {
+                const float4 s0 = ldg_f4(p.scale + (size_t)idx * 8), s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
+                w2[0] = __fmul2_rn(make_float2(w[0], w[1]), make_float2(s0.x, s0.y));
+                w2[1] = __fmul2_rn(make_float2(w[2], w[3]), make_float2(s0.z, s0.w));
+                w2[2] = __fmul2_rn(make_float2(w[4], w[5]), make_float2(s1.x, s1.y));
+                w2[3] = __fmul2_rn(make_float2(w[6], w[7]), make_float2(s1.z, s1.w));
+            } else {
 #pragma unroll
-            for (int h = 0; h < VPL; ++h) {
-                float w[8];
-                widen8<D>(nxt[h], w);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) w2[h][k] = make_float2(w[2 * k], w[2 * k + 1]);
+                for (int k = 0; k < 4; ++k) w2[k] = make_float2(w[2 * k], w[2 * k + 1]);
             }
+            float mu8[8];
+            if (MU) {
+                if (active) load8(p.mu + (size_t)idx * 8, mu8);
+                else {
 #pragma unroll
-            for (int h = 0; h < VPL; ++h) nxt[h] = make_uint4(0, 0, 0, 0);
-            if (idxl + 32 < nlv) {
-                if (VPL == 2) ldg_stream32(xrow + (size_t)(idxl + 32) * 16, nxt[0], nxt[VPL - 1]);
-                else nxt[0] = ldg_stream(xrow + (size_t)(idxl + 32) * 8);
-            }
-            float mu8[VPL][8];
-#pragma unroll
-            for (int h = 0; h < VPL; ++h) {
-                const size_t e0 = ((size_t)idxl * VPL + h) * 8;
-                if (p.scale && active) {
-                    const float4 s0 = ldg_f4(p.scale + e0), s1 = ldg_f4(p.scale + e0 + 4);
-                    w2[h][0] = __fmul2_rn(w2[h][0], make_float2(s0.x, s0.y));
-                    w2[h][1] = __fmul2_rn(w2[h][1], make_float2(s0.z, s0.w));
-                    w2[h][2] = __fmul2_rn(w2[h][2], make_float2(s1.x, s1.y));
-                    w2[h][3] = __fmul2_rn(w2[h][3], make_float2(s1.z, s1.w));
-                }
-                if (MU) {
-                    if (active) load8(p.mu + e0, mu8[h]);
-                    else {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) mu8[h][e] = 0.0f;
-                    }
+                    for (int e = 0; e < 8; ++e) mu8[e] = 0.0f;
                 }
             }
             QParams q;
@@ -246,14 +160,10 @@ warpquant_kernel(const WarpQuantParams p)
                 q = qs;
                 fl = qs_flags;
             } else {
-                float a = INFINITY, b = -INFINITY;
-#pragma unroll
-                for (int h = 0; h < VPL; ++h) {
-                    a = fminf(fminf(a, w2[h][0].x), w2[h][0].y); b = fmaxf(fmaxf(b, w2[h][0].x), w2[h][0].y);
-                    a = fminf(fminf(a, w2[h][1].x), w2[h][1].y); b = fmaxf(fmaxf(b, w2[h][1].x), w2[h][1].y);
-                    a = fminf(fminf(a, w2[h][2].x), w2[h][2].y); b = fmaxf(fmaxf(b, w2[h][2].x), w2[h][2].y);
-                    a = fminf(fminf(a, w2[h][3].x), w2[h][3].y); b = fmaxf(fmaxf(b, w2[h][3].x), w2[h][3].y);
-                }
+                float a = fminf(fminf(w2[0].x, w2[0].y), w2[1].x), b = fmaxf(fmaxf(w2[0].x, w2[0].y), w2[1].x);
+                a = fminf(fminf(a, w2[1].y), w2[2].x); b = fmaxf(fmaxf(b, w2[1].y), w2[2].x);
+                a = fminf(fminf(a, w2[2].y), w2[3].x); b = fmaxf(fmaxf(b, w2[2].y), w2[3].x);
+                a = fminf(a, w2[3].y); b = fmaxf(b, w2[3].y);
                 if (L > 1) {
                     a = redux_min(a, gmask);
                     b = redux_max(b, gmask);
@@ -261,12 +171,12 @@ warpquant_kernel(const WarpQuantParams p)
                 q = make_qparams(a, b, qmax);
                 fl = qflags(q, b, qmax);
                 if (active && (lane & (L - 1)) == 0) {
-                    step_row[idxl >> log2L] = q.step;
-                    zp_row[idxl >> log2L] = q.zp;
+                    step_row[idx >> p.log2_lanes] = q.step;
+                    zp_row[idx >> p.log2_lanes] = q.zp;
                 }
             }
             const bool all_lean = __all_sync(0xffffffffu, !active || fl == (kQFast | kQNoClamp));
-            uint32_t u[VPL][8];
+            uint32_t u[8];
             uint32_t K;
             if (all_lean) {
                 K = (uint32_t)(q.zp - kMagicBits);
@@ -274,48 +184,40 @@ warpquant_kernel(const WarpQuantParams p)
                 const float2 nstep2 = make_float2(-q.step, -q.step);
                 const float hic = (float)(qmax - q.zp), loc = (float)(-q.zp);
 #pragma unroll
-                for (int h = 0; h < VPL; ++h) {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        float2 t = __fmul2_rn(w2[h][k], inv2);
-                        if (STATIC) {
-                            t.x = fmaxf(fminf(t.x, hic), loc);
-                            t.y = fmaxf(fminf(t.y, hic), loc);
-                        }
-                        // t * 1 + magic: the same value as t + magic, but as a single FMA that
-                        // cannot be merged with the multiply that produced t (the assembler was
-                        // seen to contract a packed multiply followed by a packed add, which
-                        // changes the rounding at exact .5 ties)
-                        const float2 uf = __ffma2_rn(t, one2, magic2);
-                        u[h][2 * k] = __float_as_uint(uf.x);
-                        u[h][2 * k + 1] = __float_as_uint(uf.y);
-                        if (MU) {
-                            const float2 rq = __fadd2_rn(uf, nmagic2);                 // q - Z, exact
-                            const float2 neps = __ffma2_rn(nstep2, rq, w2[h][k]);      // -(Step (q - Z) - w^)
-                            eneg = __ffma2_rn(neps, make_float2(mu8[h][2 * k], mu8[h][2 * k + 1]), eneg);
-                        }
+                for (int k = 0; k < 4; ++k) {
+                    float2 t = __fmul2_rn(w2[k], inv2);
+                    if (STATIC) {
+                        t.x = fmaxf(fminf(t.x, hic), loc);
+                        t.y = fmaxf(fminf(t.y, hic), loc);
+                    }
+                    // t * 1 + magic: the same value as t + magic, but as a single FMA that
+                    // cannot be merged with the multiply that produced t (the assembler was
+                    // seen to contract a packed multiply followed by a packed add, which
+                    // changes the rounding at exact .5 ties)
+                    const float2 uf = __ffma2_rn(t, one2, magic2);
+                    u[2 * k] = __float_as_uint(uf.x);
+                    u[2 * k + 1] = __float_as_uint(uf.y);
+                    if (MU) {
+                        const float2 rq = __fadd2_rn(uf, nmagic2);                 // q - Z, exact
+                        const float2 neps = __ffma2_rn(nstep2, rq, w2[k]);         // -(Step (q - Z) - w^)
+                        eneg = __ffma2_rn(neps, make_float2(mu8[2 * k], mu8[2 * k + 1]), eneg);
                     }
                 }
             } else {
                 K = 0u;
 #pragma unroll
-                for (int h = 0; h < VPL; ++h) {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int c0 = code_generic(w2[h][k].x, q.inv, q.zp, qmax);
-                        const int c1 = code_generic(w2[h][k].y, q.inv, q.zp, qmax);
-                        u[h][2 * k] = (uint32_t)c0;
-                        u[h][2 * k + 1] = (uint32_t)c1;
-                        if (MU) {
-                            const float r0 = (float)((long long)c0 - (long long)q.zp);
-                            const float r1 = (float)((long long)c1 - (long long)q.zp);
-                            eneg.x = __fmaf_rn(__fmaf_rn(-q.step, r0, w2[h][k].x), mu8[h][2 * k], eneg.x);
-                            eneg.y = __fmaf_rn(__fmaf_rn(-q.step, r1, w2[h][k].y), mu8[h][2 * k + 1], eneg.y);
-                        }
+                for (int k = 0; k < 4; ++k) {
+                    const int c0 = code_generic(w2[k].x, q.inv, q.zp, qmax), c1 = code_generic(w2[k].y, q.inv, q.zp, qmax);
+                    u[2 * k] = (uint32_t)c0;
+                    u[2 * k + 1] = (uint32_t)c1;
+                    if (MU) {
+                        const float r0 = (float)((long long)c0 - (long long)q.zp), r1 = (float)((long long)c1 - (long long)q.zp);
+                        eneg.x = __fmaf_rn(__fmaf_rn(-q.step, r0, w2[k].x), mu8[2 * k], eneg.x);
+                        eneg.y = __fmaf_rn(__fmaf_rn(-q.step, r1, w2[k].y), mu8[2 * k + 1], eneg.y);
                     }
                 }
             }
-            store_lane<BITS, BYTES_OUT, VPL>(orow, idxl, u, K, bits, active, quad3, pair3, lane);
+            store_vec<BITS, BYTES_OUT>(orow, idx, u, K, bits, active, quad3, lane);
         }
         if (MU) {
             const float tot = -warp_sum(__fadd_rn(eneg.x, eneg.y));
@@ -371,14 +273,7 @@ static aweq_status launch_wq(const WarpQuantParams &p, cudaStream_t stream)
     const long long cap = (long long)kSmCount * 8 * 4;      // a few waves; warps stride over the rows beyond that
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    // two vectors per lane need an even number of vectors per row, 32-byte aligned rows and
-    // groups of at least 16 columns
-    const bool two = (p.nvec % 2 == 0) && (p.ld % 16 == 0) && ((reinterpret_cast<uintptr_t>(p.X) & 31) == 0) &&
-                     (STATIC || p.lanes_per_group >= 2);
-    if (two)
-        warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT, 2><<<(unsigned)blocks, kWqWarps * 32, 0, stream>>>(p);
-    else
-        warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT, 1><<<(unsigned)blocks, kWqWarps * 32, 0, stream>>>(p);
+    warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT><<<(unsigned)blocks, kWqWarps * 32, 0, stream>>>(p);
     AWEQ_LAUNCH_CHECK();
     return AWEQ_OK;
 }
