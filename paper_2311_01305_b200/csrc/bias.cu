@@ -11,6 +11,7 @@ __global__ void bias_apply_kernel(const float *__restrict__ epsmu, const uint16_
                                   uint16_t *__restrict__ bias_out, float *__restrict__ bias_out_f32, int bias_bf16,
                                   long long C_out)
 {
+    pdl_begin();
     const long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (o >= C_out) return;
     write_bias(o, epsmu[o], bias_in, bias_out, bias_out_f32, bias_bf16);
@@ -34,6 +35,7 @@ bias_gemv_kernel(const uint16_t *__restrict__ W, long long C_out, long long C_in
                  int bits, int gran, int group, const uint16_t *__restrict__ bias_in, uint16_t *__restrict__ bias_out,
                  float *__restrict__ bias_out_f32, int bias_bf16)
 {
+    pdl_begin();
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= C_out) return;
@@ -59,9 +61,8 @@ aweq_status run_bias_apply(const float *epsmu, const void *bias_in, void *bias_o
 {
     const int t = 256;
     const unsigned g = (unsigned)((C_out + t - 1) / t);
-    bias_apply_kernel<<<g, t, 0, stream>>>(epsmu, (const uint16_t *)bias_in, (uint16_t *)bias_out, bias_out_f32,
-                                           bias_dt == AWEQ_BF16, C_out);
-    AWEQ_LAUNCH_CHECK();
+    AWEQ_LAUNCH(bias_apply_kernel, dim3(g), dim3(t), 0, stream, epsmu, (const uint16_t *)bias_in, (uint16_t *)bias_out,
+                bias_out_f32, (int)(bias_dt == AWEQ_BF16), C_out);
     return AWEQ_OK;
 }
 
@@ -72,14 +73,13 @@ aweq_status run_bias_gemv(const void *W, aweq_dtype dt, long long C_out, long lo
 {
     const unsigned g = (unsigned)((C_out + 7) / 8);
     if (dt == AWEQ_F16)
-        bias_gemv_kernel<F16><<<g, 256, 0, stream>>>((const uint16_t *)W, C_out, C_in, ld, s, codes, step, zp,
-                                                      mu_hat, bits, gran, group, (const uint16_t *)bias_in,
-                                                      (uint16_t *)bias_out, bias_out_f32, bias_dt == AWEQ_BF16);
+        AWEQ_LAUNCH(bias_gemv_kernel<F16>, dim3(g), dim3(256), 0, stream, (const uint16_t *)W, C_out, C_in, ld, s, codes,
+                    step, zp, mu_hat, bits, gran, group, (const uint16_t *)bias_in, (uint16_t *)bias_out, bias_out_f32,
+                    (int)(bias_dt == AWEQ_BF16));
     else
-        bias_gemv_kernel<BF16><<<g, 256, 0, stream>>>((const uint16_t *)W, C_out, C_in, ld, s, codes, step, zp,
-                                                       mu_hat, bits, gran, group, (const uint16_t *)bias_in,
-                                                       (uint16_t *)bias_out, bias_out_f32, bias_dt == AWEQ_BF16);
-    AWEQ_LAUNCH_CHECK();
+        AWEQ_LAUNCH(bias_gemv_kernel<BF16>, dim3(g), dim3(256), 0, stream, (const uint16_t *)W, C_out, C_in, ld, s, codes,
+                    step, zp, mu_hat, bits, gran, group, (const uint16_t *)bias_in, (uint16_t *)bias_out, bias_out_f32,
+                    (int)(bias_dt == AWEQ_BF16));
     return AWEQ_OK;
 }
 

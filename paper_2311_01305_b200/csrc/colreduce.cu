@@ -164,6 +164,7 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
         sm->abort_flag = 0;
         mbar_init_fence();
     }
+    pdl_begin();                 // everything above overlaps the tail of the previous kernel
     __syncthreads();
 
     if (warp == kColThreads / 32) {
@@ -295,6 +296,7 @@ colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restric
 {
     __shared__ float slo[kFinLanes][kFinCols], shi[kFinLanes][kFinCols];
     __shared__ double ssum[kFinLanes][kFinCols];
+    pdl_begin();
     const int c = threadIdx.x % kFinCols, k0 = threadIdx.x / kFinCols;
     const long long j = (long long)blockIdx.x * kFinCols + c;
     float lo = INFINITY, hi = -INFINITY;
@@ -339,6 +341,7 @@ colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restric
 
 __global__ void bump_count_kernel(long long *count, long long nrows, int accumulate)
 {
+    pdl_begin();
     count[0] = (accumulate ? count[0] : 0) + nrows;
 }
 
@@ -364,17 +367,15 @@ static aweq_status launch_colreduce(const void *X, long long rows, long long col
                                       (int)colreduce_smem_bytes(kColThreads)));
     int nsplit_eff = rows > 0 ? p.nsplit : 0;
     if (rows > 0) {
-        kern<<<p.nslab * p.nsplit, kColThreads + 32, smem, stream>>>(
-            reinterpret_cast<const uint16_t *>(X), rows, ld, p.nvec, p.nslab, p.slab_w, p.rows_per_split, cols, pmin,
-            pmax, psum, st);
-        AWEQ_LAUNCH_CHECK();
+        AWEQ_LAUNCH(kern, dim3(p.nslab * p.nsplit), dim3(kColThreads + 32), smem, stream,
+                    reinterpret_cast<const uint16_t *>(X), rows, ld, p.nvec, p.nslab, p.slab_w, p.rows_per_split, cols,
+                    pmin, pmax, psum, st);
     }
-    colreduce_finalize_kernel<WITH_SUM><<<(unsigned)((cols + kFinCols - 1) / kFinCols), kFinCols * kFinLanes, 0, stream>>>(
-        pmin, pmax, psum, nsplit_eff, cols, rows, omin, omax, omean, osum, count, accumulate, st);
-    AWEQ_LAUNCH_CHECK();
+    AWEQ_LAUNCH(colreduce_finalize_kernel<WITH_SUM>, dim3((unsigned)((cols + kFinCols - 1) / kFinCols)),
+                dim3(kFinCols * kFinLanes), 0, stream, (const float *)pmin, (const float *)pmax, (const double *)psum,
+                nsplit_eff, cols, rows, omin, omax, omean, osum, (const long long *)count, accumulate, st);
     if (WITH_SUM && count) {
-        bump_count_kernel<<<1, 1, 0, stream>>>(count, rows, accumulate);
-        AWEQ_LAUNCH_CHECK();
+        AWEQ_LAUNCH(bump_count_kernel, dim3(1), dim3(1), 0, stream, count, rows, accumulate);
     }
     return AWEQ_OK;
 }

@@ -32,6 +32,40 @@ aweq_status cuda_failed(cudaError_t e);    // records the error text, returns AW
         if (e__ != cudaSuccess) return ::aweq::cuda_failed(e__); \
     } while (0)
 
+#define AWEQ_LAUNCH(...)                                     \
+    do {                                                     \
+        cudaError_t e__ = ::aweq::launch_pdl(__VA_ARGS__);   \
+        ::aweq::note_launch();                               \
+        if (e__ != cudaSuccess) return ::aweq::cuda_failed(e__); \
+    } while (0)
+
+// ------------------------------------------------------------------ programmatic dependent launch
+// Every kernel of the library is launched with programmatic stream serialisation: the next
+// kernel of the stream may be scheduled while this one drains, and waits (pdl_wait, first
+// statement that touches global memory) until everything before it has completed and is
+// visible.  That removes most of the launch gap between the many short kernels of a pass.
+template <class... KArgs, class... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+__device__ __forceinline__ void pdl_begin()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ------------------------------------------------------------------ 16-bit traits
 struct F16 {
     using T2 = __half2;

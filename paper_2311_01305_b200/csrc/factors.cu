@@ -87,6 +87,7 @@ factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, c
     __shared__ double dsum[2][kFacThreads / 32];
     __shared__ unsigned int dead_count;
     if (threadIdx.x == 0) dead_count = 0;
+    pdl_begin();
     __syncthreads();
 
     // four channels per thread and step (128-bit loads) when the arrays allow it
@@ -191,9 +192,8 @@ aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean
                         const float *wmax, long long C, float *s, float *rinv, float *mu_hat, float *pX, float *pW,
                         double *scalars, aweq_dev_status *st, cudaStream_t stream)
 {
-    factors_kernel<<<1, kFacThreads, 0, stream>>>(xmin, xmax, xmean, wmin, wmax, (int)C, s, rinv, mu_hat, pX, pW,
-                                                  scalars, st);
-    AWEQ_LAUNCH_CHECK();
+    AWEQ_LAUNCH(factors_kernel, dim3(1), dim3(kFacThreads), 0, stream, xmin, xmax, xmean, wmin, wmax, (int)C, s, rinv,
+                mu_hat, pX, pW, scalars, st);
     return AWEQ_OK;
 }
 

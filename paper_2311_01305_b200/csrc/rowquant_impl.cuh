@@ -174,6 +174,7 @@ rowquant_kernel(const RowQuantParams p)
         sm->abort_flag = 0;
         mbar_init_fence();
     }
+    pdl_begin();                 // everything above overlaps the tail of the previous kernel
     __syncthreads();
 
     // tiles of R rows, dealt round-robin to the persistent CTAs
@@ -404,8 +405,7 @@ static aweq_status rq_launch_one(const RowQuantParams &p, const RowQuantPlan &pl
 {
     auto kern = rowquant_kernel<D, V, NT, MU, BYTES_OUT>;
     AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-    kern<<<pl.grid, NT, pl.smem, stream>>>(p);
-    AWEQ_LAUNCH_CHECK();
+    AWEQ_LAUNCH(kern, dim3(pl.grid), dim3(NT), pl.smem, stream, p);
     return AWEQ_OK;
 }
 

@@ -99,6 +99,7 @@ template <class D, int BITS, bool STATIC, bool MU, bool BYTES_OUT>
 __global__ void __launch_bounds__(kWqWarps * 32, 4)
 warpquant_kernel(const WarpQuantParams p)
 {
+    pdl_begin();
     const int lane = threadIdx.x & 31;
     const long long warp0 = (long long)blockIdx.x * kWqWarps + (threadIdx.x >> 5);
     const long long nwarps = (long long)gridDim.x * kWqWarps;
@@ -235,6 +236,7 @@ __global__ void scaled_tensor_range_kernel(const float *__restrict__ cmin, const
                                            const float *__restrict__ scale, int C, float *lo_hi)
 {
     __shared__ float slo[32], shi[32];
+    pdl_begin();
     float lo = INFINITY, hi = -INFINITY;
     for (int j = threadIdx.x; j < C; j += blockDim.x) {
         const float sc = scale ? scale[j] : 1.0f;
@@ -261,8 +263,7 @@ __global__ void scaled_tensor_range_kernel(const float *__restrict__ cmin, const
 aweq_status run_scaled_tensor_range(const float *cmin, const float *cmax, const float *scale, long long C,
                                     float *lo_hi, cudaStream_t stream)
 {
-    scaled_tensor_range_kernel<<<1, 1024, 0, stream>>>(cmin, cmax, scale, (int)C, lo_hi);
-    AWEQ_LAUNCH_CHECK();
+    AWEQ_LAUNCH(scaled_tensor_range_kernel, dim3(1), dim3(1024), 0, stream, cmin, cmax, scale, (int)C, lo_hi);
     return AWEQ_OK;
 }
 
@@ -273,8 +274,8 @@ static aweq_status launch_wq(const WarpQuantParams &p, cudaStream_t stream)
     const long long cap = (long long)kSmCount * 8 * 4;      // a few waves; warps stride over the rows beyond that
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT><<<(unsigned)blocks, kWqWarps * 32, 0, stream>>>(p);
-    AWEQ_LAUNCH_CHECK();
+    AWEQ_LAUNCH((warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT>), dim3((unsigned)blocks), dim3(kWqWarps * 32), 0,
+                stream, p);
     return AWEQ_OK;
 }
 
