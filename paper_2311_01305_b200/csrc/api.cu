@@ -3,6 +3,7 @@
 // here and nothing synchronises.
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -20,6 +21,18 @@ aweq_status cuda_failed(cudaError_t e)
     snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
     return AWEQ_ERR_CUDA;
 }
+
+// AWEQ_LOG=1 in the environment: one line per entry-point call on stderr (shapes and the
+// algorithmic bytes the call moves); read once.
+static bool log_enabled()
+{
+    static const bool on = [] { const char *e = getenv("AWEQ_LOG"); return e && e[0] && e[0] != '0'; }();
+    return on;
+}
+#define AWEQ_LOGF(...)                                       \
+    do {                                                     \
+        if (::aweq::log_enabled()) fprintf(stderr, "[aweq] " __VA_ARGS__); \
+    } while (0)
 
 static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 static inline size_t round256(size_t n) { return (n + 255) & ~(size_t)255; }
@@ -112,6 +125,8 @@ aweq_status aweq_stats(const void *X, aweq_dtype dt, long long N, long long C_in
         return AWEQ_ERR_ALIGN;
     rc = check_ws(ws, ws_bytes, colreduce_ws_bytes(N, C_in));
     if (rc != AWEQ_OK) return rc;
+    AWEQ_LOGF("aweq_stats N=%lld C_in=%lld ld=%lld dtype=%d accumulate=%d bytes=%lld\n", N, C_in, ldx, (int)dt, accumulate,
+              2 * N * C_in);
     return run_stats(X, dt, N, C_in, ldx, xmin, xmax, xmean, xsum, count, accumulate, ws, st, (cudaStream_t)stream);
 }
 
@@ -123,6 +138,7 @@ aweq_status aweq_wrange(const void *W, aweq_dtype dt, long long C_out, long long
     if (!wmin || !wmax) return AWEQ_ERR_NULL;
     rc = check_ws(ws, ws_bytes, colreduce_ws_bytes(C_out, C_in));
     if (rc != AWEQ_OK) return rc;
+    AWEQ_LOGF("aweq_wrange C_out=%lld C_in=%lld accumulate=%d bytes=%lld\n", C_out, C_in, accumulate, 2 * C_out * C_in);
     return run_wrange(W, dt, C_out, C_in, ldw, wmin, wmax, accumulate, ws, st, (cudaStream_t)stream);
 }
 
@@ -150,6 +166,8 @@ static aweq_status equalize_quantize_impl(const void *W, aweq_dtype dt, long lon
     if (!aligned(codes, 16) || (s && !aligned(s, 16)) || (mu_hat && !aligned(mu_hat, 16))) return AWEQ_ERR_ALIGN;
     rc = check_ws(ws, ws_bytes, eq_ws_bytes(C_out, C_in, gran));
     if (rc != AWEQ_OK) return rc;
+    AWEQ_LOGF("aweq_equalize_quantize C_out=%lld C_in=%lld bits=%d gran=%d group=%d bytes=%lld\n", C_out, C_in, bits,
+              (int)gran, group, 2 * C_out * C_in + C_out * C_in * bits / 8);
     cudaStream_t cs = (cudaStream_t)stream;
     if (gran == AWEQ_PER_ROW) {
         if (!rowquant_supported(C_out, C_in)) return AWEQ_ERR_SHAPE;
@@ -211,6 +229,7 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
     if (bits < 2 || bits > 8) return AWEQ_ERR_BITS;
     if (!Xq || !step || !zp) return AWEQ_ERR_NULL;
     if (!aligned(Xq, 16) || (rinv && !aligned(rinv, 16))) return AWEQ_ERR_ALIGN;
+    AWEQ_LOGF("aweq_quant_act N=%lld C_in=%lld bits=%d gran=%d bytes=%lld\n", N, C_in, bits, (int)gran, 3 * N * C_in + 8 * N);
     cudaStream_t cs = (cudaStream_t)stream;
     if (gran == AWEQ_PER_ROW) {
         if (!rowquant_supported(N, C_in)) return AWEQ_ERR_SHAPE;
