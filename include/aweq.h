@@ -267,6 +267,32 @@ size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args);
 aweq_status aweq_layer_pass(const aweq_layer_args *args, void *ws, size_t ws_bytes,
                             aweq_dev_status *st, void *stream);
 
+/* ---- Forward check of a calibrated W8A8 layer (Eq. 11; the quantity ablated in the AWE / BC
+ * table) ------------------------------------------------------------------------------------
+ * Compares, on the calibration tokens, the quantised layer
+ *     y~[n,o] = sum_k Step^x_n (Xq[n,k] - Z^x_n) * Step^w_o (Wq[o,k] - Z^w_o) + bias_q[o]
+ * (Eq. 1-2 de-quantisation of the step-6 activation codes and of the 8-bit per-row step-4
+ * weight codes; bias_q is the corrected bias of Eq. 15) with the 16-bit layer
+ *     y[n,o] = sum_k X[n,k] W[o,k] + bias[o]
+ * (equalisation leaves this product unchanged, Eq. 3).  Both contractions run on the tensor
+ * cores: the integer one exactly (int32 accumulation, zero-points folded in afterwards in
+ * 64-bit integers), the 16-bit one with binary32 accumulation.  Outputs (device):
+ *   mean_err[C_out]  binary64, (1/N) sum_n (y~[n,o] - y[n,o])      -- E[y~_j - y_j] of Eq. 11
+ *   sums[4]          binary64: sum (y~ - y)^2, sum y^2, sum_o mean_err[o]^2, N * C_out
+ * Layout: Xq [N x C_in] and Wq [C_out x C_in] one byte per code, X and W 16-bit, all
+ * row-major, contiguous (no pitch) and 16-byte aligned; act_step/act_zp [N], w_step/w_zp
+ * [C_out]; bias_q (binary32, [C_out]) and bias (16-bit, [C_out]) may be NULL (= 0).
+ * C_in must be a multiple of 16, C_out a multiple of 8 (AWEQ_ERR_SHAPE otherwise).
+ * ws: aweq_forward_check_workspace_bytes(N, C_in, C_out) bytes, 256-byte aligned; nothing is
+ * allocated.  Everything is enqueued on `stream`; the caller owns all buffers.
+ * Returns AWEQ_ERR_UNSUPPORTED when the library was built without the tensor-core GEMM. */
+size_t aweq_forward_check_workspace_bytes(long long N, long long C_in, long long C_out);
+aweq_status aweq_forward_check(const unsigned char *Xq, const float *act_step, const int *act_zp,
+                               const unsigned char *Wq, const float *w_step, const int *w_zp,
+                               const float *bias_q, const void *X, const void *W, aweq_dtype dt,
+                               const void *bias, long long N, long long C_in, long long C_out,
+                               double *mean_err, double *sums, void *ws, size_t ws_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,6 +25,23 @@ NVCC_FLAGS = [
 ]
 
 
+def _cutlass_flags() -> list:
+    """Include paths of a CUTLASS 3.x/4.x header tree with the sm_100 collectives (the forward
+    check's tensor-core GEMMs are instantiated from them).  ``AWEQ_CUTLASS`` names the tree;
+    otherwise the copies vendored inside Python packages are searched.  Without one the GEMM
+    translation units compile to stubs that return AWEQ_ERR_UNSUPPORTED."""
+    import sysconfig
+    roots = [os.environ.get("AWEQ_CUTLASS")]
+    for sp in {sysconfig.get_paths()["purelib"], sysconfig.get_paths()["platlib"]}:
+        roots += [os.path.join(sp, "flashinfer", "data", "cutlass"), os.path.join(sp, "tilelang", "3rdparty", "cutlass")]
+    for r in roots:
+        if r and os.path.exists(os.path.join(r, "include", "cutlass", "gemm", "collective", "builders",
+                                             "sm100_umma_builder.inl")):
+            return ["-I" + os.path.join(r, "include"), "-I" + os.path.join(r, "tools", "util", "include"),
+                    "--expt-relaxed-constexpr"]
+    return ["-DAWEQ_NO_CUTLASS"]
+
+
 def _nvcc() -> str:
     for c in (os.environ.get("NVCC"), "/usr/local/cuda/bin/nvcc", "nvcc"):
         if c and (os.path.isabs(c) and os.path.exists(c) or not os.path.isabs(c)):
@@ -37,7 +54,8 @@ def _newest(paths) -> float:
 
 
 def _compile(src: str, obj: str, verbose: bool) -> str:
-    cmd = [_nvcc(), *NVCC_FLAGS, "-c", src, "-o", obj]
+    extra = _cutlass_flags() if os.path.basename(src).startswith("forward_gemm") else []
+    cmd = [_nvcc(), *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError("nvcc failed for %s:\n%s\n%s" % (src, r.stdout, r.stderr))

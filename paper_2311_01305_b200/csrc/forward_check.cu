@@ -1,0 +1,215 @@
+// W8A8 forward check: the calibrated layer  y~ = dequant(Xq) dequant(Wq)^T + bias'  against
+// the 16-bit layer  y = X W^T + bias  on the calibration inputs, reported as the mean output
+// error per output channel (the quantity of Eq. 11, E[y~_j - y_j], which bias correction
+// is built to remove) and as sums of squares (output MSE and signal power).
+//
+// Both products are dense contractions and run on the tensor cores (forward_gemm.cuh):
+//   S[n,o] = sum_k Xq[n,k] Wq[o,k]            unsigned 8-bit x unsigned 8-bit -> int32
+//   Y[n,o] = sum_k X[n,k] W[o,k]              fp16 / bf16 -> binary32
+// The zero-points of Eq. 1 are folded in afterwards, in integers:
+//   y~[n,o] = Step^x_n Step^w_o (S - Z^x_n cw_o - Z^w_o rx_n + K Z^x_n Z^w_o) + bias'_o
+// with rx_n = sum_k Xq[n,k] and cw_o = sum_k Wq[o,k].  A sum of K products of 8-bit codes
+// fits int32 for K <= 33025; wider layers are contracted in two K-halves that are added in
+// 64-bit.  Tokens are processed in chunks so that the [chunk x C_out] intermediates stay
+// a few hundred MB.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace aweq {
+
+constexpr long long kFcChunk = 16384;          // tokens per chunk
+constexpr int kFcRowBlock = 256;               // tokens folded by one thread of the comparison kernel
+constexpr long long kFcSplitK = 32768;         // above this C_in the integer product is taken in two halves
+constexpr size_t kFcScratch = 1 << 20;         // scratch of the GEMMs
+
+static inline size_t up256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+struct FcLayout {
+    long long chunk, nchunks, blocks_per_chunk, nblocks;
+    size_t S, S2, Y, rx, cw, partial, scratch, total;
+};
+
+static FcLayout fc_layout(long long N, long long C_in, long long C_out)
+{
+    FcLayout L;
+    L.chunk = N < kFcChunk ? N : kFcChunk;
+    L.nchunks = (N + kFcChunk - 1) / kFcChunk;
+    L.blocks_per_chunk = (L.chunk + kFcRowBlock - 1) / kFcRowBlock;
+    const long long last_rows = N - (L.nchunks - 1) * kFcChunk;
+    L.nblocks = (L.nchunks - 1) * L.blocks_per_chunk + (last_rows + kFcRowBlock - 1) / kFcRowBlock;
+    size_t off = 0;
+    L.S = off; off += up256((size_t)L.chunk * C_out * 4);
+    L.S2 = off; off += C_in > kFcSplitK ? up256((size_t)L.chunk * C_out * 4) : 0;
+    L.Y = off; off += up256((size_t)L.chunk * C_out * 4);
+    L.rx = off; off += up256((size_t)N * 4);
+    L.cw = off; off += up256((size_t)C_out * 4);
+    L.partial = off; off += up256((size_t)L.nblocks * C_out * 3 * 8);
+    L.scratch = off; off += kFcScratch;
+    L.total = off;
+    return L;
+}
+
+size_t forward_check_ws_bytes(long long N, long long C_in, long long C_out) { return fc_layout(N, C_in, C_out).total; }
+
+// sum of the bytes of every row of a row-major u8 matrix (one warp per row)
+__global__ void __launch_bounds__(256) fc_rowsum_kernel(const unsigned char *__restrict__ Q, long long rows,
+                                                        long long cols, int *__restrict__ out)
+{
+    pdl_begin();
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const uint4 *p = reinterpret_cast<const uint4 *>(Q + row * cols);
+    unsigned int acc = 0;
+    for (long long i = lane; i < cols / 16; i += 32) {
+        const uint4 v = __ldg(p + i);
+        acc = __dp4a(v.x, 0x01010101u, acc);
+        acc = __dp4a(v.y, 0x01010101u, acc);
+        acc = __dp4a(v.z, 0x01010101u, acc);
+        acc = __dp4a(v.w, 0x01010101u, acc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) out[row] = (int)acc;
+}
+
+// One thread per output channel and block of kFcRowBlock tokens: form y~ and y, fold
+// d = y~ - y, d^2 and y^2 in binary64 in token order, one partial per (block, channel).
+template <class D>
+__global__ void __launch_bounds__(256)
+fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const float *__restrict__ Y, long long rows,
+                  long long C_out, long long K, const float *__restrict__ act_step, const int *__restrict__ act_zp,
+                  const int *__restrict__ rx, const float *__restrict__ w_step, const int *__restrict__ w_zp,
+                  const int *__restrict__ cw, const float *__restrict__ bias_q, const uint16_t *__restrict__ bias,
+                  double *__restrict__ partial, long long block0)
+{
+    pdl_begin();
+    const long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= C_out) return;
+    const long long r0 = (long long)blockIdx.y * kFcRowBlock, r1 = min(rows, r0 + (long long)kFcRowBlock);
+    const double sw = (double)w_step[o];
+    const long long zw = w_zp[o], cwo = cw[o];
+    const double bq = bias_q ? (double)bias_q[o] : 0.0;
+    const double b = bias ? (double)D::one(bias[o]) : 0.0;
+    double sd = 0.0, sd2 = 0.0, sy2 = 0.0;
+    for (long long n = r0; n < r1; ++n) {
+        const long long zx = act_zp[n];
+        long long dot = S[n * C_out + o];
+        if (S2) dot += S2[n * C_out + o];
+        const long long acc = dot - zx * cwo - zw * (long long)rx[n] + K * zx * zw;
+        const double yq = (double)act_step[n] * sw * (double)acc + bq;
+        const double y = (double)Y[n * C_out + o] + b;
+        const double d = yq - y;
+        sd += d;
+        sd2 += d * d;
+        sy2 += y * y;
+    }
+    double *out = partial + ((block0 + blockIdx.y) * C_out + o) * 3;
+    out[0] = sd;
+    out[1] = sd2;
+    out[2] = sy2;
+}
+
+__global__ void __launch_bounds__(256)
+fc_finish_kernel(const double *__restrict__ partial, long long nblocks, long long C_out, long long N,
+                 double *__restrict__ mean_err, double *__restrict__ col_sums)
+{
+    pdl_begin();
+    const long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= C_out) return;
+    double sd = 0.0, sd2 = 0.0, sy2 = 0.0;
+    for (long long k = 0; k < nblocks; ++k) {
+        const double *p = partial + (k * C_out + o) * 3;
+        sd += p[0];
+        sd2 += p[1];
+        sy2 += p[2];
+    }
+    mean_err[o] = sd / (double)N;
+    col_sums[o * 2] = sd2;
+    col_sums[o * 2 + 1] = sy2;
+}
+
+// sums[0] = sum (y~ - y)^2, sums[1] = sum y^2, sums[2] = sum_o mean_err_o^2, sums[3] = N * C_out
+__global__ void __launch_bounds__(256)
+fc_total_kernel(const double *__restrict__ col_sums, const double *__restrict__ mean_err, long long C_out, long long N,
+                double *__restrict__ sums)
+{
+    pdl_begin();
+    __shared__ double sh[3][256];
+    double a = 0.0, b = 0.0, c = 0.0;
+    for (long long o = threadIdx.x; o < C_out; o += 256) {
+        a += col_sums[o * 2];
+        b += col_sums[o * 2 + 1];
+        c += mean_err[o] * mean_err[o];
+    }
+    sh[0][threadIdx.x] = a;
+    sh[1][threadIdx.x] = b;
+    sh[2][threadIdx.x] = c;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if ((int)threadIdx.x < w)
+            for (int q = 0; q < 3; ++q) sh[q][threadIdx.x] += sh[q][threadIdx.x + w];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        sums[0] = sh[0][0];
+        sums[1] = sh[1][0];
+        sums[2] = sh[2][0];
+        sums[3] = (double)N * (double)C_out;
+    }
+}
+
+aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, const int *act_zp,
+                              const unsigned char *Wq, const float *w_step, const int *w_zp, const float *bias_q,
+                              const void *X, const void *W, aweq_dtype dt, const void *bias, long long N,
+                              long long C_in, long long C_out, double *mean_err, double *sums, void *ws,
+                              size_t ws_bytes, cudaStream_t stream)
+{
+    const FcLayout L = fc_layout(N, C_in, C_out);
+    if (L.total > ws_bytes) return AWEQ_ERR_WORKSPACE;
+    char *base = reinterpret_cast<char *>(ws);
+    int *S = reinterpret_cast<int *>(base + L.S);
+    const bool split = C_in > kFcSplitK;
+    int *S2 = split ? reinterpret_cast<int *>(base + L.S2) : nullptr;
+    float *Y = reinterpret_cast<float *>(base + L.Y);
+    int *rx = reinterpret_cast<int *>(base + L.rx);
+    int *cw = reinterpret_cast<int *>(base + L.cw);
+    double *partial = reinterpret_cast<double *>(base + L.partial);
+    void *scratch = base + L.scratch;
+    // K-halves: the first one a multiple of 128 so that the second starts on a tile boundary
+    const long long K0 = split ? (C_in / 2 + 127) / 128 * 128 : C_in;
+
+    AWEQ_LAUNCH(fc_rowsum_kernel, dim3((unsigned)((N + 7) / 8)), dim3(256), 0, stream, Xq, N, C_in, rx);
+    AWEQ_LAUNCH(fc_rowsum_kernel, dim3((unsigned)((C_out + 7) / 8)), dim3(256), 0, stream, Wq, C_out, C_in, cw);
+    for (long long c = 0; c < L.nchunks; ++c) {
+        const long long n0 = c * kFcChunk;
+        const long long rows = (N - n0) < kFcChunk ? (N - n0) : kFcChunk;
+        aweq_status rc = fc_gemm_u8(Xq + n0 * C_in, Wq, S, (int)rows, (int)C_out, (int)K0, C_in, scratch, kFcScratch, stream);
+        if (rc != AWEQ_OK) return rc;
+        if (split) {
+            rc = fc_gemm_u8(Xq + n0 * C_in + K0, Wq + K0, S2, (int)rows, (int)C_out, (int)(C_in - K0), C_in, scratch,
+                            kFcScratch, stream);
+            if (rc != AWEQ_OK) return rc;
+        }
+        const uint16_t *Xc = reinterpret_cast<const uint16_t *>(X) + n0 * C_in;
+        rc = (dt == AWEQ_F16 ? fc_gemm_f16 : fc_gemm_bf16)(Xc, W, Y, (int)rows, (int)C_out, (int)C_in, C_in, scratch,
+                                                           kFcScratch, stream);
+        if (rc != AWEQ_OK) return rc;
+        const dim3 grid((unsigned)((C_out + 255) / 256), (unsigned)((rows + kFcRowBlock - 1) / kFcRowBlock));
+        if (dt == AWEQ_F16)
+            AWEQ_LAUNCH(fc_compare_kernel<F16>, grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
+                        (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
+                        w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, c * L.blocks_per_chunk);
+        else
+            AWEQ_LAUNCH(fc_compare_kernel<BF16>, grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
+                        (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
+                        w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, c * L.blocks_per_chunk);
+    }
+    double *cs = reinterpret_cast<double *>(Y);        // Y is free now: two doubles per output channel
+    AWEQ_LAUNCH(fc_finish_kernel, dim3((unsigned)((C_out + 255) / 256)), dim3(256), 0, stream, (const double *)partial,
+                L.nblocks, C_out, N, mean_err, cs);
+    AWEQ_LAUNCH(fc_total_kernel, dim3(1), dim3(256), 0, stream, (const double *)cs, (const double *)mean_err, C_out, N, sums);
+    return AWEQ_OK;
+}
+
+}  // namespace aweq

@@ -36,4 +36,19 @@ aweq_status run_bias_gemv(const void *W, aweq_dtype dt, long long C_out, long lo
                           const float *mu_hat, int bits, int gran, int group, const void *bias_in, void *bias_out,
                           float *bias_out_f32, aweq_dtype bias_dt, cudaStream_t stream);
 
+// forward check (tensor-core GEMMs + comparison)
+size_t forward_check_ws_bytes(long long N, long long C_in, long long C_out);
+aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, const int *act_zp,
+                              const unsigned char *Wq, const float *w_step, const int *w_zp, const float *bias_q,
+                              const void *X, const void *W, aweq_dtype dt, const void *bias, long long N,
+                              long long C_in, long long C_out, double *mean_err, double *sums, void *ws,
+                              size_t ws_bytes, cudaStream_t stream);
+// C[M x N] = A[M x K] B[N x K]^T on the tensor cores; A and B have ld elements per row
+aweq_status fc_gemm_u8(const void *A, const void *B, void *C, int M, int N, int K, long long ld, void *scratch,
+                       size_t scratch_bytes, cudaStream_t stream);
+aweq_status fc_gemm_f16(const void *A, const void *B, void *C, int M, int N, int K, long long ld, void *scratch,
+                        size_t scratch_bytes, cudaStream_t stream);
+aweq_status fc_gemm_bf16(const void *A, const void *B, void *C, int M, int N, int K, long long ld, void *scratch,
+                         size_t scratch_bytes, cudaStream_t stream);
+
 }  // namespace aweq
