@@ -25,6 +25,8 @@
  *   quantiser ............ Eq. 1 and Eq. 2.
  *   bias correction ...... Eq. 11 - Eq. 15 and the sentence after them
  *                          (subtract eps * E[x]); eps = W~ - W.
+ *   forward check ........ Eq. 11 (E[y~ - y]) evaluated on data from the
+ *                          Eq. 1-2 de-quantised codes and the 16-bit layer.
  *
  * Conventions the paper does not fix (parity unpinned: both sides simply
  * follow the same rule):
@@ -538,4 +540,55 @@ void oracle_quant_act(const uint16_t *X, int dtype, int64_t N, int64_t C, int64_
             Xq[n * C + j] = (uint8_t)code_of(xh[j], st, inv, z, bits, literal_division);
         free(xh);
     }
+}
+
+/* ------------------------------------------------------------------ */
+/* Forward check of a calibrated W8A8 layer.  Eq. 11 names the         */
+/* expected output error E[y~_j - y_j] that quantisation leaves behind */
+/* and that bias correction (Eq. 15) removes; this routine evaluates   */
+/* it, and the output MSE, straight from the definitions, in fp64:     */
+/*   y~[n,o] = sum_k Step^x_n (Xq[n,k]-Z^x_n) Step^w_o (Wq[o,k]-Z^w_o) */
+/*             + bias_q[o]                 (Eq. 1-2 de-quantisation)   */
+/*   y[n,o]  = sum_k X[n,k] W[o,k] + bias[o]   (the 16-bit layer; the  */
+/*             product is unchanged by equalisation, Eq. 3)            */
+/*   mean_err[o] = (1/N) sum_n (y~ - y),                               */
+/*   sums = { sum (y~-y)^2, sum y^2, sum_o mean_err[o]^2, N*C_out }.   */
+/* One byte per code; bias_q / bias may be NULL (zeros).               */
+/* ------------------------------------------------------------------ */
+void oracle_forward_check(const uint8_t *Xq, const float *act_step, const int32_t *act_zp,
+                          const uint8_t *Wq, const float *w_step, const int32_t *w_zp, const float *bias_q,
+                          const uint16_t *X, const uint16_t *W, int dtype, const uint16_t *bias,
+                          int64_t N, int64_t C_in, int64_t C_out, double *mean_err, double *sums)
+{
+    double *sq = (double *)calloc((size_t)C_out * 2, sizeof(double));
+#pragma omp parallel for schedule(static)
+    for (int64_t o = 0; o < C_out; ++o) {
+        double sd = 0.0, sd2 = 0.0, sy2 = 0.0;
+        for (int64_t n = 0; n < N; ++n) {
+            double yq = 0.0, y = 0.0;
+            for (int64_t k = 0; k < C_in; ++k) {
+                double xq = (double)act_step[n] * (double)((int64_t)Xq[n * C_in + k] - (int64_t)act_zp[n]);
+                double wq = (double)w_step[o] * (double)((int64_t)Wq[o * C_in + k] - (int64_t)w_zp[o]);
+                yq += xq * wq;
+                y += (double)decode16(X[n * C_in + k], dtype) * (double)decode16(W[o * C_in + k], dtype);
+            }
+            if (bias_q) yq += (double)bias_q[o];
+            if (bias) y += (double)decode16(bias[o], dtype);
+            double d = yq - y;
+            sd += d;
+            sd2 += d * d;
+            sy2 += y * y;
+        }
+        mean_err[o] = sd / (double)N;
+        sq[2 * o] = sd2;
+        sq[2 * o + 1] = sy2;
+    }
+    sums[0] = sums[1] = sums[2] = 0.0;
+    for (int64_t o = 0; o < C_out; ++o) {
+        sums[0] += sq[2 * o];
+        sums[1] += sq[2 * o + 1];
+        sums[2] += mean_err[o] * mean_err[o];
+    }
+    sums[3] = (double)N * (double)C_out;
+    free(sq);
 }

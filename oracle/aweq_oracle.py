@@ -221,3 +221,22 @@ def quant_act(X, dtype, rinv, gran=PER_ROW, lo_hi=None, bits=8, literal_division
     _load().oracle_quant_act(_p(X), ci(dtype), i64(N), i64(C), i64(C), _p(rinv), ci(gran), _p(lo_hi),
                              ci(bits), ci(int(literal_division)), _p(Xq), _p(step), _p(zp))
     return Xq, step, zp
+
+
+def forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, dtype, bias=None):
+    """Eq. 11 evaluated on data -> (mean_err[C_out] f64, sums[4] f64): quantised layer against
+    the 16-bit layer (one byte per code; ``bias_q`` binary32 or None; ``bias`` raw 16-bit or None)."""
+    X, W = _u16(X), _u16(W)
+    N, C_in = X.shape
+    C_out = W.shape[0]
+    Xq = np.ascontiguousarray(Xq, dtype=np.uint8)
+    Wq = np.ascontiguousarray(Wq, dtype=np.uint8)
+    assert Xq.shape == (N, C_in) and Wq.shape == (C_out, C_in)
+    mean_err = np.empty(C_out, np.float64)
+    sums = np.empty(4, np.float64)
+    bias = None if bias is None else _u16(bias)
+    _load().oracle_forward_check(_p(Xq), _p(_f32(act_step)), _p(np.ascontiguousarray(act_zp, dtype=np.int32)),
+                                 _p(Wq), _p(_f32(w_step)), _p(np.ascontiguousarray(w_zp, dtype=np.int32)),
+                                 _p(_f32(bias_q)), _p(X), _p(W), ci(dtype), _p(bias), i64(N), i64(C_in), i64(C_out),
+                                 _p(mean_err), _p(sums))
+    return mean_err, sums

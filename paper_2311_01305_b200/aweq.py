@@ -73,8 +73,12 @@ _lib.aweq_quant_act.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _i, _i, _vp, _vp, _
 _lib.aweq_layer_pass_workspace_bytes.restype = _sz
 _lib.aweq_layer_pass_workspace_bytes.argtypes = [ctypes.POINTER(LayerArgs)]
 _lib.aweq_layer_pass.argtypes = [ctypes.POINTER(LayerArgs), _vp, _sz, _vp, _vp]
+_lib.aweq_forward_check_workspace_bytes.restype = _sz
+_lib.aweq_forward_check_workspace_bytes.argtypes = [_ll, _ll, _ll]
+_lib.aweq_forward_check.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _ll, _ll, _ll, _vp, _vp, _vp,
+                                    _sz, _vp]
 for _f in ("aweq_stats", "aweq_wrange", "aweq_factors", "aweq_equalize_quantize", "aweq_bias_correct",
-           "aweq_quant_act", "aweq_layer_pass"):
+           "aweq_quant_act", "aweq_layer_pass", "aweq_forward_check"):
     getattr(_lib, _f).restype = _i
 
 
@@ -193,6 +197,25 @@ def aweq_bias_correct(epsmu, W, s, codes, step, zp, mu_hat, bits, gran, group, b
 def aweq_quant_act(X, rinv, bits, gran, tensor_lo_hi, Xq, step, zp, st=None):
     _check(_lib.aweq_quant_act(_ptr(X), dtype_tag(X), X.shape[0], X.shape[1], _ld(X), _ptr(rinv), bits, gran,
                                _ptr(tensor_lo_hi), _ptr(Xq), _ptr(step), _ptr(zp), _ptr(st), _stream()))
+
+
+def forward_check_workspace_bytes(N: int, C_in: int, C_out: int) -> int:
+    return int(_lib.aweq_forward_check_workspace_bytes(N, C_in, C_out))
+
+
+def aweq_forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, bias, mean_err, sums, ws=None):
+    """Mean output error per output channel and sums of squares of the quantised layer
+    against the 16-bit layer (argument marshalling only; see ``include/aweq.h``)."""
+    N, C_in = X.shape
+    C_out = W.shape[0]
+    if not (X.is_contiguous() and W.is_contiguous() and Xq.is_contiguous() and Wq.is_contiguous()):
+        raise ValueError("aweq_forward_check takes contiguous matrices")
+    if ws is None:
+        ws = workspace(forward_check_workspace_bytes(N, C_in, C_out), X.device)
+    _check(_lib.aweq_forward_check(_ptr(Xq), _ptr(act_step), _ptr(act_zp), _ptr(Wq), _ptr(w_step), _ptr(w_zp),
+                                   _ptr(bias_q), _ptr(X), _ptr(W), dtype_tag(X), _ptr(bias), N, C_in, C_out,
+                                   _ptr(mean_err), _ptr(sums), _ptr(ws), ws.numel(), _stream()))
+    return ws
 
 
 def _parr(tensors: Optional[Sequence[Optional[torch.Tensor]]], n: int):

@@ -1,0 +1,147 @@
+"""Forward check (tensor-core GEMMs + comparison kernels) against the CPU oracle.
+
+The oracle evaluates both layers in binary64 straight from the definitions.  The GPU takes
+the integer product exactly and folds the zero-points in 64-bit integers, so the quantised
+side agrees to binary64 rounding; the 16-bit product is accumulated in binary32 by the
+tensor cores, so that side agrees exactly only where binary32 accumulation is exact
+(small-integer operands) and otherwise within the accumulation bound
+
+    |Y_gpu - Y| <= K * 2^-23 * sum_k |x_k w_k|      (K additions, each off by at most one
+                                                      unit in the last place of a partial sum)
+
+which the realistic case asserts element-wise through the means.  All oracle inputs are
+seeded or come from the oracle itself, never from the GPU.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import aweq_oracle as orc
+from paper_2311_01305_b200 import synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _run(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, bias):
+    from paper_2311_01305_b200 import aweq
+    t = lambda a, dt=None: None if a is None else torch.as_tensor(np.ascontiguousarray(a), dtype=dt).to(DEV)
+    C_out = W.shape[0]
+    mean_err, check_me = util.guarded((C_out,), torch.float64)
+    sums, check_s = util.guarded((4,), torch.float64)
+    aweq.aweq_forward_check(t(Xq), t(act_step, torch.float32), t(act_zp, torch.int32), t(Wq), t(w_step, torch.float32),
+                            t(w_zp, torch.int32), t(bias_q, torch.float32), X.to(DEV), W.to(DEV),
+                            None if bias is None else bias.to(DEV), mean_err, sums)
+    torch.cuda.synchronize()
+    check_me()
+    check_s()
+    return mean_err.cpu().numpy(), sums.cpu().numpy()
+
+
+def _int_valued(shape, dtype, seed, lim):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randint(-lim, lim + 1, shape, generator=g).to(dtype)
+
+
+def _codes(shape, seed, lo=0, hi=256):
+    return np.random.default_rng(seed).integers(lo, hi, shape).astype(np.uint8)
+
+
+# N, C_in, C_out: ragged token blocks and tiles; two token chunks; a K wide enough for the split product
+EXACT_SHAPES = [(1000, 768, 200), (77, 16, 8), (16384 + 300, 256, 64), (300, 32768 + 128, 16), (129, 4096, 136)]
+
+
+@pytest.mark.parametrize("N,C_in,C_out", EXACT_SHAPES)
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_forward_check_exact_operands(N, C_in, C_out, dtype):
+    """Operands whose binary32 accumulation is exact (|x|, |w| <= 3, integers): every output
+    must agree with the oracle to binary64 rounding, whatever the tile, chunk or K split."""
+    seed = N + C_in + C_out
+    rng = np.random.default_rng(seed)
+    Xq, Wq = _codes((N, C_in), seed), _codes((C_out, C_in), seed + 1)
+    act_step = rng.uniform(0.01, 0.05, N).astype(np.float32)
+    act_zp = rng.integers(0, 256, N).astype(np.int32)
+    w_step = rng.uniform(0.001, 0.01, C_out).astype(np.float32)
+    w_zp = rng.integers(-40, 300, C_out).astype(np.int32)
+    bias_q = rng.standard_normal(C_out).astype(np.float32)
+    X = _int_valued((N, C_in), dtype, seed + 2, 3)
+    W = _int_valued((C_out, C_in), dtype, seed + 3, 3)
+    bias = _int_valued((C_out,), dtype, seed + 4, 5)
+    got_me, got_s = _run(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, bias)
+    dt = util.odt(X)
+    ref_me, ref_s = orc.forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, util.bits(X), util.bits(W), dt,
+                                      util.bits(bias))
+    rms = np.sqrt(ref_s[0] / ref_s[3])
+    assert np.all(np.abs(got_me - ref_me) <= 1e-11 * rms)
+    assert np.allclose(got_s, ref_s, rtol=1e-11, atol=0)
+
+
+def test_forward_check_extreme_codes_do_not_overflow():
+    """All codes 255 at the widest unsplit K and across the split: the int32 partial products
+    stay below 2^31 and the 64-bit fold is exact."""
+    for C_in in (32768, 32768 + 4096):
+        N, C_out = 40, 8
+        Xq = np.full((N, C_in), 255, np.uint8)
+        Wq = np.full((C_out, C_in), 255, np.uint8)
+        one_n, one_o = np.ones(N, np.float32), np.ones(C_out, np.float32)
+        zero_n, zero_o = np.zeros(N, np.int32), np.zeros(C_out, np.int32)
+        X = torch.zeros((N, C_in), dtype=torch.float16)
+        W = torch.zeros((C_out, C_in), dtype=torch.float16)
+        got_me, got_s = _run(Xq, one_n, zero_n, Wq, one_o, zero_o, None, X, W, None)
+        assert np.all(got_me == 255.0 * 255.0 * C_in)
+        assert got_s[1] == 0.0 and got_s[3] == N * C_out
+        # and with the largest zero-points: every term cancels
+        got_me, _ = _run(Xq, one_n, zero_n + 255, Wq, one_o, zero_o + 255, None, X, W, None)
+        assert np.all(got_me == 0.0)
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("correct", [True, False])
+def test_forward_check_of_a_calibrated_layer(dtype, correct):
+    """The whole chain on a realistic layer: oracle calibration (steps 1-6) feeds both sides."""
+    N, C_in, C_out = 1536 + 40, 768, 1024 + 8
+    Xc = util.rand16((N, C_in), dtype, 41, scale=1.0, offset=0.5, outlier_cols=4)
+    Wc = util.rand16((C_out, C_in), dtype, 42, scale=0.03)
+    bias = util.rand16((1, C_out), dtype, 43, scale=0.1)[0].contiguous()
+    cal = util.oracle_layer(Xc, [Wc], 8, orc.PER_ROW, 0, biases=[bias], bias_correct=True)
+    lin, (Xq, act_step, act_zp) = cal["linears"][0], cal["act"]
+    dt = util.odt(Xc)
+    bias_q = lin["bias_f32"] if correct else orc.decode16(util.bits(bias), dt)
+    got_me, got_s = _run(Xq, act_step, act_zp, lin["codes"], lin["step"], lin["zp"], bias_q, Xc, Wc, bias)
+    ref_me, ref_s = orc.forward_check(Xq, act_step, act_zp, lin["codes"], lin["step"], lin["zp"], bias_q,
+                                      util.bits(Xc), util.bits(Wc), dt, util.bits(bias))
+    Xa, Wa = np.abs(Xc.double().numpy()), np.abs(Wc.double().numpy())
+    bound = C_in * 2.0 ** -23 * (Xa @ Wa.T)                       # per-output accumulation bound
+    assert np.all(np.abs(got_me - ref_me) <= bound.mean(axis=0))
+    # sum d^2: |sum (d+e)^2 - sum d^2| <= 2 sqrt(sum d^2 sum e^2) + sum e^2
+    e2 = (bound ** 2).sum()
+    assert abs(got_s[0] - ref_s[0]) <= 2 * np.sqrt(ref_s[0] * e2) + e2
+    assert abs(got_s[1] - ref_s[1]) <= 2 * np.sqrt(ref_s[1] * e2) + e2
+    assert got_s[3] == ref_s[3]
+    # in practice the accumulation error is far inside the bound: the means agree to 1e-5 of the output scale
+    y_rms = np.sqrt(ref_s[1] / ref_s[3])
+    assert np.abs(got_me - ref_me).max() <= 1e-5 * y_rms
+    if correct:
+        # activation rounding is the only source of mean error left (Eq. 11-15 remove the weights' part)
+        raw = cal["linears"][0]["delta"]
+        assert np.abs(ref_me).max() < np.abs(raw).max()
+
+
+def test_forward_check_rejects_bad_arguments():
+    from paper_2311_01305_b200 import aweq
+    N, C_in, C_out = 32, 24, 8                                     # C_in not a multiple of 16
+    z = lambda shape, dt: torch.zeros(shape, dtype=dt, device=DEV)
+    with pytest.raises(aweq.AweqError) as e:
+        aweq.aweq_forward_check(z((N, C_in), torch.uint8), z(N, torch.float32), z(N, torch.int32),
+                                z((C_out, C_in), torch.uint8), z(C_out, torch.float32), z(C_out, torch.int32), None,
+                                z((N, C_in), torch.float16), z((C_out, C_in), torch.float16), None,
+                                z(C_out, torch.float64), z(4, torch.float64), ws=aweq.workspace(1 << 22))
+    assert e.value.code == 2          # AWEQ_ERR_SHAPE
+    C_in = 32
+    with pytest.raises(aweq.AweqError) as e:
+        aweq.aweq_forward_check(z((N, C_in), torch.uint8), z(N, torch.float32), z(N, torch.int32),
+                                z((C_out, C_in), torch.uint8), z(C_out, torch.float32), z(C_out, torch.int32), None,
+                                z((N, C_in), torch.float16), z((C_out, C_in), torch.float16), None,
+                                z(C_out, torch.float64), z(4, torch.float64), ws=aweq.workspace(4096))
+    assert e.value.code == 7          # AWEQ_ERR_WORKSPACE

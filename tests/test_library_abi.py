@@ -59,12 +59,21 @@ def test_validation_rejects_null_before_any_cuda_call(lib):
     assert lib.aweq_factors(None, None, None, None, None, 8, None, None, None, None, None, None, None, None) == 1
     lib.aweq_layer_pass.argtypes = [vp, vp, sz, vp, vp]
     assert lib.aweq_layer_pass(None, None, 0, None, None) == 1
+    lib.aweq_forward_check.argtypes = [vp] * 9 + [i, vp, ll, ll, ll, vp, vp, vp, sz, vp]
+    assert lib.aweq_forward_check(*([None] * 9), 0, None, 64, 64, 64, None, None, None, 0, None) == 1
+    lib.aweq_forward_check_workspace_bytes.restype = sz
+    lib.aweq_forward_check_workspace_bytes.argtypes = [ll, ll, ll]
+    small = lib.aweq_forward_check_workspace_bytes(100, 768, 768)
+    assert 0 < small < 8 << 20
+    # bounded by the token chunk: the intermediates do not grow with N
+    assert lib.aweq_forward_check_workspace_bytes(1 << 20, 4096, 4096) < 1 << 30
+    assert lib.aweq_forward_check_workspace_bytes(0, 64, 64) == 0
 
 
 def test_binding_imports_and_names_match_header():
     from paper_2311_01305_b200 import aweq
     for name in declared_functions():
         if name in ("aweq_strerror", "aweq_last_cuda_error", "aweq_version", "aweq_launch_count",
-                    "aweq_workspace_bytes", "aweq_layer_pass_workspace_bytes"):
+                    "aweq_workspace_bytes", "aweq_layer_pass_workspace_bytes", "aweq_forward_check_workspace_bytes"):
             continue
         assert hasattr(aweq, name), name

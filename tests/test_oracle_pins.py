@@ -455,3 +455,87 @@ def test_equalization_reduces_activation_quantization_error():
         Wh = Wd * sv[None, :]
         return np.mean((Xdq @ Wh.T - Xd @ Wd.T) ** 2)
     assert out_err(f["rinv"], f["s"]) < 0.2 * out_err(None, None)
+
+
+# ---------------------------------------------------------------- forward check, Eq. 11 on data
+def test_forward_check_hand_worked():
+    """A 2-token, 2-input, 3-output layer worked by hand (all values exact in binary):
+    X~ = Step^x (Xq - Z^x) = [[1, 0], [0, 4]],  W~ = Step^w (Wq - Z^w) = [[0, 4], [1, 0], [-2, 1]],
+    y~ = X~ W~^T + bias_q = [[0, 1, -2], [16, 0, 4]] + [0.5, -1, 0] = [[0.5, 0, -2], [16.5, -1, 4]],
+    y  = X W^T + bias with X = [[1, .5], [0, 4]], W = [[.5, 4], [1, .25], [-2, 1]], bias = [0, 1, 0]
+       = [[2.5, 2.125, -1.5], [16, 2, 4]],
+    d  = y~ - y = [[-2, -2.125, -0.5], [0.5, -3, 0]]."""
+    Xq = np.array([[3, 1], [2, 6]], np.uint8)
+    act_step, act_zp = [0.5, 1.0], [1, 2]
+    Wq = np.array([[2, 4], [5, 1], [0, 3]], np.uint8)
+    w_step, w_zp = [2.0, 0.25, 1.0], [2, 1, 2]
+    bias_q = np.array([0.5, -1.0, 0.0], np.float32)
+    X = f16_bits([[1, 0.5], [0, 4]])
+    W = f16_bits([[0.5, 4], [1, 0.25], [-2, 1]])
+    bias = f16_bits([0, 1, 0])
+    mean_err, sums = orc.forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, orc.F16, bias)
+    assert mean_err.tolist() == [-0.75, -2.5625, -0.25]
+    assert sums.tolist() == [4 + 4.515625 + 0.25 + 0.25 + 9 + 0,
+                             6.25 + 4.515625 + 2.25 + 256 + 4 + 16,
+                             0.5625 + 6.56640625 + 0.0625, 6.0]
+    # without the optional biases
+    mean_err0, _ = orc.forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, None, X, W, orc.F16, None)
+    assert mean_err0.tolist() == [-0.75 - 0.5, -2.5625 + 1 + 1, -0.25]
+
+
+def test_forward_check_against_numpy_matmul_and_bf16():
+    rng = np.random.default_rng(31)
+    N, C_in, C_out = 37, 48, 20
+    Xq = rng.integers(0, 256, (N, C_in)).astype(np.uint8)
+    Wq = rng.integers(0, 256, (C_out, C_in)).astype(np.uint8)
+    act_step = rng.uniform(0.01, 0.05, N).astype(np.float32)
+    act_zp = rng.integers(0, 256, N).astype(np.int32)
+    w_step = rng.uniform(0.001, 0.01, C_out).astype(np.float32)
+    w_zp = rng.integers(-40, 300, C_out).astype(np.int32)          # a zero-point may lie outside the code range
+    bias_q = rng.standard_normal(C_out).astype(np.float32)
+    for dt, to_bits in ((orc.F16, f16_bits), (orc.BF16, bf16_bits)):
+        X, W, b = to_bits(rng.standard_normal((N, C_in))), to_bits(rng.standard_normal((C_out, C_in)) * 0.1), \
+            to_bits(rng.standard_normal(C_out))
+        mean_err, sums = orc.forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, dt, b)
+        Xt = act_step.astype(np.float64)[:, None] * (Xq.astype(np.float64) - act_zp[:, None])
+        Wt = w_step.astype(np.float64)[:, None] * (Wq.astype(np.float64) - w_zp[:, None])
+        yq = Xt @ Wt.T + bias_q.astype(np.float64)[None, :]
+        y = bits_to_f64(X, dt) @ bits_to_f64(W, dt).T + bits_to_f64(b, dt)[None, :]
+        d = yq - y
+        assert np.allclose(mean_err, d.mean(axis=0), rtol=1e-12, atol=1e-12)
+        assert np.allclose(sums, [(d * d).sum(), (y * y).sum(), (d.mean(axis=0) ** 2).sum(), N * C_out], rtol=1e-12)
+
+
+def test_forward_check_sees_what_bias_correction_removes():
+    """Eq. 11-15 tie three oracle routines together.  With activations that the 8-bit grid holds
+    exactly, the mean output error of the quantised layer is eps . E[x^] (the step-4 sums), and
+    it vanishes once the step-5 bias is used."""
+    rng = np.random.default_rng(32)
+    N, C_in, C_out = 120, 32, 10
+    Xq = rng.integers(0, 256, (N, C_in)).astype(np.uint8)
+    Xq[:, 0], Xq[:, 1] = 0, 255                                    # every token spans the whole code range
+    act_zp = rng.integers(100, 140, N).astype(np.int32)
+    act_step = np.full(N, 2.0 ** -6, np.float32)
+    Xhat = (Xq.astype(np.float64) - act_zp[:, None]) * 2.0 ** -6   # |x^| < 4, multiples of 1/64: exact in fp16
+    s = np.ones(C_in, np.float32)                                  # identity equalisation: X = X^
+    mu_hat = Xhat.mean(axis=0).astype(np.float32)
+    Wd = (rng.standard_normal((C_out, C_in)) * 0.05).astype(np.float16)
+    codes, w_step, w_zp, delta = orc.equalize_quantize(Wd.view(np.uint16), orc.F16, s, mu_hat, 8, orc.PER_ROW)
+    bias = f16_bits(rng.standard_normal(C_out) * 0.1)
+    bf, _ = orc.bias_correct(delta, bias, orc.F16)
+    X = f16_bits(Xhat)
+    assert np.array_equal(bits_to_f64(X, orc.F16), Xhat)
+    # the activation quantiser reproduces these codes, so step 6 and the check agree on the grid
+    q_codes, q_step, q_zp = orc.quant_act(X, orc.F16, None)
+    assert np.array_equal(q_codes, Xq) and np.array_equal(q_zp, act_zp) and np.array_equal(q_step, act_step)
+    raw, _ = orc.forward_check(Xq, act_step, act_zp, codes, w_step, w_zp, bits_to_f64(bias, orc.F16).astype(np.float32),
+                               X, Wd.view(np.uint16), orc.F16, bias)
+    fixed, sums = orc.forward_check(Xq, act_step, act_zp, codes, w_step, w_zp, bf, X, Wd.view(np.uint16), orc.F16, bias)
+    mu64 = mu_hat.astype(np.float64)
+    scale = np.abs(delta).max()
+    assert np.allclose(raw, delta + (Xhat.mean(axis=0) - mu64) @ (orc.dequantize(codes, w_step, w_zp, C_in, 8, orc.PER_ROW)
+                                                                     - Wd.astype(np.float64)).T, rtol=0, atol=1e-9 * scale)
+    # what is left: binary32 rounding of mu_hat (relative 2^-24 of the sums) and of bias' (half an ulp)
+    assert np.abs(fixed).max() <= 1e-6 * scale + 2.0 ** -24 * np.abs(bf).max()
+    assert np.abs(raw).max() > 1000 * np.abs(fixed).max()
+    assert sums[3] == N * C_out and sums[2] == pytest.approx((fixed ** 2).sum(), rel=1e-12)
