@@ -37,6 +37,7 @@ from paper_2311_01305_b200 import synth  # noqa: E402
 DEFAULT_WORKLOAD = "llama7b_layer_w4w3_g128"
 NORTH_STAR_PEAK_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0
 
 
 def measured_peaks():
@@ -163,6 +164,57 @@ def run_reference(args, wl, bits):
     print(json.dumps(line))
 
 
+def run_forward_check(args, wl, bits):
+    """Secondary benchmark: the forward check of every linear of a calibrated W8A8 layer.
+    A step is one check of the whole layer; the work is two dense contractions per linear
+    (unsigned 8-bit and 16-bit, 2 N C_in C_out flops each), so the bound is the tensor pipe.
+    The peak is the measured 16-bit GEMM rate scaled for the mix: the 8-bit half runs at
+    twice the 16-bit rate (nominal ratio), so 2F flops take at best 1.5 F / P16."""
+    from paper_2311_01305_b200 import aweq, calibrate
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    X, W = generate(wl, dev, 0)
+    cal = calibrate.LayerCalibrator(wl, bits, X, W, None)
+    cal.run()
+    for _ in range(max(1, args.warmup)):
+        res = cal.forward_check(X, W)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.15)
+    n0 = aweq.launch_count()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        res = cal.forward_check(X, W)
+    b.record()
+    torch.cuda.synchronize()
+    launches = aweq.launch_count() - n0
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b) / args.steps
+    tokens = {i.name: i.n_tokens for i in wl.inputs}
+    flops = sum(4.0 * tokens[l.input] * l.c_in * l.c_out for l in wl.linears)
+    p16 = FALLBACK_BF16_TFLOPS
+    kind = "fallback"
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        p16, kind = float(json.load(open(pk))["bf16_tflops_sustained"]), "measured (sustained)"
+    peak = p16 * 2.0 / 1.5
+    tf = flops / ms / 1e9
+    worst = {n: float((me.abs().max() / (s4[1] / s4[3]).sqrt()).item()) for n, (me, s4) in res.items()}
+    sqnr = {n: float(10.0 * torch.log10(s4[1] / s4[0]).item()) for n, (me, s4) in res.items()}
+    print(json.dumps({
+        "metric": "aweq_forward_check_tflops", "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(1, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8 x u8 -> s32 and %s -> f32" % wl.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "tokens": tokens, "linears": [l.name for l in wl.linears],
+                   "cache": "operands (GBs) far larger than the 126 MB L2"},
+        "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                     "peak_kind": "16-bit GEMM rate of %s x 4/3 for the 8-bit / 16-bit mix" % kind, "traffic": None},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "max_abs_mean_err_over_output_rms": worst, "output_sqnr_db": sqnr}))
+
+
 def calibrate_bytes(wl, bits):
     from paper_2311_01305_b200 import calibrate
     return calibrate.algorithmic_bytes(wl, bits)
@@ -181,6 +233,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-tokens", type=int, default=131072)
+    ap.add_argument("--op", default="layer_pass", choices=["layer_pass", "forward_check"],
+                    help="forward_check: time the W8A8 forward check of the calibrated layer instead (1 GPU)")
     args = ap.parse_args()
 
     wl = synth.workloads(args.tokens_scale)[args.workload]
@@ -190,6 +244,8 @@ def main():
 
     from paper_2311_01305_b200 import aweq, calibrate
 
+    if args.op == "forward_check":
+        return run_forward_check(args, wl, bits)
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

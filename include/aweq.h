@@ -281,7 +281,8 @@ aweq_status aweq_layer_pass(const aweq_layer_args *args, void *ws, size_t ws_byt
  *   sums[4]          binary64: sum (y~ - y)^2, sum y^2, sum_o mean_err[o]^2, N * C_out
  * Layout: Xq [N x C_in] and Wq [C_out x C_in] one byte per code, X and W 16-bit, all
  * row-major, contiguous (no pitch) and 16-byte aligned; act_step/act_zp [N], w_step/w_zp
- * [C_out]; bias_q (binary32, [C_out]) and bias (16-bit, [C_out]) may be NULL (= 0).
+ * [C_out]; bias (16-bit, [C_out]) may be NULL (a layer without bias); bias_q (binary32,
+ * [C_out]) may be NULL: the quantised layer then keeps `bias` (no bias correction).
  * C_in must be a multiple of 16, C_out a multiple of 8 (AWEQ_ERR_SHAPE otherwise).
  * ws: aweq_forward_check_workspace_bytes(N, C_in, C_out) bytes, 256-byte aligned; nothing is
  * allocated.  Everything is enqueued on `stream`; the caller owns all buffers.

@@ -553,7 +553,8 @@ void oracle_quant_act(const uint16_t *X, int dtype, int64_t N, int64_t C, int64_
 /*             product is unchanged by equalisation, Eq. 3)            */
 /*   mean_err[o] = (1/N) sum_n (y~ - y),                               */
 /*   sums = { sum (y~-y)^2, sum y^2, sum_o mean_err[o]^2, N*C_out }.   */
-/* One byte per code; bias_q / bias may be NULL (zeros).               */
+/* One byte per code; bias may be NULL (zeros); bias_q may be NULL:    */
+/* the quantised layer then keeps bias (no correction applied).       */
 /* ------------------------------------------------------------------ */
 void oracle_forward_check(const uint8_t *Xq, const float *act_step, const int32_t *act_zp,
                           const uint8_t *Wq, const float *w_step, const int32_t *w_zp, const float *bias_q,
@@ -572,8 +573,9 @@ void oracle_forward_check(const uint8_t *Xq, const float *act_step, const int32_
                 yq += xq * wq;
                 y += (double)decode16(X[n * C_in + k], dtype) * (double)decode16(W[o * C_in + k], dtype);
             }
-            if (bias_q) yq += (double)bias_q[o];
             if (bias) y += (double)decode16(bias[o], dtype);
+            if (bias_q) yq += (double)bias_q[o];
+            else if (bias) yq += (double)decode16(bias[o], dtype);   /* uncorrected: the layer keeps its bias */
             double d = yq - y;
             sd += d;
             sd2 += d * d;

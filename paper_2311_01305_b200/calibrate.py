@@ -86,11 +86,36 @@ class LayerCalibrator:
             self.passes.append(lp)
         self.ws = aweq.workspace(ws_bytes, dev)
         self.status = aweq.new_status(dev)
+        self._fc_ws, self._fc_out = None, {}
 
     def run(self) -> None:
         """One calibration pass of the whole layer: one library call per input."""
         for lp in self.passes:
             lp(self.ws, self.status)
+
+    def forward_check(self, X, W, bias=None, corrected: bool = True):
+        """``aweq_forward_check`` for every linear of a W8A8 workload after ``run()``:
+        {linear name: (mean_err[C_out], sums[4])} as binary64 device tensors.  ``corrected``
+        gives the quantised layer the step-5 bias; otherwise it keeps the original one."""
+        wl = self.wl
+        if not (wl.act_quant and self.bits == 8 and wl.w_gran == "row"):
+            raise ValueError("the forward check covers W8A8 workloads with row-wise weight scales")
+        dev = self.ws.device
+        need = max(aweq.forward_check_workspace_bytes(X[l.input].shape[0], l.c_in, l.c_out) for l in wl.linears)
+        if self._fc_ws is None or self._fc_ws.numel() < need:
+            self._fc_ws = aweq.workspace(need, dev)
+        res = {}
+        for l in wl.linears:
+            o, lo = self.out[l.input], self.out[l.name]
+            if l.name not in self._fc_out:
+                self._fc_out[l.name] = (torch.empty(l.c_out, dtype=torch.float64, device=dev),
+                                        torch.empty(4, dtype=torch.float64, device=dev))
+            mean_err, sums = self._fc_out[l.name]
+            aweq.aweq_forward_check(o["Xq"], o["act_step"], o["act_zp"], lo["codes"], lo["step"], lo["zp"],
+                                    lo["bias_f32"] if corrected else None, X[l.input], W[l.name],
+                                    None if bias is None else bias.get(l.name), mean_err, sums, ws=self._fc_ws)
+            res[l.name] = (mean_err, sums)
+        return res
 
 
 def allreduce_stats(xmin: torch.Tensor, xmax: torch.Tensor, xsum: torch.Tensor, count: torch.Tensor, group=None) -> None:

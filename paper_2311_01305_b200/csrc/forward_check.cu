@@ -89,8 +89,8 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
     const long long r0 = (long long)blockIdx.y * kFcRowBlock, r1 = min(rows, r0 + (long long)kFcRowBlock);
     const double sw = (double)w_step[o];
     const long long zw = w_zp[o], cwo = cw[o];
-    const double bq = bias_q ? (double)bias_q[o] : 0.0;
     const double b = bias ? (double)D::one(bias[o]) : 0.0;
+    const double bq = bias_q ? (double)bias_q[o] : b;           // no corrected bias: the layer keeps its own
     double sd = 0.0, sd2 = 0.0, sy2 = 0.0;
     for (long long n = r0; n < r1; ++n) {
         const long long zx = act_zp[n];

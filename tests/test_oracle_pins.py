@@ -478,9 +478,13 @@ def test_forward_check_hand_worked():
     assert sums.tolist() == [4 + 4.515625 + 0.25 + 0.25 + 9 + 0,
                              6.25 + 4.515625 + 2.25 + 256 + 4 + 16,
                              0.5625 + 6.56640625 + 0.0625, 6.0]
-    # without the optional biases
-    mean_err0, _ = orc.forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, None, X, W, orc.F16, None)
+    # without biases the products alone are compared; an uncorrected layer (bias_q None) keeps its bias,
+    # which cancels in y~ - y but counts in sum y^2
+    mean_err0, sums0 = orc.forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, None, X, W, orc.F16, None)
     assert mean_err0.tolist() == [-0.75 - 0.5, -2.5625 + 1 + 1, -0.25]
+    mean_err1, sums1 = orc.forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, None, X, W, orc.F16, bias)
+    assert mean_err1.tolist() == mean_err0.tolist() and sums1[0] == sums0[0]
+    assert sums0[1] == 6.25 + 1.265625 + 2.25 + 256 + 1 + 16 and sums1[1] == sums[1]
 
 
 def test_forward_check_against_numpy_matmul_and_bf16():
@@ -528,8 +532,7 @@ def test_forward_check_sees_what_bias_correction_removes():
     # the activation quantiser reproduces these codes, so step 6 and the check agree on the grid
     q_codes, q_step, q_zp = orc.quant_act(X, orc.F16, None)
     assert np.array_equal(q_codes, Xq) and np.array_equal(q_zp, act_zp) and np.array_equal(q_step, act_step)
-    raw, _ = orc.forward_check(Xq, act_step, act_zp, codes, w_step, w_zp, bits_to_f64(bias, orc.F16).astype(np.float32),
-                               X, Wd.view(np.uint16), orc.F16, bias)
+    raw, _ = orc.forward_check(Xq, act_step, act_zp, codes, w_step, w_zp, None, X, Wd.view(np.uint16), orc.F16, bias)
     fixed, sums = orc.forward_check(Xq, act_step, act_zp, codes, w_step, w_zp, bf, X, Wd.view(np.uint16), orc.F16, bias)
     mu64 = mu_hat.astype(np.float64)
     scale = np.abs(delta).max()
