@@ -18,12 +18,11 @@ namespace aweq {
 using namespace cute;
 
 
-template <class EA, class EB, class EC, class EAcc, int AlignAB, class Tile>
+template <class EA, class EB, class EC, class EAcc, int AlignAB, class Tile, class Cluster = Shape<_1, _1, _1>>
 struct FcGemm {
     using LayoutA = cutlass::layout::RowMajor;       // [M x K], K contiguous
     using LayoutB = cutlass::layout::ColumnMajor;    // [N x K] stored row-major = K contiguous
     using LayoutC = cutlass::layout::RowMajor;
-    using Cluster = Shape<_1, _1, _1>;
     static constexpr int AlignC = 128 / cutlass::sizeof_bits<EC>::value;
     using Epi = typename cutlass::epilogue::collective::CollectiveBuilder<
         cutlass::arch::Sm100, cutlass::arch::OpClassTensorOp, Tile, Cluster,
