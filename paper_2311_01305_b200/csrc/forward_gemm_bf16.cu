@@ -6,7 +6,7 @@ namespace aweq {
 aweq_status fc_gemm_bf16(const void *A, const void *B, void *C, int M, int N, int K, long long ld, void *scratch,
         size_t scratch_bytes, cudaStream_t stream)
 {
-    using G = FcGemm<cutlass::bfloat16_t, cutlass::bfloat16_t, float, float, 8, Shape<_128, _128, _64>>;
+    using G = FcGemm<cutlass::bfloat16_t, cutlass::bfloat16_t, float, float, 8, Shape<_256, _256, _64>, Shape<_2, _1, _1>>;
     return G::run(reinterpret_cast<const cutlass::bfloat16_t *>(A), reinterpret_cast<const cutlass::bfloat16_t *>(B), reinterpret_cast<float *>(C), M, N,
                   K, ld, scratch, scratch_bytes, stream);
 }

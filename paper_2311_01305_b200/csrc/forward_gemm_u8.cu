@@ -6,7 +6,7 @@ namespace aweq {
 aweq_status fc_gemm_u8(const void *A, const void *B, void *C, int M, int N, int K, long long ld, void *scratch,
         size_t scratch_bytes, cudaStream_t stream)
 {
-    using G = FcGemm<uint8_t, uint8_t, int32_t, int32_t, 16, Shape<_128, _128, _128>>;
+    using G = FcGemm<uint8_t, uint8_t, int32_t, int32_t, 16, Shape<_256, _256, _128>, Shape<_2, _1, _1>>;
     return G::run(reinterpret_cast<const uint8_t *>(A), reinterpret_cast<const uint8_t *>(B), reinterpret_cast<int32_t *>(C), M, N,
                   K, ld, scratch, scratch_bytes, stream);
 }
