@@ -203,6 +203,22 @@ def run_forward_check(args, wl, bits):
     tf = flops / ms / 1e9
     worst = {n: float((me.abs().max() / (s4[1] / s4[3]).sqrt()).item()) for n, (me, s4) in res.items()}
     sqnr = {n: float(10.0 * torch.log10(s4[1] / s4[0]).item()) for n, (me, s4) in res.items()}
+    # ablation (outside the timed region): equalisation and bias correction switched on and off
+    del cal
+    ablation = {}
+    for eq in (True, False):
+        for bc in (True, False):
+            flags = (0 if eq else aweq.FLAG_NO_EQUALIZE) | (0 if bc else aweq.FLAG_NO_BIAS_CORRECT)
+            c = calibrate.LayerCalibrator(wl, bits, X, W, None, flags=flags)
+            c.run()
+            r = c.forward_check(X, W, corrected=bc)
+            torch.cuda.synchronize()
+            ablation[("AWE" if eq else "no AWE") + (" + BC" if bc else "")] = {
+                "output_sqnr_db": {n: round(float(10.0 * torch.log10(s4[1] / s4[0]).item()), 3)
+                                   for n, (me, s4) in r.items()},
+                "rms_mean_err_over_output_rms": {n: float(((s4[2] / me.numel()) / (s4[1] / s4[3])).sqrt().item())
+                                                 for n, (me, s4) in r.items()}}
+            del c, r
     print(json.dumps({
         "metric": "aweq_forward_check_tflops", "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
         "warmup": max(1, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -212,7 +228,7 @@ def run_forward_check(args, wl, bits):
         "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
                      "peak_kind": "16-bit GEMM rate of %s x 4/3 for the 8-bit / 16-bit mix" % kind, "traffic": None},
         "clocks": clocks, "gpu_launches": int(launches),
-        "max_abs_mean_err_over_output_rms": worst, "output_sqnr_db": sqnr}))
+        "max_abs_mean_err_over_output_rms": worst, "output_sqnr_db": sqnr, "ablation": ablation}))
 
 
 def calibrate_bytes(wl, bits):
