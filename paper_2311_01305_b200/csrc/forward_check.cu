@@ -18,7 +18,7 @@
 namespace aweq {
 
 constexpr long long kFcChunk = 16384;          // tokens per chunk
-constexpr int kFcRowBlock = 256;               // tokens folded by one thread of the comparison kernel
+constexpr int kFcRowBlock = 128;               // tokens per CTA of the comparison kernel
 constexpr long long kFcSplitK = 32768;         // above this C_in the integer product is taken in two halves
 constexpr size_t kFcScratch = 1 << 20;         // scratch of the GEMMs
 
@@ -35,8 +35,7 @@ static FcLayout fc_layout(long long N, long long C_in, long long C_out)
     L.chunk = N < kFcChunk ? N : kFcChunk;
     L.nchunks = (N + kFcChunk - 1) / kFcChunk;
     L.blocks_per_chunk = (L.chunk + kFcRowBlock - 1) / kFcRowBlock;
-    const long long last_rows = N - (L.nchunks - 1) * kFcChunk;
-    L.nblocks = (L.nchunks - 1) * L.blocks_per_chunk + (last_rows + kFcRowBlock - 1) / kFcRowBlock;
+    L.nblocks = L.blocks_per_chunk;            // every chunk adds into the same slots
     size_t off = 0;
     L.S = off; off += up256((size_t)L.chunk * C_out * 4);
     L.S2 = off; off += C_in > kFcSplitK ? up256((size_t)L.chunk * C_out * 4) : 0;
@@ -73,41 +72,80 @@ __global__ void __launch_bounds__(256) fc_rowsum_kernel(const unsigned char *__r
     if (lane == 0) out[row] = (int)acc;
 }
 
-// One thread per output channel and block of kFcRowBlock tokens: form y~ and y, fold
-// d = y~ - y, d^2 and y^2 in binary64 in token order, one partial per (block, channel).
+// Comparison of one token chunk.  A CTA covers kFcRowBlock tokens x 128 output channels: a lane
+// owns four adjacent channels (16-byte loads of S and Y), the eight warps take the tokens
+// round-robin, and the per-warp sums are added in warp order through shared memory, so the
+// result does not depend on scheduling.  The integer part is formed in binary64, where it is
+// exact (every term is an integer below 2^53):
+//   acc = S - Z^x cw_o + Z^w (K Z^x - rx_n)
+// The CTA's sums of d = y~ - y, d^2 and y^2 go to partial[block][channel]; chunk after chunk
+// adds into the same slots in stream order.
 template <class D>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const float *__restrict__ Y, long long rows,
                   long long C_out, long long K, const float *__restrict__ act_step, const int *__restrict__ act_zp,
                   const int *__restrict__ rx, const float *__restrict__ w_step, const int *__restrict__ w_zp,
                   const int *__restrict__ cw, const float *__restrict__ bias_q, const uint16_t *__restrict__ bias,
-                  double *__restrict__ partial, long long block0)
+                  double *__restrict__ partial, int accumulate)
 {
     pdl_begin();
-    const long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= C_out) return;
+    __shared__ double sh[8][3][128];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long o0 = (long long)blockIdx.x * 128 + lane * 4;
     const long long r0 = (long long)blockIdx.y * kFcRowBlock, r1 = min(rows, r0 + (long long)kFcRowBlock);
-    const double sw = (double)w_step[o];
-    const long long zw = w_zp[o], cwo = cw[o];
-    const double b = bias ? (double)D::one(bias[o]) : 0.0;
-    const double bq = bias_q ? (double)bias_q[o] : b;           // no corrected bias: the layer keeps its own
-    double sd = 0.0, sd2 = 0.0, sy2 = 0.0;
-    for (long long n = r0; n < r1; ++n) {
-        const long long zx = act_zp[n];
-        long long dot = S[n * C_out + o];
-        if (S2) dot += S2[n * C_out + o];
-        const long long acc = dot - zx * cwo - zw * (long long)rx[n] + K * zx * zw;
-        const double yq = (double)act_step[n] * sw * (double)acc + bq;
-        const double y = (double)Y[n * C_out + o] + b;
-        const double d = yq - y;
-        sd += d;
-        sd2 += d * d;
-        sy2 += y * y;
+    double sw[4], zw[4], cwd[4], bq[4], b[4];
+    double sd[4] = {0, 0, 0, 0}, sd2[4] = {0, 0, 0, 0}, sy2[4] = {0, 0, 0, 0};
+    const bool live = o0 < C_out;                    // C_out is a multiple of 8: a lane's four channels are all in or all out
+    if (live) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            sw[c] = (double)w_step[o0 + c];
+            zw[c] = (double)w_zp[o0 + c];
+            cwd[c] = (double)cw[o0 + c];
+            b[c] = bias ? (double)D::one(bias[o0 + c]) : 0.0;
+            bq[c] = bias_q ? (double)bias_q[o0 + c] : b[c];      // no corrected bias: the layer keeps its own
+        }
+#pragma unroll 4
+        for (long long n = r0 + warp; n < r1; n += 8) {
+            const int4 s4 = __ldg(reinterpret_cast<const int4 *>(S + n * C_out + o0));
+            int4 t4 = make_int4(0, 0, 0, 0);
+            if (S2) t4 = __ldg(reinterpret_cast<const int4 *>(S2 + n * C_out + o0));
+            const float4 y4 = __ldg(reinterpret_cast<const float4 *>(Y + n * C_out + o0));
+            const double zx = (double)act_zp[n];
+            const double u = (double)K * zx - (double)rx[n];
+            const double sx = (double)act_step[n];
+            const int sv[4] = {s4.x, s4.y, s4.z, s4.w}, tv[4] = {t4.x, t4.y, t4.z, t4.w};
+            const float yv[4] = {y4.x, y4.y, y4.z, y4.w};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const double acc = ((double)sv[c] + (double)tv[c]) - zx * cwd[c] + zw[c] * u;
+                const double yq = sx * sw[c] * acc + bq[c];
+                const double y = (double)yv[c] + b[c];
+                const double d = yq - y;
+                sd[c] += d;
+                sd2[c] += d * d;
+                sy2[c] += y * y;
+            }
+        }
     }
-    double *out = partial + ((block0 + blockIdx.y) * C_out + o) * 3;
-    out[0] = sd;
-    out[1] = sd2;
-    out[2] = sy2;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        sh[warp][0][lane * 4 + c] = sd[c];
+        sh[warp][1][lane * 4 + c] = sd2[c];
+        sh[warp][2][lane * 4 + c] = sy2[c];
+    }
+    __syncthreads();
+    // 384 (quantity, channel) sums, 256 threads
+    for (int i = threadIdx.x; i < 384; i += 256) {
+        const int q = i / 128, c = i % 128;
+        const long long o = (long long)blockIdx.x * 128 + c;
+        if (o >= C_out) continue;
+        double a = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) a += sh[w][q][c];
+        double *out = partial + ((long long)blockIdx.y * C_out + o) * 3 + q;
+        *out = accumulate ? *out + a : a;
+    }
 }
 
 __global__ void __launch_bounds__(256)
@@ -195,15 +233,16 @@ aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, co
         rc = (dt == AWEQ_F16 ? fc_gemm_f16 : fc_gemm_bf16)(Xc, W, Y, (int)rows, (int)C_out, (int)C_in, C_in, scratch,
                                                            kFcScratch, stream);
         if (rc != AWEQ_OK) return rc;
-        const dim3 grid((unsigned)((C_out + 255) / 256), (unsigned)((rows + kFcRowBlock - 1) / kFcRowBlock));
+        // the grid always spans a full chunk's row blocks so that a short last chunk adds zeros, not garbage
+        const dim3 grid((unsigned)((C_out + 127) / 128), (unsigned)L.blocks_per_chunk);
         if (dt == AWEQ_F16)
             AWEQ_LAUNCH(fc_compare_kernel<F16>, grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
                         (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
-                        w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, c * L.blocks_per_chunk);
+                        w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, (int)(c > 0));
         else
             AWEQ_LAUNCH(fc_compare_kernel<BF16>, grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
                         (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
-                        w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, c * L.blocks_per_chunk);
+                        w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, (int)(c > 0));
     }
     double *cs = reinterpret_cast<double *>(Y);        // Y is free now: two doubles per output channel
     AWEQ_LAUNCH(fc_finish_kernel, dim3((unsigned)((C_out + 255) / 256)), dim3(256), 0, stream, (const double *)partial,
