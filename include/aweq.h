@@ -267,6 +267,19 @@ size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args);
 aweq_status aweq_layer_pass(const aweq_layer_args *args, void *ws, size_t ws_bytes,
                             aweq_dev_status *st, void *stream);
 
+/* ---- Folding diag(s)^-1 into the producer of a layer input (Section 3.1, text after Eq. 3:
+ * the division by s is fused into the previous block) -------------------------------------
+ *     out[r, c] = round16( float(P[r, c]) * rinv[r] )     r < rows, c < cols
+ * (binary32 product, one round-to-nearest-even to the 16-bit type).  P is a 16-bit row-major
+ * matrix with pitch ld elements: the weight matrix of the linear layer whose output channel
+ * r is input channel r of the calibrated layer (rows = C_in of that layer), or, with
+ * cols = 1, a bias vector or a normalisation layer's gain / shift.  rinv[rows] is step 3's
+ * 1/s.  out (pitch ld_out) may be P itself (in place) but must not otherwise overlap it.
+ * Any cols >= 1; 16-byte vector accesses are used when cols, ld, ld_out are multiples of 8
+ * and both pointers are 16-byte aligned.  Device pointers; enqueued on `stream`. */
+aweq_status aweq_fold_scale(const void *P, aweq_dtype dt, long long rows, long long cols, long long ld,
+                            const float *rinv, void *out, long long ld_out, void *stream);
+
 /* ---- Forward check of a calibrated W8A8 layer (Eq. 11; the quantity ablated in the AWE / BC
  * table) ------------------------------------------------------------------------------------
  * Compares, on the calibration tokens, the quantised layer

@@ -594,3 +594,19 @@ void oracle_forward_check(const uint8_t *Xq, const float *act_step, const int32_
     sums[3] = (double)N * (double)C_out;
     free(sq);
 }
+
+/* ------------------------------------------------------------------ */
+/* Folding diag(s)^-1 into the producer of a layer input (Section 3.1, */
+/* after Eq. 3: X^ = X diag(s)^-1 is obtained by scaling what produces */
+/* X -- row j of the previous linear layer and element j of its bias,  */
+/* or the gain and shift of a normalisation layer -- by 1/s_j).        */
+/*   out[r,c] = round16( (binary32) P[r,c] * rinv[r] )                 */
+/* ------------------------------------------------------------------ */
+void oracle_fold_scale(const uint16_t *P, int dtype, int64_t rows, int64_t cols, const float *rinv, uint16_t *out)
+{
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t c = 0; c < cols; ++c) {
+            volatile float prod = decode16(P[r * cols + c], dtype) * rinv[r];
+            out[r * cols + c] = encode16((double)prod, dtype);
+        }
+}

@@ -240,3 +240,13 @@ def forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, dtype, b
                                  _p(_f32(bias_q)), _p(X), _p(W), ci(dtype), _p(bias), i64(N), i64(C_in), i64(C_out),
                                  _p(mean_err), _p(sums))
     return mean_err, sums
+
+
+def fold_scale(P, dtype, rinv):
+    """Row r of the 16-bit matrix (or element r of the vector) P times rinv[r], as raw 16-bit bits."""
+    P = _u16(P)
+    rows = P.shape[0]
+    cols = 1 if P.ndim == 1 else P.shape[1]
+    out = np.empty_like(P)
+    _load().oracle_fold_scale(_p(P), ci(dtype), i64(rows), i64(cols), _p(_f32(rinv)), _p(out))
+    return out

@@ -73,6 +73,8 @@ _lib.aweq_quant_act.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _i, _i, _vp, _vp, _
 _lib.aweq_layer_pass_workspace_bytes.restype = _sz
 _lib.aweq_layer_pass_workspace_bytes.argtypes = [ctypes.POINTER(LayerArgs)]
 _lib.aweq_layer_pass.argtypes = [ctypes.POINTER(LayerArgs), _vp, _sz, _vp, _vp]
+_lib.aweq_fold_scale.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _ll, _vp]
+_lib.aweq_fold_scale.restype = _i
 _lib.aweq_forward_check_workspace_bytes.restype = _sz
 _lib.aweq_forward_check_workspace_bytes.argtypes = [_ll, _ll, _ll]
 _lib.aweq_forward_check.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _ll, _ll, _ll, _vp, _vp, _vp,
@@ -197,6 +199,18 @@ def aweq_bias_correct(epsmu, W, s, codes, step, zp, mu_hat, bits, gran, group, b
 def aweq_quant_act(X, rinv, bits, gran, tensor_lo_hi, Xq, step, zp, st=None):
     _check(_lib.aweq_quant_act(_ptr(X), dtype_tag(X), X.shape[0], X.shape[1], _ld(X), _ptr(rinv), bits, gran,
                                _ptr(tensor_lo_hi), _ptr(Xq), _ptr(step), _ptr(zp), _ptr(st), _stream()))
+
+
+def aweq_fold_scale(P, rinv, out=None):
+    """Scale row r of a 16-bit matrix (or element r of a vector) by ``rinv[r]``; in place when
+    ``out`` is None."""
+    out = P if out is None else out
+    if P.dim() == 1:
+        rows, cols, ld, ld_out = P.shape[0], 1, P.stride(0), out.stride(0)
+    else:
+        rows, cols, ld, ld_out = P.shape[0], P.shape[1], _ld(P), _ld(out)
+    _check(_lib.aweq_fold_scale(_ptr(P), dtype_tag(P), rows, cols, ld, _ptr(rinv), _ptr(out), ld_out, _stream()))
+    return out
 
 
 def forward_check_workspace_bytes(N: int, C_in: int, C_out: int) -> int:

@@ -118,6 +118,63 @@ class LayerCalibrator:
         return res
 
 
+class DecoderWalk:
+    """Calibration of one decoder layer in the order that folding diag(s)^-1 into the
+    producers requires (Section 3.1: the division by s is fused into the previous block).
+
+    An input produced by a linear layer (``o_in`` by ``v``, ``down_in`` by ``up``, ``fc2_in`` by
+    ``fc1``) changes that layer's weights: its factors are computed first (steps 1-3 on the
+    input and its consumers), rows of the producer's weight and bias are scaled by 1/s with
+    ``aweq_fold_scale``, and only then is every input calibrated with ``aweq_layer_pass`` -- the
+    producer is quantised with the fold already in it.  Inputs produced by a normalisation
+    layer get the fold in the gain and shift.  ``W`` and ``bias`` are copied; ``artifacts()``
+    returns everything a quantised layer needs.  Buffer management and call order only."""
+
+    def __init__(self, wl: synth.Workload, bits: int, X, W, bias=None, norms=None, flags: int = 0):
+        self.wl, self.bits, self.X = wl, bits, X
+        self.W = {k: v.clone() for k, v in W.items()}
+        self.bias = None if bias is None else {k: v.clone() for k, v in bias.items()}
+        self.norms = {} if norms is None else {k: tuple(None if t is None else t.clone() for t in v)
+                                               for k, v in norms.items()}
+        self.producers = synth.producers(wl)
+        self.cal = LayerCalibrator(wl, bits, X, self.W, self.bias, flags)
+        self.folded = []
+
+    def run(self) -> None:
+        wl, cal = self.wl, self.cal
+        # 1. inputs whose producer is a linear layer of this workload: factors, then fold
+        for inp in wl.inputs:
+            kind, prod = self.producers[inp.name]
+            if kind != "linear":
+                continue
+            o = cal.out[inp.name]
+            aweq.aweq_stats(self.X[inp.name], o["xmin"], o["xmax"], o["xmean"], ws=cal.ws, st=cal.status)
+            for i, l in enumerate(l for l in wl.linears if l.input == inp.name):
+                aweq.aweq_wrange(self.W[l.name], o["wmin"], o["wmax"], accumulate=i > 0, ws=cal.ws, st=cal.status)
+            aweq.aweq_factors(o["xmin"], o["xmax"], o["xmean"], o["wmin"], o["wmax"], o["s"], o["rinv"], o["mu_hat"],
+                              st=cal.status)
+            aweq.aweq_fold_scale(self.W[prod], o["rinv"])
+            if self.bias is not None and self.bias.get(prod) is not None:
+                aweq.aweq_fold_scale(self.bias[prod], o["rinv"])
+            self.folded.append((inp.name, "linear", prod))
+        # 2. every input with the folded producers in place
+        cal.run()
+        # 3. normalisation layers take the fold in their gain and shift
+        for inp in wl.inputs:
+            kind, prod = self.producers[inp.name]
+            if kind == "norm" and prod in self.norms:
+                for t in self.norms[prod]:
+                    if t is not None:
+                        aweq.aweq_fold_scale(t, cal.out[inp.name]["rinv"])
+                self.folded.append((inp.name, "norm", prod))
+
+    def artifacts(self) -> dict:
+        """{linear: codes, step, zp, bias}, {input: s, rinv, act_step, act_zp ...}, folded norms."""
+        return {"linears": {l.name: self.cal.out[l.name] for l in self.wl.linears},
+                "inputs": {i.name: self.cal.out[i.name] for i in self.wl.inputs if i.name in self.cal.out},
+                "norms": self.norms, "folded": list(self.folded)}
+
+
 def allreduce_stats(xmin: torch.Tensor, xmax: torch.Tensor, xsum: torch.Tensor, count: torch.Tensor, group=None) -> None:
     """The one exchange of a token-sharded calibration pass: per-channel minima, maxima,
     binary64 sums and the token count of all ranks are merged in place (min / max / sum /

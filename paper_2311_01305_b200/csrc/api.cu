@@ -345,6 +345,19 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     return AWEQ_OK;
 }
 
+// ------------------------------------------------------------------ folding 1/s into the producer
+aweq_status aweq_fold_scale(const void *P, aweq_dtype dt, long long rows, long long cols, long long ld,
+                            const float *rinv, void *out, long long ld_out, void *stream)
+{
+    if (!P || !rinv || !out) return AWEQ_ERR_NULL;
+    if (dt != AWEQ_F16 && dt != AWEQ_BF16) return AWEQ_ERR_DTYPE;
+    if (rows <= 0 || cols <= 0 || rows > (1ll << 40) || cols > (1ll << 30)) return AWEQ_ERR_SHAPE;
+    if (ld < cols || ld_out < cols) return AWEQ_ERR_ALIGN;
+    if (!aligned(P, 2) || !aligned(out, 2) || !aligned(rinv, 4)) return AWEQ_ERR_ALIGN;
+    AWEQ_LOGF("aweq_fold_scale rows=%lld cols=%lld bytes=%lld\n", rows, cols, 4 * rows * cols + 4 * rows);
+    return run_fold_scale(P, dt, rows, cols, ld, rinv, out, ld_out, (cudaStream_t)stream);
+}
+
 // ------------------------------------------------------------------ forward check
 size_t aweq_forward_check_workspace_bytes(long long N, long long C_in, long long C_out)
 {

@@ -36,6 +36,9 @@ aweq_status run_bias_gemv(const void *W, aweq_dtype dt, long long C_out, long lo
                           const float *mu_hat, int bits, int gran, int group, const void *bias_in, void *bias_out,
                           float *bias_out_f32, aweq_dtype bias_dt, cudaStream_t stream);
 
+aweq_status run_fold_scale(const void *P, aweq_dtype dt, long long rows, long long cols, long long ld,
+                           const float *rinv, void *out, long long ld_out, cudaStream_t stream);
+
 // forward check (tensor-core GEMMs + comparison)
 size_t forward_check_ws_bytes(long long N, long long C_in, long long C_out);
 aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, const int *act_zp,

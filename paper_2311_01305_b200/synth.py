@@ -123,6 +123,33 @@ def workloads(n_tokens_scale: float = 1.0) -> dict:
     return w
 
 
+def producers(wl: Workload) -> dict:
+    """What produces each layer input of a decoder-shaped workload: {input name: (kind, name)}
+    with kind "norm" (a normalisation layer's output: its gain and shift take 1/s) or
+    "linear" (channel j of the input is a positive multiple of output channel j of that
+    linear layer: the value projection seen through the attention weights, ``up`` through the
+    gate, ``fc1`` through ReLU).  Structure only; the folding itself is the library's."""
+    table = {"attn_in": ("norm", "ln_attn"), "o_in": ("linear", "v"), "mlp_in": ("norm", "ln_mlp"),
+             "down_in": ("linear", "up"), "fc1_in": ("norm", "ln_mlp"), "fc2_in": ("linear", "fc1"),
+             "x": ("norm", "ln")}
+    names = {l.name for l in wl.linears}
+    out = {}
+    for i in wl.inputs:
+        kind, name = table[i.name]
+        if kind == "linear" and name not in names:
+            kind, name = "none", ""            # the producer is not part of this workload
+        out[i.name] = (kind, name)
+    return out
+
+
+def make_norm(c: int, dtype: str, seed: int, device="cpu", shift: bool = True):
+    """Gain (around 1) and shift (around 0) of a normalisation layer, 16-bit."""
+    g = _generator(seed, "cpu")
+    gain = (1.0 + 0.1 * torch.randn(c, generator=g)).to(torch_dtype(dtype)).to(device)
+    beta = (0.05 * torch.randn(c, generator=g)).to(torch_dtype(dtype)).to(device) if shift else None
+    return gain, beta
+
+
 def torch_dtype(name: str) -> torch.dtype:
     return {"f16": torch.float16, "bf16": torch.bfloat16}[name]
 

@@ -542,3 +542,75 @@ def test_forward_check_sees_what_bias_correction_removes():
     assert np.abs(fixed).max() <= 1e-6 * scale + 2.0 ** -24 * np.abs(bf).max()
     assert np.abs(raw).max() > 1000 * np.abs(fixed).max()
     assert sums[3] == N * C_out and sums[2] == pytest.approx((fixed ** 2).sum(), rel=1e-12)
+
+
+# ---------------------------------------------------------------- folding 1/s into the producer (after Eq. 3)
+def test_fold_scale_against_library_casts_and_exact_cases():
+    rng = np.random.default_rng(41)
+    P = rng.standard_normal((9, 13)) * 3
+    rinv = np.exp(rng.standard_normal(9)).astype(np.float32)
+    # fp16: NumPy's float32 -> float16 cast rounds to nearest even
+    Pb = f16_bits(P)
+    got = orc.fold_scale(Pb, orc.F16, rinv)
+    ref = (Pb.view(np.float16).astype(np.float32) * rinv[:, None]).astype(np.float16).view(np.uint16)
+    assert np.array_equal(got, ref)
+    # bf16: PyTorch's cast
+    Pb = bf16_bits(P)
+    got = orc.fold_scale(Pb, orc.BF16, rinv)
+    prod = torch.from_numpy(bits_to_f64(Pb, orc.BF16).astype(np.float32) * rinv[:, None])
+    assert np.array_equal(got, prod.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+    # powers of two are exact; a vector is a one-column matrix
+    v = f16_bits([1.5, -3.0, 0.125, 7.0])
+    out = orc.fold_scale(v, orc.F16, np.array([2.0, 0.5, 4.0, 0.25], np.float32))
+    assert bits_to_f64(out, orc.F16).tolist() == [3.0, -1.5, 0.5, 1.75]
+    # the scale belongs to the ROW (a transposed fold fails here)
+    M = f16_bits([[1, 2], [3, 4]])
+    out = orc.fold_scale(M, orc.F16, np.array([2.0, 0.5], np.float32))
+    assert bits_to_f64(out, orc.F16).tolist() == [[2.0, 4.0], [1.5, 2.0]]
+
+
+def test_folds_leave_a_decoder_block_unchanged():
+    """Eq. 3 through the producers: scaling the gain / shift of a normalisation layer, the value
+    projection (seen through the attention weights), ``up`` (seen through the gate) and ``fc1``
+    (seen through ReLU) by 1/s gives exactly the equalised input X diag(s)^-1 of the next layer,
+    up to the 16-bit rounding of the folded parameters."""
+    rng = np.random.default_rng(42)
+    T, h, f = 24, 16, 40
+    x = rng.standard_normal((T, h))
+    s = np.exp(rng.standard_normal(h) * 0.5).astype(np.float32)
+    sf = np.exp(rng.standard_normal(f) * 0.5).astype(np.float32)
+    rinv, rinvf = (1.0 / s).astype(np.float32), (1.0 / sf).astype(np.float32)
+    dec = lambda b: bits_to_f64(b, orc.F16)
+    fold = lambda a, r: dec(orc.fold_scale(f16_bits(a), orc.F16, r))
+    q16 = lambda a: dec(f16_bits(a))
+    tol = 2.0 ** -10                                           # one 16-bit rounding of each folded parameter
+
+    # normalisation layer: (x - mean) / std * gain + shift
+    gain, shift = q16(1 + 0.1 * rng.standard_normal(h)), q16(0.1 * rng.standard_normal(h))
+    z = (x - x.mean(axis=1, keepdims=True)) / x.std(axis=1, keepdims=True)
+    ln = z * gain + shift
+    ln_f = z * fold(gain, rinv) + fold(shift, rinv)
+    assert np.allclose(ln_f, ln * rinv, rtol=0, atol=tol * (np.abs(z) * np.abs(gain) + np.abs(shift)).max() * rinv.max())
+
+    # value projection through softmax attention: o_in = A (x Wv^T + bv)
+    Wv, bv = q16(rng.standard_normal((h, h)) * 0.2), q16(rng.standard_normal(h) * 0.1)
+    A = np.exp(rng.standard_normal((T, T)))
+    A /= A.sum(axis=1, keepdims=True)
+    o_in = A @ (x @ Wv.T + bv)
+    o_in_f = A @ (x @ fold(Wv, rinv).T + fold(bv, rinv))
+    scale = (np.abs(A) @ (np.abs(x) @ np.abs(Wv).T + np.abs(bv))) * rinv
+    assert np.all(np.abs(o_in_f - o_in * rinv) <= tol * scale)
+
+    # gated MLP: down_in = silu(x Wg^T) * (x Wu^T)
+    Wg, Wu = q16(rng.standard_normal((f, h)) * 0.2), q16(rng.standard_normal((f, h)) * 0.2)
+    g = x @ Wg.T
+    act = g / (1 + np.exp(-g))
+    down_in = act * (x @ Wu.T)
+    down_in_f = act * (x @ fold(Wu, rinvf).T)
+    assert np.all(np.abs(down_in_f - down_in * rinvf) <= tol * np.abs(act) * (np.abs(x) @ np.abs(Wu).T) * rinvf)
+
+    # ReLU MLP: fc2_in = relu(x W1^T + b1); needs s > 0
+    W1, b1 = q16(rng.standard_normal((f, h)) * 0.2), q16(rng.standard_normal(f) * 0.1)
+    fc2_in = np.maximum(x @ W1.T + b1, 0)
+    fc2_in_f = np.maximum(x @ fold(W1, rinvf).T + fold(b1, rinvf), 0)
+    assert np.all(np.abs(fc2_in_f - fc2_in * rinvf) <= tol * (np.abs(x) @ np.abs(W1).T + np.abs(b1)) * rinvf)
