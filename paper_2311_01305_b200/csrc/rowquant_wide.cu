@@ -5,8 +5,10 @@
 // and, worse, a second read of the per-channel factors from L1 / L2 (a 36864-channel factor
 // vector is 147 KB: larger than what L1 keeps beside the staging buffers).  Here the whole
 // CTA (512 or 1024 threads) works on a tile of R rows at a time; a thread owns the same V <= 5
-// column vectors in every row, so their factors stay in registers for the whole kernel, and
-// the rows are read twice from shared memory instead of being kept in registers:
+// column vectors in every row, so their factors stay on chip for the whole kernel (in
+// registers; with 1024 threads, where a thread has 64 registers, those of the fourth and
+// fifth vector sit in shared memory), and the rows are read twice from shared memory instead
+// of being kept in registers:
 //   pass 1  x^ = x * (1/s), running min / max of each of the R rows     (no global loads)
 //   reduce  warp redux -> shared -> warp r finishes row r: Step, 1/Step, Z (Eq. 2)
 //   pass 2  x^ again, codes (Eq. 1), 8-byte coalesced stores
@@ -27,12 +29,18 @@ struct RwSmem {
 };
 static_assert(sizeof(RwSmem) <= kRwHeader, "header");
 
+// vectors per thread whose factors live in registers; the rest (1024-thread shape only) in shared memory
+__host__ __device__ constexpr int rw_reg_vectors(int V, int NT) { return NT == 1024 && V > 3 ? 3 : V; }
+__host__ __device__ constexpr size_t rw_scale_smem(int V, int NT) { return (size_t)(V - rw_reg_vectors(V, NT)) * NT * 32; }
+
 template <class D, int V, int NT>
 __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     RwSmem *sm = reinterpret_cast<RwSmem *>(smem_raw);
-    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw + kRwHeader);
+    constexpr int VR = rw_reg_vectors(V, NT);
+    float4 *ssc = reinterpret_cast<float4 *>(smem_raw + kRwHeader);       // [(v - VR) * 2 + half][thread]
+    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw + kRwHeader + rw_scale_smem(V, NT));
     constexpr int NW = NT / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int R = p.rows_per_stage, S = p.stages;
@@ -57,18 +65,33 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
             rq_issue_tile(p, &sm->ring, stage_base, next_issue, S, R, stage_vecs, lane);
 
     // the factors of this thread's columns (no equalisation = ones, which is exact)
-    float2 sc[V][4];
+    float2 sc[VR][4];
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         const int idx = threadIdx.x + v * NT;
+        float4 s0 = make_float4(1.0f, 1.0f, 1.0f, 1.0f), s1 = s0;
         if (p.scale && idx < p.nvec) {
-            const float4 s0 = ldg_f4(p.scale + (size_t)idx * 8), s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
+            s0 = ldg_f4(p.scale + (size_t)idx * 8);
+            s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
+        }
+        if (v < VR) {
             sc[v][0] = make_float2(s0.x, s0.y); sc[v][1] = make_float2(s0.z, s0.w);
             sc[v][2] = make_float2(s1.x, s1.y); sc[v][3] = make_float2(s1.z, s1.w);
-        } else {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) sc[v][k] = make_float2(1.0f, 1.0f);
+        } else {                                   // only this thread reads these back
+            ssc[((v - VR) * 2 + 0) * NT + threadIdx.x] = s0;
+            ssc[((v - VR) * 2 + 1) * NT + threadIdx.x] = s1;
         }
+    }
+#define AWEQ_RW_SCALES(v, f)                                                           \
+    float2 f[4];                                                                       \
+    if (v < VR) {                                                                      \
+        f[0] = sc[v < VR ? v : 0][0]; f[1] = sc[v < VR ? v : 0][1];                    \
+        f[2] = sc[v < VR ? v : 0][2]; f[3] = sc[v < VR ? v : 0][3];                    \
+    } else {                                                                           \
+        const float4 a = ssc[((v - VR) * 2 + 0) * NT + threadIdx.x];                   \
+        const float4 b = ssc[((v - VR) * 2 + 1) * NT + threadIdx.x];                   \
+        f[0] = make_float2(a.x, a.y); f[1] = make_float2(a.z, a.w);                    \
+        f[2] = make_float2(b.x, b.y); f[3] = make_float2(b.z, b.w);                    \
     }
 
     bool ok = true;
@@ -104,9 +127,10 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
                         if (v < V - 1 || idx < p.nvec) {
                             const uint4 raw = rowp[idx];
                             const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+                            AWEQ_RW_SCALES(v, f)
 #pragma unroll
                             for (int c = 0; c < 4; ++c) {
-                                const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w[c])), sc[v][c]);
+                                const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w[c])), f[c]);
                                 lo[r] = fminf(fminf(lo[r], x.x), x.y);
                                 hi[r] = fmaxf(fmaxf(hi[r], x.x), x.y);
                             }
@@ -158,10 +182,11 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
                         const uint4 raw = rowp[idx];
                         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
                         uint32_t u[8];
+                        AWEQ_RW_SCALES(v, f)
                         if (lean) {
 #pragma unroll
                             for (int c = 0; c < 4; ++c) {
-                                const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w[c])), sc[v][c]);
+                                const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w[c])), f[c]);
                                 const float2 t = __fmul2_rn(x, inv2);
                                 // t * 1 + magic as one FMA: equal to t + magic, and it cannot be
                                 // contracted with the multiply above (which would change ties)
@@ -173,7 +198,7 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
                         } else {
 #pragma unroll
                             for (int c = 0; c < 4; ++c) {
-                                const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w[c])), sc[v][c]);
+                                const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w[c])), f[c]);
                                 u[2 * c] = (uint32_t)code_generic(x.x, inv, zp, qmax);
                                 u[2 * c + 1] = (uint32_t)code_generic(x.y, inv, zp, qmax);
                             }
@@ -186,6 +211,7 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm->ring.empty[s]);
     }
+#undef AWEQ_RW_SCALES
     if (!ok && threadIdx.x == 0) {
         if (p.st) atomicAdd(&p.st->wait_timeout, 1ull);
         // copies that were already requested may still land in this CTA's shared memory
@@ -204,7 +230,8 @@ bool plan_rowquant_wide(long long nrows, long long cols, RowQuantPlan *out)
     p.team = p.NT;
     p.V = (nvec + p.NT - 1) / p.NT;
     const size_t row_bytes = (size_t)nvec * 16;
-    const size_t budget = 226 * 1024 - kRwHeader;
+    const size_t scale_smem = rw_scale_smem(p.V, p.NT);
+    const size_t budget = 226 * 1024 - kRwHeader - scale_smem;
     int S = 2;
     int R = (int)(budget / (2 * row_bytes));
     if (R > kRwMaxR) R = kRwMaxR;
@@ -219,7 +246,7 @@ bool plan_rowquant_wide(long long nrows, long long cols, RowQuantPlan *out)
     if ((long long)R > nrows) R = (int)nrows;
     p.rows_per_stage = R;
     p.stages = S;
-    p.smem = kRwHeader + (size_t)S * R * row_bytes;
+    p.smem = kRwHeader + scale_smem + (size_t)S * R * row_bytes;
     p.ntiles = (nrows + R - 1) / R;
     long long g = kSmCount;
     if (g > p.ntiles) g = p.ntiles;
