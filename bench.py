@@ -336,7 +336,7 @@ def main():
     if wl.act_quant:
         act_ms = [sum(ea[0].elapsed_time(ea[1]) for _, ea in hooks[k]) for k in range(args.steps)]
         act_bytes = sum(3 * i.n_tokens * i.c_in + 8 * i.n_tokens for i in wl.inputs)
-        dom = {"kernel": "rowquant_kernel (aweq_quant_act)", "bytes": act_bytes, "ms": statistics.mean(act_ms),
+        dom = {"kernel": "rowquant_kernel / rowquant_wide_kernel (aweq_quant_act)", "bytes": act_bytes, "ms": statistics.mean(act_ms),
                "launches_per_step": len(cal.passes), "stats_gbs": stats_bytes / statistics.mean(stats_ms) / 1e6}
     peak, peak_kind = measured_peaks()
     achieved = dom["bytes"] / dom["ms"] / 1e6
