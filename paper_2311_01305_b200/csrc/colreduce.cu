@@ -47,15 +47,42 @@ constexpr int kColTargetCtas = kColCtasPerSm * kSmCount;
 
 struct ColPlan {
     int nvec, nslab, slab_w, nsplit;
+    int phases;          // thread groups that share a slab's columns and split a stage's rows
+    int stage_rows;      // rows per stage
     long long rows_per_split;
 };
+
+// Slab width and row phases.  With the widest slabs (ceil(nvec / 256) of them) a slab of w
+// vectors keeps only w of the 256 consumer threads busy; when w <= 128 the idle threads take
+// a second (fourth, eighth) share of every stage's rows and write partials of their own, and
+// narrower slabs of at least 128 vectors are taken when that fills the CTA better.
+static void pick_slabs(int nvec, int *nslab_out, int *slab_w_out, int *phases_out)
+{
+    const int base = (nvec + kColThreads - 1) / kColThreads;
+    double best = -1.0;
+    for (int nslab = base; nslab <= 4 * base; ++nslab) {
+        const int w = (nvec + nslab - 1) / nslab;
+        if (nslab > base && w < 128) break;
+        const int wpad = (w + 31) / 32 * 32;
+        int ph = 1;
+        while (ph < 8 && 2 * ph * wpad <= kColThreads) ph *= 2;
+        int nsplit = kColTargetCtas / nslab;
+        if (nsplit < 1) nsplit = 1;
+        const double lanes = (double)w * ph / kColThreads;                       // busy consumer threads
+        const double sms = (double)(nslab * nsplit) / kColTargetCtas;            // busy SMs
+        const double pad = (double)nvec / ((double)nslab * w);                   // columns that exist
+        double util = lanes * (sms > 1.0 ? 1.0 : sms) * pad;
+        if (nslab > base) util -= 0.10;                                          // only for a clear gain
+        if (util > best) { best = util; *nslab_out = nslab; *slab_w_out = w; *phases_out = ph; }
+    }
+}
 
 ColPlan plan_colreduce(long long rows, long long cols)
 {
     ColPlan p;
     p.nvec = (int)(cols / 8);
-    p.nslab = (p.nvec + kColThreads - 1) / kColThreads;
-    p.slab_w = (p.nvec + p.nslab - 1) / p.nslab;
+    pick_slabs(p.nvec, &p.nslab, &p.slab_w, &p.phases);
+    p.stage_rows = p.phases == 1 ? kColRows : (p.phases <= 4 ? 32 : 64);
     int nsplit = kColTargetCtas / p.nslab;
     if (nsplit < 1) nsplit = 1;
     long long max_split = (rows + 7) / 8;
@@ -72,15 +99,16 @@ ColPlan plan_colreduce(long long rows, long long cols)
 
 size_t colreduce_ws_bytes(long long rows, long long cols)
 {
-    // pmin, pmax: float[nsplit][cols]; psum: double[nsplit][cols].  Sized for the
+    // pmin, pmax: float[nsplit * phases][cols]; psum: double[nsplit * phases][cols].  Sized for the
     // largest number of row splits any row count can get, so that a buffer sized
     // for N rows also serves every call with fewer rows (streamed chunks).
     (void)rows;
     const int nvec = (int)(cols / 8);
-    const int nslab = (nvec + kColThreads - 1) / kColThreads;
-    int max_split = kColTargetCtas / (nslab > 0 ? nslab : 1);
+    int nslab = 1, slab_w = 1, phases = 1;
+    pick_slabs(nvec > 0 ? nvec : 1, &nslab, &slab_w, &phases);
+    int max_split = kColTargetCtas / nslab;
     if (max_split < 1) max_split = 1;
-    return (size_t)max_split * (size_t)cols * 16 + 256;
+    return (size_t)max_split * phases * (size_t)cols * 16 + 256;
 }
 
 constexpr int kFlushRows = 8;           // rows summed in binary32 before the error-free fold
@@ -138,8 +166,8 @@ struct ColSmem {
 template <class D, bool WITH_SUM>
 __global__ void __launch_bounds__(kColThreads + 32, kColCtasPerSm)
 colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, int nvec, int nslab, int slab_w,
-                 long long rows_per_split, long long cols, float *__restrict__ pmin, float *__restrict__ pmax,
-                 double *__restrict__ psum, aweq_dev_status *st)
+                 int phases, int stage_rows, long long rows_per_split, long long cols, float *__restrict__ pmin,
+                 float *__restrict__ pmax, double *__restrict__ psum, aweq_dev_status *st)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     ColSmem *sm = reinterpret_cast<ColSmem *>(smem_raw);
@@ -151,10 +179,13 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
     const int w = min(slab_w, nvec - v0);                 // vectors in this slab (> 0)
     const long long r0 = (long long)split * rows_per_split;
     const long long r1 = min(nrows, r0 + rows_per_split);
-    const int ntiles = r1 > r0 ? (int)((r1 - r0 + kColRows - 1) / kColRows) : 0;
+    const int ntiles = r1 > r0 ? (int)((r1 - r0 + stage_rows - 1) / stage_rows) : 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int active_warps = (w + 31) / 32;
-    const size_t stage_vecs = (size_t)kColRows * slab_w;
+    // phase p of the consumer threads takes rows [p, p + 1) * stage_rows / phases of every stage;
+    // a phase is a whole number of warps
+    const int wpad = (slab_w + 31) / 32 * 32;
+    const int active_warps = phases * wpad / 32;
+    const size_t stage_vecs = (size_t)stage_rows * slab_w;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kColStages; ++s) {
@@ -179,16 +210,17 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
             }
-            const long long row0 = r0 + (long long)t * kColRows;
-            const int rows = (int)min((long long)kColRows, r1 - row0);
+            const long long row0 = r0 + (long long)t * stage_rows;
+            const int rows = (int)min((long long)stage_rows, r1 - row0);
             uint4 *dst = stage_base + (size_t)s * stage_vecs;
             if (lane == 0) mbar_arrive_expect_tx(&sm->full[s], (uint32_t)rows * w * 16u);
             __syncwarp();
             if (contiguous) {
                 if (lane == 0) bulk_g2s(dst, X + row0 * ld, (uint32_t)rows * w * 16u, &sm->full[s]);
-            } else if (lane < rows) {
-                bulk_g2s(dst + (size_t)lane * w, X + (row0 + lane) * ld + (long long)v0 * 8, (uint32_t)w * 16u,
-                         &sm->full[s]);
+            } else {
+                for (int r = lane; r < rows; r += 32)
+                    bulk_g2s(dst + (size_t)r * w, X + (row0 + r) * ld + (long long)v0 * 8, (uint32_t)w * 16u,
+                             &sm->full[s]);
             }
         }
         if (!ok && lane == 0) {
@@ -197,8 +229,10 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
         }
     } else if (warp < active_warps) {
         // ---------------- consumer warps: thread <-> one vector column
-        const int t_col = threadIdx.x;
+        const int phase = threadIdx.x / wpad;
+        const int t_col = threadIdx.x - phase * wpad;
         const bool mine = t_col < w;
+        const int rows_per_phase = stage_rows / phases;          // a multiple of kFlushRows
         typename D::T2 mn[4], mx[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -214,13 +248,14 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
             const uint32_t use = t / kColStages;
             ok = mbar_wait(&sm->full[s], use & 1);
             if (!ok || *reinterpret_cast<volatile int *>(&sm->abort_flag)) { ok = false; break; }
-            const long long row0 = r0 + (long long)t * kColRows;
-            const int rows = (int)min((long long)kColRows, r1 - row0);
+            const long long row0 = r0 + (long long)t * stage_rows;
+            const int rows_in_stage = (int)min((long long)stage_rows, r1 - row0);
+            const int rows = min(rows_in_stage, (phase + 1) * rows_per_phase);      // end of my share
             const uint4 *src = stage_base + (size_t)s * stage_vecs + t_col;
             if (mine) {
                 // groups of kFlushRows rows: binary32 partial sums, then an error-free
                 // addition into the (hi, lo) running sum
-                for (int rb = 0; rb < rows; rb += kFlushRows) {
+                for (int rb = phase * rows_per_phase; rb < rows; rb += kFlushRows) {
                     float acc32[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) acc32[k] = 0.0f;
@@ -249,7 +284,7 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
             if (st) atomicAdd(&st->wait_timeout, 1ull);
         }
         if (mine) {
-            const size_t o = (size_t)split * (size_t)cols + (size_t)(v0 + t_col) * 8;
+            const size_t o = ((size_t)split * phases + phase) * (size_t)cols + (size_t)(v0 + t_col) * 8;
             float lo[8], hi[8];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -345,9 +380,9 @@ __global__ void bump_count_kernel(long long *count, long long nrows, int accumul
     count[0] = (accumulate ? count[0] : 0) + nrows;
 }
 
-static size_t colreduce_smem_bytes(int slab_w)
+static size_t colreduce_smem_bytes(int slab_w, int stage_rows)
 {
-    return 128 + (size_t)kColStages * kColRows * slab_w * 16;
+    return 128 + (size_t)kColStages * stage_rows * slab_w * 16;
 }
 
 template <class D, bool WITH_SUM>
@@ -358,18 +393,19 @@ static aweq_status launch_colreduce(const void *X, long long rows, long long col
     ColPlan p = plan_colreduce(rows, cols);
     char *base = reinterpret_cast<char *>(ws);
     float *pmin = reinterpret_cast<float *>(base);
-    float *pmax = pmin + (size_t)p.nsplit * cols;
-    double *psum = reinterpret_cast<double *>(base + (size_t)p.nsplit * cols * 8);
-    const size_t smem = colreduce_smem_bytes(p.slab_w);
+    const size_t nparts = (size_t)p.nsplit * p.phases;
+    float *pmax = pmin + nparts * cols;
+    double *psum = reinterpret_cast<double *>(base + nparts * cols * 8);
+    const size_t smem = colreduce_smem_bytes(p.slab_w, p.stage_rows);
     auto kern = colreduce_kernel<D, WITH_SUM>;
     // set on every launch: the attribute belongs to the current device, which may change between calls
     AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)colreduce_smem_bytes(kColThreads)));
-    int nsplit_eff = rows > 0 ? p.nsplit : 0;
+                                      (int)colreduce_smem_bytes(kColThreads, kColRows)));
+    int nsplit_eff = rows > 0 ? (int)nparts : 0;
     if (rows > 0) {
         AWEQ_LAUNCH(kern, dim3(p.nslab * p.nsplit), dim3(kColThreads + 32), smem, stream,
-                    reinterpret_cast<const uint16_t *>(X), rows, ld, p.nvec, p.nslab, p.slab_w, p.rows_per_split, cols,
-                    pmin, pmax, psum, st);
+                    reinterpret_cast<const uint16_t *>(X), rows, ld, p.nvec, p.nslab, p.slab_w, p.phases, p.stage_rows,
+                    p.rows_per_split, cols, pmin, pmax, psum, st);
     }
     AWEQ_LAUNCH(colreduce_finalize_kernel<WITH_SUM>, dim3((unsigned)((cols + kFinCols - 1) / kFinCols)),
                 dim3(kFinCols * kFinLanes), 0, stream, (const float *)pmin, (const float *)pmax, (const double *)psum,
