@@ -44,6 +44,7 @@ constexpr int kColRows = AWEQ_COL_ROWS;         // rows per stage
 constexpr int kColStages = AWEQ_COL_STAGES;
 constexpr int kColCtasPerSm = AWEQ_COL_CTAS_PER_SM;
 constexpr int kColTargetCtas = kColCtasPerSm * kSmCount;
+constexpr int kFlushRowsHost = 8;               // rows summed in binary32 before the error-free fold
 
 struct ColPlan {
     int nvec, nslab, slab_w, nsplit;
@@ -52,37 +53,33 @@ struct ColPlan {
     long long rows_per_split;
 };
 
-// Slab width and row phases.  With the widest slabs (ceil(nvec / 256) of them) a slab of w
-// vectors keeps only w of the 256 consumer threads busy; when w <= 128 the idle threads take
-// a second (fourth, eighth) share of every stage's rows and write partials of their own, and
-// narrower slabs of at least 128 vectors are taken when that fills the CTA better.
-static void pick_slabs(int nvec, int *nslab_out, int *slab_w_out, int *phases_out)
+// Row phases and stage height.  A slab of w vectors keeps only w of the 256 consumer threads
+// busy; when w <= 128 the idle threads take a second (fourth, eighth) share of every stage's
+// rows and write partials of their own.  A stage holds as many rows as fit 96 KB (24 rows of a
+// full slab): narrow matrices get taller stages, so that one bulk copy still moves ~96 KB.
+// (Narrower slabs with more phases were tried instead of idle threads and were slower.)
+static void pick_slabs(int nvec, int *nslab_out, int *slab_w_out, int *phases_out, int *stage_rows_out)
 {
-    const int base = (nvec + kColThreads - 1) / kColThreads;
-    double best = -1.0;
-    for (int nslab = base; nslab <= 4 * base; ++nslab) {
-        const int w = (nvec + nslab - 1) / nslab;
-        if (nslab > base && w < 128) break;
-        const int wpad = (w + 31) / 32 * 32;
-        int ph = 1;
-        while (ph < 8 && 2 * ph * wpad <= kColThreads) ph *= 2;
-        int nsplit = kColTargetCtas / nslab;
-        if (nsplit < 1) nsplit = 1;
-        const double lanes = (double)w * ph / kColThreads;                       // busy consumer threads
-        const double sms = (double)(nslab * nsplit) / kColTargetCtas;            // busy SMs
-        const double pad = (double)nvec / ((double)nslab * w);                   // columns that exist
-        double util = lanes * (sms > 1.0 ? 1.0 : sms) * pad;
-        if (nslab > base) util -= 0.10;                                          // only for a clear gain
-        if (util > best) { best = util; *nslab_out = nslab; *slab_w_out = w; *phases_out = ph; }
-    }
+    const int nslab = (nvec + kColThreads - 1) / kColThreads;
+    const int w = (nvec + nslab - 1) / nslab;
+    const int wpad = (w + 31) / 32 * 32;
+    int ph = 1;
+    while (ph < 8 && 2 * ph * wpad <= kColThreads) ph *= 2;
+    const int unit = kFlushRowsHost * ph;                      // every phase gets whole eight-row groups
+    int rows = (int)((size_t)kColRows * kColThreads / w) / unit * unit;
+    if (rows < unit) rows = unit;
+    if (rows > 256) rows = 256 / unit * unit;
+    *nslab_out = nslab;
+    *slab_w_out = w;
+    *phases_out = ph;
+    *stage_rows_out = rows;
 }
 
 ColPlan plan_colreduce(long long rows, long long cols)
 {
     ColPlan p;
     p.nvec = (int)(cols / 8);
-    pick_slabs(p.nvec, &p.nslab, &p.slab_w, &p.phases);
-    p.stage_rows = p.phases == 1 ? kColRows : (p.phases <= 4 ? 32 : 64);
+    pick_slabs(p.nvec, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
     int nsplit = kColTargetCtas / p.nslab;
     if (nsplit < 1) nsplit = 1;
     long long max_split = (rows + 7) / 8;
@@ -104,14 +101,14 @@ size_t colreduce_ws_bytes(long long rows, long long cols)
     // for N rows also serves every call with fewer rows (streamed chunks).
     (void)rows;
     const int nvec = (int)(cols / 8);
-    int nslab = 1, slab_w = 1, phases = 1;
-    pick_slabs(nvec > 0 ? nvec : 1, &nslab, &slab_w, &phases);
+    int nslab = 1, slab_w = 1, phases = 1, stage_rows = 8;
+    pick_slabs(nvec > 0 ? nvec : 1, &nslab, &slab_w, &phases, &stage_rows);
     int max_split = kColTargetCtas / nslab;
     if (max_split < 1) max_split = 1;
     return (size_t)max_split * phases * (size_t)cols * 16 + 256;
 }
 
-constexpr int kFlushRows = 8;           // rows summed in binary32 before the error-free fold
+constexpr int kFlushRows = kFlushRowsHost;
 static_assert(kColRows % kFlushRows == 0, "stage rows must be a multiple of the flush period");
 
 // acc += widen(16-bit value): one mixed-precision add per element (exact widening,
