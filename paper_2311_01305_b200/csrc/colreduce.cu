@@ -54,21 +54,24 @@ struct ColPlan {
 };
 
 // Row phases and stage height.  A slab of w vectors keeps only w of the 256 consumer threads
-// busy; when w <= 128 the idle threads take a second (fourth, eighth) share of every stage's
-// rows and write partials of their own.  A stage holds as many rows as fit 96 KB (24 rows of a
-// full slab): narrow matrices get taller stages, so that one bulk copy still moves ~96 KB.
+// busy; when w <= 128 the idle threads take a second share of every stage's rows and write
+// partials of their own (more than two phases multiply the partials the finalize kernel has
+// to walk and were slower).  A stage holds as many rows as fit 96 KB (24 rows of a full slab):
+// narrow matrices get taller stages, so that one bulk copy still moves ~96 KB -- but a split
+// keeps at least a dozen stages, or filling and draining the two-stage ring shows.
 // (Narrower slabs with more phases were tried instead of idle threads and were slower.)
-static void pick_slabs(int nvec, int *nslab_out, int *slab_w_out, int *phases_out, int *stage_rows_out)
+static void pick_slabs(int nvec, long long rows_per_split, int *nslab_out, int *slab_w_out, int *phases_out,
+                       int *stage_rows_out)
 {
     const int nslab = (nvec + kColThreads - 1) / kColThreads;
     const int w = (nvec + nslab - 1) / nslab;
     const int wpad = (w + 31) / 32 * 32;
-    int ph = 1;
-    while (ph < 8 && 2 * ph * wpad <= kColThreads) ph *= 2;
+    const int ph = 2 * wpad <= kColThreads ? 2 : 1;
     const int unit = kFlushRowsHost * ph;                      // every phase gets whole eight-row groups
     int rows = (int)((size_t)kColRows * kColThreads / w) / unit * unit;
-    if (rows < unit) rows = unit;
     if (rows > 256) rows = 256 / unit * unit;
+    if (rows_per_split > 0 && rows > rows_per_split / 12) rows = (int)(rows_per_split / 12) / unit * unit;
+    if (rows < unit) rows = unit;
     *nslab_out = nslab;
     *slab_w_out = w;
     *phases_out = ph;
@@ -79,7 +82,7 @@ ColPlan plan_colreduce(long long rows, long long cols)
 {
     ColPlan p;
     p.nvec = (int)(cols / 8);
-    pick_slabs(p.nvec, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
+    pick_slabs(p.nvec, 0, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
     int nsplit = kColTargetCtas / p.nslab;
     if (nsplit < 1) nsplit = 1;
     long long max_split = (rows + 7) / 8;
@@ -89,6 +92,7 @@ ColPlan plan_colreduce(long long rows, long long cols)
     rps = (rps + 7) / 8 * 8;            // whole eight-row groups; the last stage of a split may be partial
     if (rps < 8) rps = 8;
     p.rows_per_split = rps;
+    pick_slabs(p.nvec, rps, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
     p.nsplit = (int)((rows + rps - 1) / rps);
     if (p.nsplit < 1) p.nsplit = 1;
     return p;
@@ -102,7 +106,7 @@ size_t colreduce_ws_bytes(long long rows, long long cols)
     (void)rows;
     const int nvec = (int)(cols / 8);
     int nslab = 1, slab_w = 1, phases = 1, stage_rows = 8;
-    pick_slabs(nvec > 0 ? nvec : 1, &nslab, &slab_w, &phases, &stage_rows);
+    pick_slabs(nvec > 0 ? nvec : 1, 0, &nslab, &slab_w, &phases, &stage_rows);
     int max_split = kColTargetCtas / nslab;
     if (max_split < 1) max_split = 1;
     return (size_t)max_split * phases * (size_t)cols * 16 + 256;
