@@ -54,7 +54,7 @@ struct ColPlan {
 };
 
 // Row phases and stage height.  A slab of w vectors keeps only w of the 256 consumer threads
-// busy; when w <= 128 the idle threads take a second share of every stage's rows and write
+// busy; when w <= 96 the idle threads take a second share of every stage's rows and write
 // partials of their own (more than two phases multiply the partials the finalize kernel has
 // to walk and were slower).  A stage holds as many rows as fit 96 KB (24 rows of a full slab):
 // narrow matrices get taller stages, so that one bulk copy still moves ~96 KB -- but a split
@@ -66,9 +66,9 @@ static void pick_slabs(int nvec, long long rows_per_split, int *nslab_out, int *
     const int nslab = (nvec + kColThreads - 1) / kColThreads;
     const int w = (nvec + nslab - 1) / nslab;
     const int wpad = (w + 31) / 32 * 32;
-    const int ph = 2 * wpad <= kColThreads ? 2 : 1;
+    const int ph = wpad <= 96 ? 2 : 1;                         // from four warps per slab on, phases gained nothing
     const int unit = kFlushRowsHost * ph;                      // every phase gets whole eight-row groups
-    int rows = (int)((size_t)kColRows * kColThreads / w) / unit * unit;
+    int rows = ph == 1 ? kColRows : (int)((size_t)kColRows * kColThreads / w) / unit * unit;
     if (rows > 256) rows = 256 / unit * unit;
     if (rows_per_split > 0 && rows > rows_per_split / 12) rows = (int)(rows_per_split / 12) / unit * unit;
     if (rows < unit) rows = unit;
