@@ -119,31 +119,40 @@ __global__ void __launch_bounds__(NT, 1) rowquant_tile_kernel(const RowQuantPara
         const int rows = (int)min((long long)R, p.nrows - row0);
         const uint4 *tile = stage_base + (size_t)s * stage_vecs;
 
-        // ---- pass 1: extremes of my group's rows (scaled).  The row loop is kept rolled (two rows
-        // per trip): unrolled over a whole tile the kernel outgrows the instruction cache.
+        // ---- pass 1: extremes of my group's rows (scaled)
+        float lo[RPG], hi[RPG];
+#pragma unroll
+        for (int i = 0; i < RPG; ++i) { lo[i] = INFINITY; hi[i] = -INFINITY; }
         if (ok) {
-#pragma unroll (NT == 1024 ? 1 : 2)
-            for (int r = g; r < rows; r += G) {
-                const uint4 *rowp = tile + (size_t)r * p.nvec;
-                float lo = INFINITY, hi = -INFINITY;
 #pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    const int idx = col + v * W;
-                    if (v < V - 1 || idx < p.nvec) {
-                        const uint4 raw = rowp[idx];
-                        const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-                        AWEQ_RT_SCALES(v, f)
+            for (int i = 0; i < RPG; ++i) {
+                const int r = g + i * G;
+                if (r < rows) {
+                    const uint4 *rowp = tile + (size_t)r * p.nvec;
 #pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w4[c])), f[c]);
-                            lo = fminf(fminf(lo, x.x), x.y);
-                            hi = fmaxf(fmaxf(hi, x.x), x.y);
+                    for (int v = 0; v < V; ++v) {
+                        const int idx = col + v * W;
+                        if (v < V - 1 || idx < p.nvec) {
+                            const uint4 raw = rowp[idx];
+                            const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+                            AWEQ_RT_SCALES(v, f)
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w4[c])), f[c]);
+                                lo[i] = fminf(fminf(lo[i], x.x), x.y);
+                                hi[i] = fmaxf(fmaxf(hi[i], x.x), x.y);
+                            }
                         }
                     }
                 }
-                lo = redux_min(lo, 0xffffffffu);
-                hi = redux_max(hi, 0xffffffffu);
-                if (lane == 0) sm->red[r * wpg + wig] = make_float2(lo, hi);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < RPG; ++i) {
+            const int r = g + i * G;
+            if (r < rows) {
+                const float l = redux_min(lo[i], 0xffffffffu), h = redux_max(hi[i], 0xffffffffu);
+                if (lane == 0) sm->red[r * wpg + wig] = make_float2(l, h);
             }
         }
         // the barrier doubles as the agreement on a timed-out wait: everybody leaves or nobody
@@ -167,9 +176,10 @@ __global__ void __launch_bounds__(NT, 1) rowquant_tile_kernel(const RowQuantPara
         __syncthreads();
 
         // ---- pass 2: codes
-#pragma unroll (NT == 1024 ? 1 : 2)
-        for (int r = g; r < rows; r += G) {
-            {
+#pragma unroll
+        for (int i = 0; i < RPG; ++i) {
+            const int r = g + i * G;
+            if (r < rows) {
                 const float4 qv = sm->q[r];
                 const float inv = qv.y;
                 const int zp = __float_as_int(qv.z), fl = __float_as_int(qv.w);
