@@ -75,7 +75,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
                          cudaStream_t stream)
 {
     RowQuantPlan pl;
-    const bool wide = !weights && plan_rowquant_tile(nrows, cols, &pl);
+    const bool wide = !weights && plan_rowquant_wide(nrows, cols, &pl);
     if (!wide && !plan_rowquant(nrows, cols, &pl)) return AWEQ_ERR_SHAPE;
     RowQuantParams p;
     p.X = reinterpret_cast<const uint16_t *>(X);
@@ -85,7 +85,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     p.step = step; p.zp = zp; p.epsmu = epsmu; p.bits = bits; p.bias = bias;
     p.team = pl.team; p.rows_per_stage = pl.rows_per_stage; p.stages = pl.stages; p.ntiles = pl.ntiles;
     p.st = st;
-    if (wide) return run_rowquant_tile(p, pl, dt, stream);
+    if (wide) return run_rowquant_wide(p, pl, dt, stream);
     const int mode = !weights ? 0 : ((mu && epsmu) ? 1 : 2);
     return dt == AWEQ_F16 ? rq_launch_f16(p, pl, mode, stream) : rq_launch_bf16(p, pl, mode, stream);
 }

@@ -62,8 +62,8 @@ struct RowQuantPlan {
 };
 
 bool plan_rowquant(long long nrows, long long cols, RowQuantPlan *out);
-// tile form of step 6 (rowquant_tile.cu): cols <= 40960
-bool plan_rowquant_tile(long long nrows, long long cols, RowQuantPlan *out);
+// wide rows of step 6 (rowquant_wide.cu): a plan exists for 10240 < cols <= 40960
+bool plan_rowquant_wide(long long nrows, long long cols, RowQuantPlan *out);
 
 struct RqSmem {
     uint64_t full[kRqStagesMax];
@@ -435,7 +435,7 @@ static aweq_status rq_launch(const RowQuantParams &p, const RowQuantPlan &pl, in
     return rq_launch_v<D, false, false>(p, pl, stream);
 }
 
-aweq_status run_rowquant_tile(const RowQuantParams &p, const RowQuantPlan &pl, aweq_dtype dt, cudaStream_t stream);
+aweq_status run_rowquant_wide(const RowQuantParams &p, const RowQuantPlan &pl, aweq_dtype dt, cudaStream_t stream);
 aweq_status rq_launch_f16(const RowQuantParams &p, const RowQuantPlan &pl, int mode, cudaStream_t stream);
 aweq_status rq_launch_bf16(const RowQuantParams &p, const RowQuantPlan &pl, int mode, cudaStream_t stream);
 
