@@ -318,10 +318,10 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
 }
 
 // Reduce the per-split partials in a fixed order; merge with the running state
-// when accumulating.  A block handles 32 columns with 8 threads each: thread
-// (c, k) folds splits k, k+8, ... and the eight partial results of a column are
-// then combined in order of k, so the result does not depend on timing.
-constexpr int kFinCols = 32, kFinLanes = 8;
+// when accumulating.  A block handles 32 columns with 32 threads each: thread
+// (c, k) folds partials k, k+32, ... and the 32 results of a column are then
+// combined in order of k, so the result does not depend on timing.
+constexpr int kFinCols = 32, kFinLanes = 32;
 
 template <bool WITH_SUM>
 __global__ void __launch_bounds__(kFinCols * kFinLanes)
