@@ -248,7 +248,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-tokens", type=int, default=131072)
+    ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
     ap.add_argument("--op", default="layer_pass", choices=["layer_pass", "forward_check"],
                     help="forward_check: time the W8A8 forward check of the calibrated layer instead (1 GPU)")
     args = ap.parse_args()
