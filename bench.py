@@ -340,13 +340,13 @@ def main():
                "launches_per_step": len(cal.passes), "stats_gbs": stats_bytes / statistics.mean(stats_ms) / 1e6}
     peak, peak_kind = measured_peaks()
     achieved = dom["bytes"] / dom["ms"] / 1e6
-    # DRAM traffic per launch from the ncu capture summarised in
-    # profiles/stats_and_groupquant_llama7b_small.md (1/8 of the rows: reads 1.00011 x the
-    # algorithmic bytes and scale with the rows; the per-split partials, 4.4 MB, do not).
-    # Only the statistics kernel has a capture that covers its whole output.
+    # DRAM traffic per launch from the ncu counters summarised in
+    # profiles/stats_and_groupquant_llama7b_small.md (current kernel, 1/8 of the rows: reads are
+    # 1.0001 x the algorithmic bytes and scale with the rows; the per-split partials, at most
+    # 4.4 MB, do not).  Only the statistics kernel has counters that cover its whole output.
     traffic = None
     if not wl.act_quant:
-        traffic = (dom["bytes"] / dom["launches_per_step"]) * 1.00011 + 4.42e6
+        traffic = (dom["bytes"] / dom["launches_per_step"]) * 1.0001 + 4.4e6
     roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
                 "launch_ms": dom["ms"] / dom["launches_per_step"],
