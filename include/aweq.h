@@ -96,6 +96,16 @@ const char *aweq_last_cuda_error(void);          /* text of the last CUDA error 
 int aweq_version(void);
 /* Number of kernels this library has launched in this process (diagnostic). */
 unsigned long long aweq_launch_count(void);
+/* Launch geometry the library would use for an operation on a rows x cols matrix (host logic
+ * only, no CUDA call; for diagnostics and tests).  op is AWEQ_OP_STATS / AWEQ_OP_WRANGE (the
+ * column reduction), AWEQ_OP_EQUALIZE_QUANTIZE (row-wise weights) or AWEQ_OP_QUANT_ACT (per
+ * token).  plan[8] receives
+ *   column reduction: {CTAs, threads, shared bytes, column slabs, slab width in 16-byte vectors,
+ *                      row splits, row phases, rows per stage}
+ *   row quantisers:   {CTAs, threads, shared bytes, threads per row, vectors per thread,
+ *                      rows per stage, stages, 1 if the wide-row kernel is used}
+ * Returns AWEQ_ERR_SHAPE when the shape is not supported, AWEQ_ERR_UNSUPPORTED for other ops. */
+aweq_status aweq_plan_query(int op, long long rows, long long cols, long long plan[8]);
 
 /* Scratch bytes an operation needs for the given shape: rows x cols is
  * N x C_in for AWEQ_OP_STATS / AWEQ_OP_QUANT_ACT and C_out x C_in for the

@@ -73,6 +73,8 @@ _lib.aweq_quant_act.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _i, _i, _vp, _vp, _
 _lib.aweq_layer_pass_workspace_bytes.restype = _sz
 _lib.aweq_layer_pass_workspace_bytes.argtypes = [ctypes.POINTER(LayerArgs)]
 _lib.aweq_layer_pass.argtypes = [ctypes.POINTER(LayerArgs), _vp, _sz, _vp, _vp]
+_lib.aweq_plan_query.argtypes = [_i, _ll, _ll, ctypes.POINTER(_ll * 8)]
+_lib.aweq_plan_query.restype = _i
 _lib.aweq_fold_scale.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _ll, _vp]
 _lib.aweq_fold_scale.restype = _i
 _lib.aweq_forward_check_workspace_bytes.restype = _sz
@@ -199,6 +201,14 @@ def aweq_bias_correct(epsmu, W, s, codes, step, zp, mu_hat, bits, gran, group, b
 def aweq_quant_act(X, rinv, bits, gran, tensor_lo_hi, Xq, step, zp, st=None):
     _check(_lib.aweq_quant_act(_ptr(X), dtype_tag(X), X.shape[0], X.shape[1], _ld(X), _ptr(rinv), bits, gran,
                                _ptr(tensor_lo_hi), _ptr(Xq), _ptr(step), _ptr(zp), _ptr(st), _stream()))
+
+
+def aweq_plan_query(op: int, rows: int, cols: int):
+    """Launch geometry for an operation on a rows x cols matrix as a tuple of 8 integers
+    (see ``include/aweq.h``); host logic only."""
+    plan = (_ll * 8)()
+    _check(_lib.aweq_plan_query(op, rows, cols, ctypes.byref(plan)))
+    return tuple(plan)
 
 
 def aweq_fold_scale(P, rinv, out=None):

@@ -101,6 +101,19 @@ const char *aweq_last_cuda_error(void) { return g_cuda_error; }
 int aweq_version(void) { return 100; }
 unsigned long long aweq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+aweq_status aweq_plan_query(int op, long long rows, long long cols, long long plan[8])
+{
+    if (!plan) return AWEQ_ERR_NULL;
+    if (rows <= 0 || cols <= 0 || cols % 8 || cols > (1ll << 30)) return AWEQ_ERR_SHAPE;
+    if (op == AWEQ_OP_STATS || op == AWEQ_OP_WRANGE) {
+        colreduce_describe(rows, cols, plan);
+        return AWEQ_OK;
+    }
+    if (op == AWEQ_OP_EQUALIZE_QUANTIZE || op == AWEQ_OP_QUANT_ACT)
+        return rowquant_describe(rows, cols, op == AWEQ_OP_EQUALIZE_QUANTIZE, plan) ? AWEQ_OK : AWEQ_ERR_SHAPE;
+    return AWEQ_ERR_UNSUPPORTED;
+}
+
 size_t aweq_workspace_bytes(int op, long long rows, long long cols, int bits, int gran, int group)
 {
     (void)bits; (void)group;

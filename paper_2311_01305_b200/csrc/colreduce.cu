@@ -417,6 +417,19 @@ static aweq_status launch_colreduce(const void *X, long long rows, long long col
     return AWEQ_OK;
 }
 
+void colreduce_describe(long long rows, long long cols, long long plan[8])
+{
+    const ColPlan p = plan_colreduce(rows, cols);
+    plan[0] = (long long)p.nslab * p.nsplit;
+    plan[1] = kColThreads + 32;
+    plan[2] = (long long)colreduce_smem_bytes(p.slab_w, p.stage_rows);
+    plan[3] = p.nslab;
+    plan[4] = p.slab_w;
+    plan[5] = p.nsplit;
+    plan[6] = p.phases;
+    plan[7] = p.stage_rows;
+}
+
 aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin, float *xmax,
                       float *xmean, double *xsum, long long *count, int accumulate, void *ws, aweq_dev_status *st,
                       cudaStream_t stream)

@@ -9,6 +9,8 @@
 namespace aweq {
 
 size_t colreduce_ws_bytes(long long rows, long long cols);
+void colreduce_describe(long long rows, long long cols, long long plan[8]);
+bool rowquant_describe(long long rows, long long cols, bool weights, long long plan[8]);
 
 aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin, float *xmax,
                       float *xmean, double *xsum, long long *count, int accumulate, void *ws, aweq_dev_status *st,

@@ -68,6 +68,16 @@ bool rowquant_supported(long long nrows, long long cols)
     return plan_rowquant(nrows, cols, &pl);
 }
 
+bool rowquant_describe(long long rows, long long cols, bool weights, long long plan[8])
+{
+    RowQuantPlan pl;
+    const bool wide = !weights && plan_rowquant_wide(rows, cols, &pl);
+    if (!wide && !plan_rowquant(rows, cols, &pl)) return false;
+    plan[0] = pl.grid; plan[1] = pl.NT; plan[2] = (long long)pl.smem; plan[3] = pl.team; plan[4] = pl.V;
+    plan[5] = pl.rows_per_stage; plan[6] = pl.stages; plan[7] = wide ? 1 : 0;
+    return true;
+}
+
 // weights == true: packed bit stream + optional eps.mu sums; false: one byte per code
 aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
                          const float *scale, const float *mu, int bits, bool weights, unsigned char *out,

@@ -79,3 +79,55 @@ def test_binding_imports_and_names_match_header():
                     "aweq_workspace_bytes", "aweq_layer_pass_workspace_bytes", "aweq_forward_check_workspace_bytes"):
             continue
         assert hasattr(aweq, name), name
+
+
+# ---------------------------------------------------------------- launch planners (host logic)
+SMEM_LIMIT = 227 * 1024           # opt-in shared memory per CTA on sm_100
+WIDTHS = sorted(set(list(range(8, 2049, 8)) + list(range(2048, 40961, 248)) +
+                    [768, 3072, 4096, 5120, 9216, 10240, 10248, 11008, 13824, 20480, 20488, 36864, 40960]))
+
+
+def _plan(lib, op, rows, cols):
+    arr = (ctypes.c_longlong * 8)()
+    lib.aweq_plan_query.argtypes = [ctypes.c_int, ctypes.c_longlong, ctypes.c_longlong, ctypes.POINTER(ctypes.c_longlong * 8)]
+    rc = lib.aweq_plan_query(op, rows, cols, ctypes.byref(arr))
+    return rc, tuple(arr)
+
+
+def test_column_reduction_plans_fit_the_hardware(lib):
+    lib.aweq_workspace_bytes.restype = ctypes.c_size_t
+    lib.aweq_workspace_bytes.argtypes = [ctypes.c_int] + [ctypes.c_longlong] * 2 + [ctypes.c_int] * 3
+    for cols in WIDTHS:
+        for rows in (1, 7, 100, 4096, 262144):
+            rc, (ctas, threads, smem, nslab, slab_w, nsplit, phases, stage_rows) = _plan(lib, 1, rows, cols)
+            assert rc == 0
+            nvec = cols // 8
+            assert 1 <= ctas <= 148 and ctas == nslab * nsplit and threads == 288
+            assert smem <= SMEM_LIMIT and smem == 128 + 2 * stage_rows * slab_w * 16
+            assert nslab * slab_w >= nvec and slab_w <= 256                 # every column has an owner
+            assert phases in (1, 2) and stage_rows % (8 * phases) == 0      # whole eight-row groups per phase
+            assert phases * ((slab_w + 31) // 32 * 32) <= 256               # phases fit the consumer threads
+            assert stage_rows * slab_w * 16 <= (1 << 20) - 1                # one mbarrier transaction count
+            # the partials of the largest split count fit the advertised workspace
+            assert nsplit * phases * cols * 16 + 256 <= lib.aweq_workspace_bytes(1, rows, cols, 0, 0, 0)
+
+
+def test_row_quantiser_plans_fit_the_hardware(lib):
+    for op in (4, 6):
+        for cols in WIDTHS:
+            for rows in (1, 5, 300, 65536):
+                rc, (ctas, threads, smem, team, V, R, S, wide) = _plan(lib, op, rows, cols)
+                assert rc == 0, (op, rows, cols)
+                nvec = cols // 8
+                assert 1 <= ctas <= 296 and threads in (256, 512, 1024) and smem <= SMEM_LIMIT
+                assert team % 32 == 0 and threads % team == 0 and team * V >= nvec      # the row is covered
+                assert S >= 2 and R >= 1
+                if wide:
+                    assert op == 6 and cols > 10240 and V <= 5 and team == threads and R <= 4
+                    assert smem >= 4096 + S * R * nvec * 16
+                else:
+                    assert V <= 10 and smem == 512 + S * R * nvec * 16
+                    assert R % (threads // team) == 0 or R >= rows              # whole rounds of teams per stage
+    # beyond the supported width the query says so instead of planning something that cannot launch
+    assert _plan(lib, 6, 100, 40968)[0] == 2 and _plan(lib, 4, 100, 81920)[0] == 2
+    assert _plan(lib, 6, 100, 36)[0] == 2 and _plan(lib, 5, 100, 64)[0] == 9
