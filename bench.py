@@ -199,7 +199,8 @@ def run_forward_check(args, wl, bits):
     pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(pk):
         p16, kind = float(json.load(open(pk))["bf16_tflops_sustained"]), "measured (sustained)"
-    peak = p16 * 2.0 / 1.5
+    w8a8 = wl.act_quant and bits == 8 and wl.w_gran == "row"
+    peak = p16 * 2.0 / 1.5 if w8a8 else p16           # weight-only: both contractions are 16-bit
     tf = flops / ms / 1e9
     worst = {n: float((me.abs().max() / (s4[1] / s4[3]).sqrt()).item()) for n, (me, s4) in res.items()}
     sqnr = {n: float(10.0 * torch.log10(s4[1] / s4[0]).item()) for n, (me, s4) in res.items()}
@@ -222,11 +223,13 @@ def run_forward_check(args, wl, bits):
     print(json.dumps({
         "metric": "aweq_forward_check_tflops", "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
         "warmup": max(1, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "u8 x u8 -> s32 and %s -> f32" % wl.dtype, "data": "synthetic",
+        "vs_baseline": None, "dtype": ("u8 x u8 -> s32 and %s -> f32" if w8a8 else "%s -> f32 (two contractions)") % wl.dtype,
+        "data": "synthetic",
         "config": {"workload": wl.name, "tokens": tokens, "linears": [l.name for l in wl.linears],
                    "cache": "operands (GBs) far larger than the 126 MB L2"},
         "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
-                     "peak_kind": "16-bit GEMM rate of %s x 4/3 for the 8-bit / 16-bit mix" % kind, "traffic": None},
+                     "peak_kind": ("16-bit GEMM rate of %s x 4/3 for the 8-bit / 16-bit mix" if w8a8
+                                   else "16-bit GEMM rate of %s") % kind, "traffic": None},
         "clocks": clocks, "gpu_launches": int(launches),
         "max_abs_mean_err_over_output_rms": worst, "output_sqnr_db": sqnr, "ablation": ablation}))
 

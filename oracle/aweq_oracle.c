@@ -610,3 +610,65 @@ void oracle_fold_scale(const uint16_t *P, int dtype, int64_t rows, int64_t cols,
             out[r * cols + c] = encode16((double)prod, dtype);
         }
 }
+
+/* ------------------------------------------------------------------ */
+/* Forward check of a weight-only layer: Eq. 11 evaluated on data with */
+/* 16-bit activations.  The equalised input is x^ = x * rinv (Eq. 3;   */
+/* rinv is the binary32 1/s of step 3, NULL = ones) and the weights    */
+/* are the de-quantised step-4 codes W~ = Step (q - Z) (Eq. 1-2), at   */
+/* any bit-width and granularity:                                      */
+/*   y~[n,o] = sum_j x^[n,j] W~[o,j] + bias_q[o]                       */
+/*   y[n,o]  = sum_j X[n,j] W[o,j] + bias[o]                           */
+/* Outputs as oracle_forward_check.  Everything in binary64.           */
+/* ------------------------------------------------------------------ */
+void oracle_forward_check_weights(const uint8_t *codes, const float *step, const int32_t *zp, int bits, int gran,
+                                  int64_t group, const float *rinv, const float *bias_q, const uint16_t *X,
+                                  const uint16_t *W, int dtype, const uint16_t *bias, int64_t N, int64_t C_in,
+                                  int64_t C_out, double *mean_err, double *sums)
+{
+    int64_t pitch = C_in * bits / 8;
+    int64_t glen = gran == ORACLE_PER_GROUP ? group : C_in;
+    int64_t ngroups = C_in / glen;
+    double *sq = (double *)calloc((size_t)C_out * 2, sizeof(double));
+#pragma omp parallel for schedule(static)
+    for (int64_t o = 0; o < C_out; ++o) {
+        double *wq = (double *)malloc((size_t)C_in * sizeof(double));
+        double *w = (double *)malloc((size_t)C_in * sizeof(double));
+        for (int64_t j = 0; j < C_in; ++j) {
+            int64_t k = gran == ORACLE_PER_TENSOR ? 0 : o * ngroups + j / glen;
+            int32_t q = get_code(codes + o * pitch, j, bits);
+            wq[j] = (double)step[k] * (double)((int64_t)q - (int64_t)zp[k]);
+            w[j] = (double)decode16(W[o * C_in + j], dtype);
+        }
+        double sd = 0.0, sd2 = 0.0, sy2 = 0.0;
+        for (int64_t n = 0; n < N; ++n) {
+            double yq = 0.0, y = 0.0;
+            for (int64_t j = 0; j < C_in; ++j) {
+                double x = (double)decode16(X[n * C_in + j], dtype);
+                double xh = rinv ? x * (double)rinv[j] : x;
+                yq += xh * wq[j];
+                y += x * w[j];
+            }
+            if (bias) y += (double)decode16(bias[o], dtype);
+            if (bias_q) yq += (double)bias_q[o];
+            else if (bias) yq += (double)decode16(bias[o], dtype);
+            double d = yq - y;
+            sd += d;
+            sd2 += d * d;
+            sy2 += y * y;
+        }
+        mean_err[o] = sd / (double)N;
+        sq[2 * o] = sd2;
+        sq[2 * o + 1] = sy2;
+        free(wq);
+        free(w);
+    }
+    sums[0] = sums[1] = sums[2] = 0.0;
+    for (int64_t o = 0; o < C_out; ++o) {
+        sums[0] += sq[2 * o];
+        sums[1] += sq[2 * o + 1];
+        sums[2] += mean_err[o] * mean_err[o];
+    }
+    sums[3] = (double)N * (double)C_out;
+    free(sq);
+}

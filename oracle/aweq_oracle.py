@@ -250,3 +250,20 @@ def fold_scale(P, dtype, rinv):
     out = np.empty_like(P)
     _load().oracle_fold_scale(_p(P), ci(dtype), i64(rows), i64(cols), _p(_f32(rinv)), _p(out))
     return out
+
+
+def forward_check_weights(codes, step, zp, bits, gran, group, rinv, bias_q, X, W, dtype, bias=None):
+    """Eq. 11 on data for a weight-only layer -> (mean_err[C_out] f64, sums[4] f64); packed codes as
+    ``equalize_quantize`` returns them, ``rinv`` binary32 or None."""
+    X, W = _u16(X), _u16(W)
+    N, C_in = X.shape
+    C_out = W.shape[0]
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    assert codes.shape == (C_out, C_in * bits // 8)
+    mean_err = np.empty(C_out, np.float64)
+    sums = np.empty(4, np.float64)
+    bias = None if bias is None else _u16(bias)
+    _load().oracle_forward_check_weights(_p(codes), _p(_f32(step)), _p(np.ascontiguousarray(zp, dtype=np.int32)),
+                                         ci(bits), ci(gran), i64(group), _p(_f32(rinv)), _p(_f32(bias_q)), _p(X), _p(W),
+                                         ci(dtype), _p(bias), i64(N), i64(C_in), i64(C_out), _p(mean_err), _p(sums))
+    return mean_err, sums

@@ -81,6 +81,11 @@ _lib.aweq_forward_check_workspace_bytes.restype = _sz
 _lib.aweq_forward_check_workspace_bytes.argtypes = [_ll, _ll, _ll]
 _lib.aweq_forward_check.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i, _vp, _ll, _ll, _ll, _vp, _vp, _vp,
                                     _sz, _vp]
+_lib.aweq_forward_check_weights_workspace_bytes.restype = _sz
+_lib.aweq_forward_check_weights_workspace_bytes.argtypes = [_ll, _ll, _ll]
+_lib.aweq_forward_check_weights.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _ll, _ll, _ll, _vp, _vp,
+                                            _vp, _sz, _vp]
+_lib.aweq_forward_check_weights.restype = _i
 for _f in ("aweq_stats", "aweq_wrange", "aweq_factors", "aweq_equalize_quantize", "aweq_bias_correct",
            "aweq_quant_act", "aweq_layer_pass", "aweq_forward_check"):
     getattr(_lib, _f).restype = _i
@@ -239,6 +244,24 @@ def aweq_forward_check(Xq, act_step, act_zp, Wq, w_step, w_zp, bias_q, X, W, bia
     _check(_lib.aweq_forward_check(_ptr(Xq), _ptr(act_step), _ptr(act_zp), _ptr(Wq), _ptr(w_step), _ptr(w_zp),
                                    _ptr(bias_q), _ptr(X), _ptr(W), dtype_tag(X), _ptr(bias), N, C_in, C_out,
                                    _ptr(mean_err), _ptr(sums), _ptr(ws), ws.numel(), _stream()))
+    return ws
+
+
+def forward_check_weights_workspace_bytes(N: int, C_in: int, C_out: int) -> int:
+    return int(_lib.aweq_forward_check_weights_workspace_bytes(N, C_in, C_out))
+
+
+def aweq_forward_check_weights(codes, step, zp, bits, gran, group, rinv, bias_q, X, W, bias, mean_err, sums, ws=None):
+    """Forward check of a weight-only layer (argument marshalling only; see ``include/aweq.h``)."""
+    N, C_in = X.shape
+    C_out = W.shape[0]
+    if not (X.is_contiguous() and W.is_contiguous() and codes.is_contiguous()):
+        raise ValueError("aweq_forward_check_weights takes contiguous matrices")
+    if ws is None:
+        ws = workspace(forward_check_weights_workspace_bytes(N, C_in, C_out), X.device)
+    _check(_lib.aweq_forward_check_weights(_ptr(codes), _ptr(step), _ptr(zp), bits, gran, group, _ptr(rinv), _ptr(bias_q),
+                                           _ptr(X), _ptr(W), dtype_tag(X), _ptr(bias), N, C_in, C_out, _ptr(mean_err),
+                                           _ptr(sums), _ptr(ws), ws.numel(), _stream()))
     return ws
 
 

@@ -87,6 +87,7 @@ class LayerCalibrator:
         self.ws = aweq.workspace(ws_bytes, dev)
         self.status = aweq.new_status(dev)
         self._fc_ws, self._fc_out = None, {}
+        self.equalized = not (flags & aweq.FLAG_NO_EQUALIZE)
 
     def run(self) -> None:
         """One calibration pass of the whole layer: one library call per input."""
@@ -94,14 +95,17 @@ class LayerCalibrator:
             lp(self.ws, self.status)
 
     def forward_check(self, X, W, bias=None, corrected: bool = True):
-        """``aweq_forward_check`` for every linear of a W8A8 workload after ``run()``:
-        {linear name: (mean_err[C_out], sums[4])} as binary64 device tensors.  ``corrected``
-        gives the quantised layer the step-5 bias; otherwise it keeps the original one."""
+        """The forward check of every linear after ``run()``: {linear name: (mean_err[C_out],
+        sums[4])} as binary64 device tensors.  W8A8 workloads with row-wise 8-bit weights go
+        through ``aweq_forward_check`` (integer GEMM on the codes of steps 4 and 6), everything
+        else through ``aweq_forward_check_weights`` (16-bit activations).  ``corrected`` gives the
+        quantised layer the step-5 bias; otherwise it keeps the original one."""
         wl = self.wl
-        if not (wl.act_quant and self.bits == 8 and wl.w_gran == "row"):
-            raise ValueError("the forward check covers W8A8 workloads with row-wise weight scales")
+        w8a8 = wl.act_quant and self.bits == 8 and wl.w_gran == "row"
+        gran = aweq.PER_ROW if wl.w_gran == "row" else aweq.PER_GROUP
         dev = self.ws.device
-        need = max(aweq.forward_check_workspace_bytes(X[l.input].shape[0], l.c_in, l.c_out) for l in wl.linears)
+        size = aweq.forward_check_workspace_bytes if w8a8 else aweq.forward_check_weights_workspace_bytes
+        need = max(size(X[l.input].shape[0], l.c_in, l.c_out) for l in wl.linears)
         if self._fc_ws is None or self._fc_ws.numel() < need:
             self._fc_ws = aweq.workspace(need, dev)
         res = {}
@@ -111,9 +115,15 @@ class LayerCalibrator:
                 self._fc_out[l.name] = (torch.empty(l.c_out, dtype=torch.float64, device=dev),
                                         torch.empty(4, dtype=torch.float64, device=dev))
             mean_err, sums = self._fc_out[l.name]
-            aweq.aweq_forward_check(o["Xq"], o["act_step"], o["act_zp"], lo["codes"], lo["step"], lo["zp"],
-                                    lo["bias_f32"] if corrected else None, X[l.input], W[l.name],
-                                    None if bias is None else bias.get(l.name), mean_err, sums, ws=self._fc_ws)
+            b = None if bias is None else bias.get(l.name)
+            bq = lo["bias_f32"] if corrected else None
+            if w8a8:
+                aweq.aweq_forward_check(o["Xq"], o["act_step"], o["act_zp"], lo["codes"], lo["step"], lo["zp"], bq,
+                                        X[l.input], W[l.name], b, mean_err, sums, ws=self._fc_ws)
+            else:
+                aweq.aweq_forward_check_weights(lo["codes"], lo["step"], lo["zp"], self.bits, gran, wl.group,
+                                                o["rinv"] if self.equalized else None, bq, X[l.input], W[l.name], b,
+                                                mean_err, sums, ws=self._fc_ws)
             res[l.name] = (mean_err, sums)
         return res
 

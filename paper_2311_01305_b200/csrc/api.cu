@@ -395,4 +395,30 @@ aweq_status aweq_forward_check(const unsigned char *Xq, const float *act_step, c
                              sums, ws, ws_bytes, (cudaStream_t)stream);
 }
 
+size_t aweq_forward_check_weights_workspace_bytes(long long N, long long C_in, long long C_out)
+{
+    if (N <= 0 || C_in <= 0 || C_out <= 0) return 0;
+    return forward_check_weights_ws_bytes(N, C_in, C_out);
+}
+
+aweq_status aweq_forward_check_weights(const unsigned char *codes, const float *step, const int *zp, int bits,
+                                       aweq_gran gran, int group, const float *rinv, const float *bias_q,
+                                       const void *X, const void *W, aweq_dtype dt, const void *bias, long long N,
+                                       long long C_in, long long C_out, double *mean_err, double *sums, void *ws,
+                                       size_t ws_bytes, void *stream)
+{
+    if (!codes || !step || !zp || !X || !W || !mean_err || !sums) return AWEQ_ERR_NULL;
+    if (dt != AWEQ_F16 && dt != AWEQ_BF16) return AWEQ_ERR_DTYPE;
+    if (N <= 0 || C_in <= 0 || C_out <= 0 || C_in % 16 || C_out % 8) return AWEQ_ERR_SHAPE;
+    if (C_in > (1ll << 30) || C_out > (1ll << 30) || N > (1ll << 34)) return AWEQ_ERR_SHAPE;
+    aweq_status rc = check_quant(bits, gran, group, C_in);
+    if (rc != AWEQ_OK) return rc;
+    if (!aligned(X, 16) || !aligned(W, 16) || (rinv && !aligned(rinv, 16))) return AWEQ_ERR_ALIGN;
+    if (!ws || !aligned(ws, 256) || ws_bytes < forward_check_weights_ws_bytes(N, C_in, C_out)) return AWEQ_ERR_WORKSPACE;
+    AWEQ_LOGF("aweq_forward_check_weights N=%lld C_in=%lld C_out=%lld bits=%d flops=%.3e\n", N, C_in, C_out, bits,
+              4.0 * N * C_in * C_out);
+    return run_forward_check_weights(codes, step, zp, bits, gran, group, rinv, bias_q, X, W, dt, bias, N, C_in, C_out,
+                                     mean_err, sums, ws, ws_bytes, (cudaStream_t)stream);
+}
+
 }  // extern "C"

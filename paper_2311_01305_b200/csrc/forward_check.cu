@@ -80,9 +80,11 @@ __global__ void __launch_bounds__(256) fc_rowsum_kernel(const unsigned char *__r
 //   acc = S - Z^x cw_o + Z^w (K Z^x - rx_n)
 // The CTA's sums of d = y~ - y, d^2 and y^2 go to partial[block][channel]; chunk after chunk
 // adds into the same slots in stream order.
-template <class D>
+// Weight-only mode (WO): the GEMM already produced d = x (W~ / s - W) in Dm; no integer part.
+template <class D, bool WO>
 __global__ void __launch_bounds__(256, 2)
-fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const float *__restrict__ Y, long long rows,
+fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const float *__restrict__ Dm,
+                  const float *__restrict__ Y, long long rows,
                   long long C_out, long long K, const float *__restrict__ act_step, const int *__restrict__ act_zp,
                   const int *__restrict__ rx, const float *__restrict__ w_step, const int *__restrict__ w_zp,
                   const int *__restrict__ cw, const float *__restrict__ bias_q, const uint16_t *__restrict__ bias,
@@ -99,29 +101,45 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
     if (live) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            sw[c] = (double)w_step[o0 + c];
-            zw[c] = (double)w_zp[o0 + c];
-            cwd[c] = (double)cw[o0 + c];
+            if (!WO) {
+                sw[c] = (double)w_step[o0 + c];
+                zw[c] = (double)w_zp[o0 + c];
+                cwd[c] = (double)cw[o0 + c];
+            }
             b[c] = bias ? (double)D::one(bias[o0 + c]) : 0.0;
             bq[c] = bias_q ? (double)bias_q[o0 + c] : b[c];      // no corrected bias: the layer keeps its own
         }
 #pragma unroll 4
         for (long long n = r0 + warp; n < r1; n += 8) {
-            const int4 s4 = __ldg(reinterpret_cast<const int4 *>(S + n * C_out + o0));
-            int4 t4 = make_int4(0, 0, 0, 0);
-            if (S2) t4 = __ldg(reinterpret_cast<const int4 *>(S2 + n * C_out + o0));
             const float4 y4 = __ldg(reinterpret_cast<const float4 *>(Y + n * C_out + o0));
-            const double zx = (double)act_zp[n];
-            const double u = (double)K * zx - (double)rx[n];
-            const double sx = (double)act_step[n];
-            const int sv[4] = {s4.x, s4.y, s4.z, s4.w}, tv[4] = {t4.x, t4.y, t4.z, t4.w};
             const float yv[4] = {y4.x, y4.y, y4.z, y4.w};
+            int sv[4] = {0, 0, 0, 0}, tv[4] = {0, 0, 0, 0};
+            float dv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            double zx = 0.0, u = 0.0, sx = 0.0;
+            if (WO) {
+                const float4 d4 = __ldg(reinterpret_cast<const float4 *>(Dm + n * C_out + o0));
+                dv[0] = d4.x; dv[1] = d4.y; dv[2] = d4.z; dv[3] = d4.w;
+            } else {
+                const int4 s4 = __ldg(reinterpret_cast<const int4 *>(S + n * C_out + o0));
+                sv[0] = s4.x; sv[1] = s4.y; sv[2] = s4.z; sv[3] = s4.w;
+                if (S2) {
+                    const int4 t4 = __ldg(reinterpret_cast<const int4 *>(S2 + n * C_out + o0));
+                    tv[0] = t4.x; tv[1] = t4.y; tv[2] = t4.z; tv[3] = t4.w;
+                }
+                zx = (double)act_zp[n];
+                u = (double)K * zx - (double)rx[n];
+                sx = (double)act_step[n];
+            }
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const double acc = ((double)sv[c] + (double)tv[c]) - zx * cwd[c] + zw[c] * u;
-                const double yq = sx * sw[c] * acc + bq[c];
                 const double y = (double)yv[c] + b[c];
-                const double d = yq - y;
+                double d;
+                if (WO) {
+                    d = (double)dv[c] + (bq[c] - b[c]);
+                } else {
+                    const double acc = ((double)sv[c] + (double)tv[c]) - zx * cwd[c] + zw[c] * u;
+                    d = (sx * sw[c] * acc + bq[c]) - y;
+                }
                 sd[c] += d;
                 sd2[c] += d * d;
                 sy2[c] += y * y;
@@ -236,17 +254,135 @@ aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, co
         // the grid always spans a full chunk's row blocks so that a short last chunk adds zeros, not garbage
         const dim3 grid((unsigned)((C_out + 127) / 128), (unsigned)L.blocks_per_chunk);
         if (dt == AWEQ_F16)
-            AWEQ_LAUNCH(fc_compare_kernel<F16>, grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
-                        (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
+            AWEQ_LAUNCH((fc_compare_kernel<F16, false>), grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
+                        (const float *)nullptr, (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
                         w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, (int)(c > 0));
         else
-            AWEQ_LAUNCH(fc_compare_kernel<BF16>, grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
-                        (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
+            AWEQ_LAUNCH((fc_compare_kernel<BF16, false>), grid, dim3(256), 0, stream, (const int *)S, (const int *)S2,
+                        (const float *)nullptr, (const float *)Y, rows, C_out, C_in, act_step + n0, act_zp + n0, (const int *)(rx + n0), w_step,
                         w_zp, (const int *)cw, bias_q, (const uint16_t *)bias, partial, (int)(c > 0));
     }
     double *cs = reinterpret_cast<double *>(Y);        // Y is free now: two doubles per output channel
     AWEQ_LAUNCH(fc_finish_kernel, dim3((unsigned)((C_out + 255) / 256)), dim3(256), 0, stream, (const double *)partial,
                 L.nblocks, C_out, N, mean_err, cs);
+    AWEQ_LAUNCH(fc_total_kernel, dim3(1), dim3(256), 0, stream, (const double *)cs, (const double *)mean_err, C_out, N, sums);
+    return AWEQ_OK;
+}
+
+// ------------------------------------------------------------------ weight-only check
+// dW[o, j] = round16( Step (q - Z) * (1/s_j) - W[o, j] ): what the quantised, equalised weights
+// differ by from the original ones once the 1/s of the input is folded back (Eq. 3), so that
+// x . dW is the output error of a weight-only layer.  One thread per eight columns.
+template <class D>
+__global__ void __launch_bounds__(256)
+fc_delta_kernel(const unsigned char *__restrict__ codes, const float *__restrict__ step, const int *__restrict__ zp,
+                int bits, int gran, int group, const float *__restrict__ rinv, const uint16_t *__restrict__ W,
+                long long C_out, long long C_in, uint16_t *__restrict__ dW)
+{
+    pdl_begin();
+    const long long nvec = C_in / 8;
+    const long long total = C_out * nvec;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long o = i / nvec, v = i - o * nvec;
+        const long long j0 = v * 8;
+        const long long k = gran == AWEQ_PER_TENSOR ? 0 : (gran == AWEQ_PER_ROW ? o : o * (C_in / group) + j0 / group);
+        const float st = __ldg(step + k);
+        const int z = __ldg(zp + k);
+        // eight codes = `bits` bytes of the row's little-endian bit stream
+        const unsigned char *src = codes + o * (C_in * bits / 8) + v * bits;
+        unsigned long long word = 0;
+        for (int t = 0; t < bits; ++t) word |= (unsigned long long)src[t] << (8 * t);
+        float w8[8], r8[8];
+        widen8<D>(ldg_stream(W + o * C_in + j0), w8);
+        if (rinv) load8(rinv + j0, r8);
+        uint32_t outw[4];
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+            uint32_t pair = 0;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int q = (int)((word >> ((e + h) * bits)) & ((1u << bits) - 1u));
+                float t = __fmul_rn(st, (float)((long long)q - (long long)z));
+                if (rinv) t = __fmul_rn(t, r8[e + h]);
+                pair |= (uint32_t)D::encode(__fsub_rn(t, w8[e + h])) << (16 * h);
+            }
+            outw[e / 2] = pair;
+        }
+        *reinterpret_cast<uint4 *>(dW + o * C_in + j0) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+    }
+}
+
+struct FcwLayout {
+    long long chunk, nchunks, blocks_per_chunk;
+    size_t dW, Dm, Y, partial, scratch, total;
+};
+
+static FcwLayout fcw_layout(long long N, long long C_in, long long C_out)
+{
+    FcwLayout L;
+    L.chunk = N < kFcChunk ? N : kFcChunk;
+    L.nchunks = (N + kFcChunk - 1) / kFcChunk;
+    L.blocks_per_chunk = (L.chunk + kFcRowBlock - 1) / kFcRowBlock;
+    size_t off = 0;
+    L.dW = off; off += up256((size_t)C_out * C_in * 2);
+    L.Dm = off; off += up256((size_t)L.chunk * C_out * 4);
+    L.Y = off; off += up256((size_t)L.chunk * C_out * 4);
+    L.partial = off; off += up256((size_t)L.blocks_per_chunk * C_out * 3 * 8);
+    L.scratch = off; off += kFcScratch;
+    L.total = off;
+    return L;
+}
+
+size_t forward_check_weights_ws_bytes(long long N, long long C_in, long long C_out)
+{
+    return fcw_layout(N, C_in, C_out).total;
+}
+
+aweq_status run_forward_check_weights(const unsigned char *codes, const float *step, const int *zp, int bits, int gran,
+                                      int group, const float *rinv, const float *bias_q, const void *X, const void *W,
+                                      aweq_dtype dt, const void *bias, long long N, long long C_in, long long C_out,
+                                      double *mean_err, double *sums, void *ws, size_t ws_bytes, cudaStream_t stream)
+{
+    const FcwLayout L = fcw_layout(N, C_in, C_out);
+    if (L.total > ws_bytes) return AWEQ_ERR_WORKSPACE;
+    char *base = reinterpret_cast<char *>(ws);
+    uint16_t *dW = reinterpret_cast<uint16_t *>(base + L.dW);
+    float *Dm = reinterpret_cast<float *>(base + L.Dm);
+    float *Y = reinterpret_cast<float *>(base + L.Y);
+    double *partial = reinterpret_cast<double *>(base + L.partial);
+    void *scratch = base + L.scratch;
+    long long blocks = (C_out * (C_in / 8) + 255) / 256;
+    if (blocks > (long long)kSmCount * 16) blocks = (long long)kSmCount * 16;
+    if (dt == AWEQ_F16)
+        AWEQ_LAUNCH(fc_delta_kernel<F16>, dim3((unsigned)blocks), dim3(256), 0, stream, codes, step, zp, bits, gran, group,
+                    rinv, (const uint16_t *)W, C_out, C_in, dW);
+    else
+        AWEQ_LAUNCH(fc_delta_kernel<BF16>, dim3((unsigned)blocks), dim3(256), 0, stream, codes, step, zp, bits, gran,
+                    group, rinv, (const uint16_t *)W, C_out, C_in, dW);
+    auto gemm = dt == AWEQ_F16 ? fc_gemm_f16 : fc_gemm_bf16;
+    for (long long c = 0; c < L.nchunks; ++c) {
+        const long long n0 = c * kFcChunk;
+        const long long rows = (N - n0) < kFcChunk ? (N - n0) : kFcChunk;
+        const uint16_t *Xc = reinterpret_cast<const uint16_t *>(X) + n0 * C_in;
+        aweq_status rc = gemm(Xc, dW, Dm, (int)rows, (int)C_out, (int)C_in, C_in, scratch, kFcScratch, stream);
+        if (rc != AWEQ_OK) return rc;
+        rc = gemm(Xc, W, Y, (int)rows, (int)C_out, (int)C_in, C_in, scratch, kFcScratch, stream);
+        if (rc != AWEQ_OK) return rc;
+        const dim3 grid((unsigned)((C_out + 127) / 128), (unsigned)L.blocks_per_chunk);
+        if (dt == AWEQ_F16)
+            AWEQ_LAUNCH((fc_compare_kernel<F16, true>), grid, dim3(256), 0, stream, (const int *)nullptr,
+                        (const int *)nullptr, (const float *)Dm, (const float *)Y, rows, C_out, C_in,
+                        (const float *)nullptr, (const int *)nullptr, (const int *)nullptr, (const float *)nullptr,
+                        (const int *)nullptr, (const int *)nullptr, bias_q, (const uint16_t *)bias, partial, (int)(c > 0));
+        else
+            AWEQ_LAUNCH((fc_compare_kernel<BF16, true>), grid, dim3(256), 0, stream, (const int *)nullptr,
+                        (const int *)nullptr, (const float *)Dm, (const float *)Y, rows, C_out, C_in,
+                        (const float *)nullptr, (const int *)nullptr, (const int *)nullptr, (const float *)nullptr,
+                        (const int *)nullptr, (const int *)nullptr, bias_q, (const uint16_t *)bias, partial, (int)(c > 0));
+    }
+    double *cs = reinterpret_cast<double *>(Y);        // Y is free now: two doubles per output channel
+    AWEQ_LAUNCH(fc_finish_kernel, dim3((unsigned)((C_out + 255) / 256)), dim3(256), 0, stream, (const double *)partial,
+                L.blocks_per_chunk, C_out, N, mean_err, cs);
     AWEQ_LAUNCH(fc_total_kernel, dim3(1), dim3(256), 0, stream, (const double *)cs, (const double *)mean_err, C_out, N, sums);
     return AWEQ_OK;
 }

@@ -48,6 +48,11 @@ aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, co
                               const void *X, const void *W, aweq_dtype dt, const void *bias, long long N,
                               long long C_in, long long C_out, double *mean_err, double *sums, void *ws,
                               size_t ws_bytes, cudaStream_t stream);
+size_t forward_check_weights_ws_bytes(long long N, long long C_in, long long C_out);
+aweq_status run_forward_check_weights(const unsigned char *codes, const float *step, const int *zp, int bits, int gran,
+                                      int group, const float *rinv, const float *bias_q, const void *X, const void *W,
+                                      aweq_dtype dt, const void *bias, long long N, long long C_in, long long C_out,
+                                      double *mean_err, double *sums, void *ws, size_t ws_bytes, cudaStream_t stream);
 // C[M x N] = A[M x K] B[N x K]^T on the tensor cores; A and B have ld elements per row
 aweq_status fc_gemm_u8(const void *A, const void *B, void *C, int M, int N, int K, long long ld, void *scratch,
                        size_t scratch_bytes, cudaStream_t stream);

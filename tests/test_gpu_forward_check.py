@@ -145,3 +145,87 @@ def test_forward_check_rejects_bad_arguments():
                                 z((N, C_in), torch.float16), z((C_out, C_in), torch.float16), None,
                                 z(C_out, torch.float64), z(4, torch.float64), ws=aweq.workspace(4096))
     assert e.value.code == 7          # AWEQ_ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------ weight-only forward check
+def _run_weights(codes, step, zp, bits, gran, group, rinv, bias_q, X, W, bias):
+    from paper_2311_01305_b200 import aweq
+    t = lambda a, dt=None: None if a is None else torch.as_tensor(np.ascontiguousarray(a), dtype=dt).to(DEV)
+    C_out = W.shape[0]
+    mean_err, check_me = util.guarded((C_out,), torch.float64)
+    sums, check_s = util.guarded((4,), torch.float64)
+    aweq.aweq_forward_check_weights(t(codes), t(step, torch.float32), t(zp, torch.int32), bits, gran, group,
+                                    t(rinv, torch.float32), t(bias_q, torch.float32), X.to(DEV), W.to(DEV),
+                                    None if bias is None else bias.to(DEV), mean_err, sums)
+    torch.cuda.synchronize()
+    check_me()
+    check_s()
+    return mean_err.cpu().numpy(), sums.cpu().numpy()
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("N,C_in,C_out,bits,gran,group", [
+    (1000, 256, 72, 4, orc.PER_GROUP, 128), (16384 + 77, 64, 40, 3, orc.PER_GROUP, 16),
+    (130, 4096, 136, 8, orc.PER_ROW, 0), (77, 48, 8, 5, orc.PER_TENSOR, 0), (90, 160, 24, 2, orc.PER_GROUP, 32)])
+def test_forward_check_weights_exact_operands(N, C_in, C_out, bits, gran, group, dtype):
+    """Power-of-two Step and 1/s and small-integer operands: dW = W~/s - W is exact in 16 bits and both
+    GEMMs are exact in binary32, so every output must agree with the oracle to binary64 rounding for
+    every bit-width, granularity, tile and chunk shape."""
+    seed = N + C_in + bits
+    rng = np.random.default_rng(seed)
+    glen = {orc.PER_ROW: C_in, orc.PER_TENSOR: C_out * C_in, orc.PER_GROUP: group}[gran]
+    npairs = C_out * C_in // glen
+    step = (2.0 ** rng.integers(-1, 1, npairs)).astype(np.float32)                # 0.5 or 1
+    zp = rng.integers(0, 1 << bits, npairs).astype(np.int32)
+    # codes within 12 of their zero-point: |W~ / s - W| <= 15 in quarters, exact even in bf16
+    q = np.clip(np.repeat(zp, glen).reshape(C_out, C_in) + rng.integers(-12, 13, (C_out, C_in)), 0, (1 << bits) - 1)
+    codes = orc.pack(q.astype(np.int32), bits)
+    rinv = (2.0 ** rng.integers(-1, 1, C_in)).astype(np.float32)                  # 0.5 or 1
+    X = _int_valued((N, C_in), dtype, seed + 2, 3)
+    W = _int_valued((C_out, C_in), dtype, seed + 3, 3)
+    bias = _int_valued((C_out,), dtype, seed + 4, 5)
+    bias_q = rng.standard_normal(C_out).astype(np.float32)
+    got_me, got_s = _run_weights(codes, step, zp, bits, gran, group, rinv, bias_q, X, W, bias)
+    ref_me, ref_s = orc.forward_check_weights(codes, step, zp, bits, gran, group, rinv, bias_q, util.bits(X), util.bits(W),
+                                              util.odt(X), util.bits(bias))
+    rms = np.sqrt(ref_s[0] / ref_s[3])
+    assert np.all(np.abs(got_me - ref_me) <= 1e-11 * rms)
+    assert np.allclose(got_s, ref_s, rtol=1e-11, atol=0)
+
+
+@pytest.mark.parametrize("dtype,bits,gran,group", [(torch.bfloat16, 4, orc.PER_GROUP, 128), (torch.bfloat16, 3, orc.PER_GROUP, 128),
+                                                   (torch.float16, 8, orc.PER_ROW, 0)])
+@pytest.mark.parametrize("correct", [True, False])
+def test_forward_check_weights_of_a_calibrated_layer(dtype, bits, gran, group, correct):
+    """Oracle calibration (steps 1-5) feeds both sides.  The GPU rounds dW = W~/s - W to 16 bits
+    (relative 2^-m, m = 9 for bf16 and 12 for fp16, plus three binary32 roundings of W~/s) and
+    accumulates both GEMMs in binary32 (K 2^-23 of the absolute sum): the bound below, per output."""
+    N, C_in, C_out = 1536 + 40, 768, 512 + 8
+    Xc = util.rand16((N, C_in), dtype, 61, scale=1.0, offset=0.5, outlier_cols=4)
+    Wc = util.rand16((C_out, C_in), dtype, 62, scale=0.03)
+    bias = util.rand16((1, C_out), dtype, 63, scale=0.1)[0].contiguous()
+    cal = util.oracle_layer(Xc, [Wc], bits, gran, group, biases=[bias], act_quant=False)
+    lin, f = cal["linears"][0], cal["factors"]
+    dt = util.odt(Xc)
+    bias_q = lin["bias_f32"] if correct else None
+    got_me, got_s = _run_weights(lin["codes"], lin["step"], lin["zp"], bits, gran, group, f["rinv"], bias_q, Xc, Wc, bias)
+    ref_me, ref_s = orc.forward_check_weights(lin["codes"], lin["step"], lin["zp"], bits, gran, group, f["rinv"], bias_q,
+                                              util.bits(Xc), util.bits(Wc), dt, util.bits(bias))
+    Wq = orc.dequantize(lin["codes"], lin["step"], lin["zp"], C_in, bits, gran, group) * f["rinv"].astype(np.float64)[None, :]
+    W64 = Wc.double().numpy()
+    Xa = np.abs(Xc.double().numpy())
+    m = 9 if dtype == torch.bfloat16 else 12
+    e_w = 2.0 ** -m * np.abs(Wq - W64) + 3 * 2.0 ** -24 * (np.abs(Wq) + np.abs(W64))      # rounding of dW
+    bound = Xa @ e_w.T + C_in * 2.0 ** -23 * (Xa @ (np.abs(Wq - W64) + e_w).T)           # d, per output
+    assert np.all(np.abs(got_me - ref_me) <= bound.mean(axis=0))
+    e2 = (bound ** 2).sum()
+    assert abs(got_s[0] - ref_s[0]) <= 2 * np.sqrt(ref_s[0] * e2) + e2
+    ybound = C_in * 2.0 ** -23 * (Xa @ np.abs(W64).T)
+    y2 = (ybound ** 2).sum()
+    assert abs(got_s[1] - ref_s[1]) <= 2 * np.sqrt(ref_s[1] * y2) + y2
+    assert got_s[3] == ref_s[3]
+    # in practice: the means agree to 2e-4 of the error's own RMS (bf16 dW), far inside the bound
+    d_rms = np.sqrt(ref_s[0] / ref_s[3])
+    assert np.abs(got_me - ref_me).max() <= 2e-4 * d_rms
+    if correct:
+        assert np.abs(ref_me).max() < 1e-3 * np.abs(lin["delta"]).max() + 1e-7      # Eq. 15 removed the mean error

@@ -614,3 +614,58 @@ def test_folds_leave_a_decoder_block_unchanged():
     fc2_in = np.maximum(x @ W1.T + b1, 0)
     fc2_in_f = np.maximum(x @ fold(W1, rinvf).T + fold(b1, rinvf), 0)
     assert np.all(np.abs(fc2_in_f - fc2_in * rinvf) <= tol * (np.abs(x) @ np.abs(W1).T + np.abs(b1)) * rinvf)
+
+
+# ---------------------------------------------------------------- weight-only forward check
+def test_forward_check_weights_hand_worked():
+    """2 tokens, 4 inputs, 2 outputs, 4-bit codes, groups of 2 (values exact in binary).
+    rinv = [1, .5, 2, 1];  X = [[1, 2, .5, -1], [0, 4, 1, 2]]  ->  x^ = [[1, 1, 1, -1], [0, 2, 2, 2]]
+    row 0: codes [3, 5 | 9, 1], Step [.5, .25], Z [3, 1]  ->  W~ = [0, 1, 2, 0]
+    row 1: codes [0, 15 | 4, 4], Step [1, 2],  Z [8, 4]   ->  W~ = [-8, 7, 0, 0]
+    y~ = x^ W~^T = [[3, -1], [6, 14]];  W = [[.5, .5, 1, 0], [-8, 3, 0, .5]]  ->  y = [[2, -2.5], [3, 13]]
+    d = [[1, 1.5], [3, 1]]  (no biases)."""
+    q = np.array([[3, 5, 9, 1], [0, 15, 4, 4]], np.int32)
+    codes = orc.pack(q, 4)
+    step, zp = np.array([0.5, 0.25, 1.0, 2.0], np.float32), np.array([3, 1, 8, 4], np.int32)
+    rinv = np.array([1, 0.5, 2, 1], np.float32)
+    X = f16_bits([[1, 2, 0.5, -1], [0, 4, 1, 2]])
+    W = f16_bits([[0.5, 0.5, 1, 0], [-8, 3, 0, 0.5]])
+    me, sums = orc.forward_check_weights(codes, step, zp, 4, orc.PER_GROUP, 2, rinv, None, X, W, orc.F16)
+    assert me.tolist() == [2.0, 1.25]
+    assert sums.tolist() == [1 + 2.25 + 9 + 1, 4 + 6.25 + 9 + 169, 4 + 1.5625, 4.0]
+    # biases: bias' - bias shifts every d of the channel; an uncorrected layer keeps its bias
+    bias = f16_bits([1.0, -2.0])
+    me_b, _ = orc.forward_check_weights(codes, step, zp, 4, orc.PER_GROUP, 2, rinv, np.array([0.5, -2.0], np.float32), X, W,
+                                        orc.F16, bias)
+    assert me_b.tolist() == [1.5, 1.25]
+    me_k, _ = orc.forward_check_weights(codes, step, zp, 4, orc.PER_GROUP, 2, rinv, None, X, W, orc.F16, bias)
+    assert me_k.tolist() == [2.0, 1.25]
+
+
+@pytest.mark.parametrize("bits,gran,group", [(8, orc.PER_ROW, 0), (4, orc.PER_GROUP, 8), (3, orc.PER_GROUP, 16),
+                                             (5, orc.PER_TENSOR, 0)])
+def test_forward_check_weights_against_numpy_and_bias_correction(bits, gran, group):
+    """NumPy matmul on the de-quantised weights; and Eq. 11-15 for a weight-only layer: after the
+    step-5 correction the mean output error vanishes (down to the binary32 rounding of mu_hat and
+    bias'), before it it is the step-4 sum eps . E[x^]."""
+    rng = np.random.default_rng(51 + bits)
+    X, W, Xd, Wd = _layer(rng, N=150, C_in=32, C_out=11, offset=True)
+    _, f = _factors_for(X, W)
+    codes, step, zp, delta = orc.equalize_quantize(W, orc.F16, f["s"], f["mu_hat"], bits, gran, group)
+    bias = f16_bits(rng.standard_normal(11) * 0.1)
+    bf, _ = orc.bias_correct(delta, bias, orc.F16)
+    raw, sums_raw = orc.forward_check_weights(codes, step, zp, bits, gran, group, f["rinv"], None, X, W, orc.F16, bias)
+    fixed, _ = orc.forward_check_weights(codes, step, zp, bits, gran, group, f["rinv"], bf, X, W, orc.F16, bias)
+    Wq = orc.dequantize(codes, step, zp, 32, bits, gran, group)
+    Xh = Xd.astype(np.float64) * f["rinv"].astype(np.float64)[None, :]
+    b64 = bits_to_f64(bias, orc.F16)
+    y = Xd.astype(np.float64) @ Wd.astype(np.float64).T + b64
+    d = (Xh @ Wq.T + b64) - y
+    assert np.allclose(raw, d.mean(axis=0), rtol=1e-10, atol=1e-12)
+    assert np.allclose(sums_raw, [(d * d).sum(), (y * y).sum(), (d.mean(axis=0) ** 2).sum(), d.size], rtol=1e-10)
+    # eps is taken against W^ = fl(W s) and E[x^] = fl(mean x * rinv): binary32 roundings of the equalised
+    # operands separate the two routes by parts in 1e-6 of the terms
+    scale = (np.abs(Wq) * np.abs(Xh).mean(axis=0)[None, :]).sum(axis=1)
+    assert np.all(np.abs(raw - delta) <= 3e-6 * scale)
+    assert np.all(np.abs(fixed) <= 3e-6 * scale + 2.0 ** -24 * np.abs(bf))
+    assert np.abs(raw).max() > 20 * np.abs(fixed).max()
