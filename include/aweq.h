@@ -325,10 +325,12 @@ aweq_status aweq_forward_check(const unsigned char *Xq, const float *act_step, c
  * step 3, NULL = no equalisation) and W~ = Step (q - Z) the de-quantised step-4 codes,
  *     y~[n,o] = sum_j (X[n,j] rinv[j]) W~[o,j] + bias_q[o]        y[n,o] = sum_j X[n,j] W[o,j] + bias[o]
  * and the outputs are those of aweq_forward_check (mean_err[C_out], sums[4]; bias_q NULL = the
- * layer keeps bias).  The library forms dW = round16(W~ rinv - W) once ([C_out x C_in], 16-bit)
- * and runs two 16-bit tensor-core GEMMs per token chunk, X dW^T (the error itself) and X W^T.
+ * layer keeps bias).  The library forms dW = W~ rinv - W once; the mean error, linear in x, is
+ * E[x] . dW from the binary64 column sums of X and the unrounded dW; the sums of squares come
+ * from two 16-bit tensor-core GEMMs per token chunk, X round16(dW)^T (the error) and X W^T.
  * codes / step / zp / bits / gran / group exactly as aweq_equalize_quantize wrote them; X and W
- * contiguous, 16-byte aligned; C_in a multiple of 16, C_out of 8.
+ * contiguous, 16-byte aligned; C_in a multiple of 16 and within the range of aweq_stats, C_out
+ * a multiple of 8.
  * ws: aweq_forward_check_weights_workspace_bytes(N, C_in, C_out), 256-byte aligned. */
 size_t aweq_forward_check_weights_workspace_bytes(long long N, long long C_in, long long C_out);
 aweq_status aweq_forward_check_weights(const unsigned char *codes, const float *step, const int *zp, int bits,

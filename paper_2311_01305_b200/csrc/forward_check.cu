@@ -168,7 +168,7 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
 
 __global__ void __launch_bounds__(256)
 fc_finish_kernel(const double *__restrict__ partial, long long nblocks, long long C_out, long long N,
-                 double *__restrict__ mean_err, double *__restrict__ col_sums)
+                 double *__restrict__ mean_err, double *__restrict__ col_sums, int write_mean)
 {
     pdl_begin();
     const long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -180,7 +180,7 @@ fc_finish_kernel(const double *__restrict__ partial, long long nblocks, long lon
         sd2 += p[1];
         sy2 += p[2];
     }
-    mean_err[o] = sd / (double)N;
+    if (write_mean) mean_err[o] = sd / (double)N;
     col_sums[o * 2] = sd2;
     col_sums[o * 2 + 1] = sy2;
 }
@@ -264,57 +264,74 @@ aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, co
     }
     double *cs = reinterpret_cast<double *>(Y);        // Y is free now: two doubles per output channel
     AWEQ_LAUNCH(fc_finish_kernel, dim3((unsigned)((C_out + 255) / 256)), dim3(256), 0, stream, (const double *)partial,
-                L.nblocks, C_out, N, mean_err, cs);
+                L.nblocks, C_out, N, mean_err, cs, 1);
     AWEQ_LAUNCH(fc_total_kernel, dim3(1), dim3(256), 0, stream, (const double *)cs, (const double *)mean_err, C_out, N, sums);
     return AWEQ_OK;
 }
 
 // ------------------------------------------------------------------ weight-only check
-// dW[o, j] = round16( Step (q - Z) * (1/s_j) - W[o, j] ): what the quantised, equalised weights
-// differ by from the original ones once the 1/s of the input is folded back (Eq. 3), so that
-// x . dW is the output error of a weight-only layer.  One thread per eight columns.
+// dW[o, j] = Step (q - Z) * (1/s_j) - W[o, j]: what the quantised, equalised weights differ by
+// from the original ones once the 1/s of the input is folded back (Eq. 3), so that x . dW is
+// the output error of a weight-only layer.  One warp per output row.  dW goes to memory
+// rounded to 16 bits for the GEMM (good enough for the sums of squares); the MEAN error is
+// linear in x, E[x . dW] = E[x] . dW, and is taken here from the unrounded dW and the binary64
+// column sums of X, so it is not limited by the 16-bit rounding:
+//     mean_err[o] = (sum_j xsum[j] dW[o, j]) / N + (bias_q[o] - bias[o])
 template <class D>
 __global__ void __launch_bounds__(256)
 fc_delta_kernel(const unsigned char *__restrict__ codes, const float *__restrict__ step, const int *__restrict__ zp,
                 int bits, int gran, int group, const float *__restrict__ rinv, const uint16_t *__restrict__ W,
-                long long C_out, long long C_in, uint16_t *__restrict__ dW)
+                long long C_out, long long C_in, uint16_t *__restrict__ dW, const double *__restrict__ xsum,
+                long long N, const float *__restrict__ bias_q, const uint16_t *__restrict__ bias,
+                double *__restrict__ mean_err)
 {
     pdl_begin();
+    const int lane = threadIdx.x & 31;
     const long long nvec = C_in / 8;
-    const long long total = C_out * nvec;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const long long o = i / nvec, v = i - o * nvec;
-        const long long j0 = v * 8;
-        const long long k = gran == AWEQ_PER_TENSOR ? 0 : (gran == AWEQ_PER_ROW ? o : o * (C_in / group) + j0 / group);
-        const float st = __ldg(step + k);
-        const int z = __ldg(zp + k);
-        // eight codes = `bits` bytes of the row's little-endian bit stream
-        const unsigned char *src = codes + o * (C_in * bits / 8) + v * bits;
-        unsigned long long word = 0;
-        for (int t = 0; t < bits; ++t) word |= (unsigned long long)src[t] << (8 * t);
-        float w8[8], r8[8];
-        widen8<D>(ldg_stream(W + o * C_in + j0), w8);
-        if (rinv) load8(rinv + j0, r8);
-        uint32_t outw[4];
+    for (long long o = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); o < C_out; o += (long long)gridDim.x * 8) {
+        double dot = 0.0;
+        for (long long v = lane; v < nvec; v += 32) {
+            const long long j0 = v * 8;
+            const long long k = gran == AWEQ_PER_TENSOR ? 0 : (gran == AWEQ_PER_ROW ? o : o * (C_in / group) + j0 / group);
+            const float st = __ldg(step + k);
+            const int z = __ldg(zp + k);
+            // eight codes = `bits` bytes of the row's little-endian bit stream
+            const unsigned char *src = codes + o * (C_in * bits / 8) + v * bits;
+            unsigned long long word = 0;
+            for (int t = 0; t < bits; ++t) word |= (unsigned long long)src[t] << (8 * t);
+            float w8[8], r8[8];
+            widen8<D>(ldg_stream(W + o * C_in + j0), w8);
+            if (rinv) load8(rinv + j0, r8);
+            uint32_t outw[4];
 #pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-            uint32_t pair = 0;
+            for (int e = 0; e < 8; e += 2) {
+                uint32_t pair = 0;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int q = (int)((word >> ((e + h) * bits)) & ((1u << bits) - 1u));
-                float t = __fmul_rn(st, (float)((long long)q - (long long)z));
-                if (rinv) t = __fmul_rn(t, r8[e + h]);
-                pair |= (uint32_t)D::encode(__fsub_rn(t, w8[e + h])) << (16 * h);
+                for (int h = 0; h < 2; ++h) {
+                    const int q = (int)((word >> ((e + h) * bits)) & ((1u << bits) - 1u));
+                    float t = __fmul_rn(st, (float)((long long)q - (long long)z));
+                    if (rinv) t = __fmul_rn(t, r8[e + h]);
+                    const float dw = __fsub_rn(t, w8[e + h]);
+                    dot += xsum[j0 + e + h] * (double)dw;
+                    pair |= (uint32_t)D::encode(dw) << (16 * h);
+                }
+                outw[e / 2] = pair;
             }
-            outw[e / 2] = pair;
+            *reinterpret_cast<uint4 *>(dW + o * C_in + j0) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
         }
-        *reinterpret_cast<uint4 *>(dW + o * C_in + j0) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, w);
+        if (lane == 0) {
+            const double b = bias ? (double)D::one(bias[o]) : 0.0;
+            const double bq = bias_q ? (double)bias_q[o] : b;
+            mean_err[o] = dot / (double)N + (bq - b);
+        }
     }
 }
 
 struct FcwLayout {
     long long chunk, nchunks, blocks_per_chunk;
-    size_t dW, Dm, Y, partial, scratch, total;
+    size_t dW, Dm, Y, partial, xsum, xtmp, colws, scratch, total;
 };
 
 static FcwLayout fcw_layout(long long N, long long C_in, long long C_out)
@@ -328,6 +345,9 @@ static FcwLayout fcw_layout(long long N, long long C_in, long long C_out)
     L.Dm = off; off += up256((size_t)L.chunk * C_out * 4);
     L.Y = off; off += up256((size_t)L.chunk * C_out * 4);
     L.partial = off; off += up256((size_t)L.blocks_per_chunk * C_out * 3 * 8);
+    L.xsum = off; off += up256((size_t)C_in * 8);
+    L.xtmp = off; off += up256((size_t)C_in * 4) * 3;                 // min, max, mean of the column sweep (unused)
+    L.colws = off; off += up256(colreduce_ws_bytes(N, C_in));
     L.scratch = off; off += kFcScratch;
     L.total = off;
     return L;
@@ -351,14 +371,23 @@ aweq_status run_forward_check_weights(const unsigned char *codes, const float *s
     float *Y = reinterpret_cast<float *>(base + L.Y);
     double *partial = reinterpret_cast<double *>(base + L.partial);
     void *scratch = base + L.scratch;
-    long long blocks = (C_out * (C_in / 8) + 255) / 256;
-    if (blocks > (long long)kSmCount * 16) blocks = (long long)kSmCount * 16;
+    // binary64 column sums of X (the step-1 sweep), for the mean error
+    double *xsum = reinterpret_cast<double *>(base + L.xsum);
+    float *xtmp = reinterpret_cast<float *>(base + L.xtmp);
+    const size_t tstride = up256((size_t)C_in * 4) / 4;
+    aweq_status rs = run_stats(X, dt, N, C_in, C_in, xtmp, xtmp + tstride, xtmp + 2 * tstride, xsum, nullptr, 0,
+                               base + L.colws, nullptr, stream);
+    if (rs != AWEQ_OK) return rs;
+    long long blocks = (C_out + 7) / 8;
+    if (blocks > (long long)kSmCount * 8) blocks = (long long)kSmCount * 8;
     if (dt == AWEQ_F16)
         AWEQ_LAUNCH(fc_delta_kernel<F16>, dim3((unsigned)blocks), dim3(256), 0, stream, codes, step, zp, bits, gran, group,
-                    rinv, (const uint16_t *)W, C_out, C_in, dW);
+                    rinv, (const uint16_t *)W, C_out, C_in, dW, (const double *)xsum, N, bias_q, (const uint16_t *)bias,
+                    mean_err);
     else
         AWEQ_LAUNCH(fc_delta_kernel<BF16>, dim3((unsigned)blocks), dim3(256), 0, stream, codes, step, zp, bits, gran,
-                    group, rinv, (const uint16_t *)W, C_out, C_in, dW);
+                    group, rinv, (const uint16_t *)W, C_out, C_in, dW, (const double *)xsum, N, bias_q,
+                    (const uint16_t *)bias, mean_err);
     auto gemm = dt == AWEQ_F16 ? fc_gemm_f16 : fc_gemm_bf16;
     for (long long c = 0; c < L.nchunks; ++c) {
         const long long n0 = c * kFcChunk;
@@ -382,7 +411,7 @@ aweq_status run_forward_check_weights(const unsigned char *codes, const float *s
     }
     double *cs = reinterpret_cast<double *>(Y);        // Y is free now: two doubles per output channel
     AWEQ_LAUNCH(fc_finish_kernel, dim3((unsigned)((C_out + 255) / 256)), dim3(256), 0, stream, (const double *)partial,
-                L.blocks_per_chunk, C_out, N, mean_err, cs);
+                L.blocks_per_chunk, C_out, N, mean_err, cs, 0);
     AWEQ_LAUNCH(fc_total_kernel, dim3(1), dim3(256), 0, stream, (const double *)cs, (const double *)mean_err, C_out, N, sums);
     return AWEQ_OK;
 }
