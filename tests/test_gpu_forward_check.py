@@ -227,9 +227,9 @@ def test_forward_check_weights_of_a_calibrated_layer(dtype, bits, gran, group, c
     y2 = (ybound ** 2).sum()
     assert abs(got_s[1] - ref_s[1]) <= 2 * np.sqrt(ref_s[1] * y2) + y2
     assert got_s[3] == ref_s[3]
-    # in practice: the means agree to 1e-6 of the error's RMS, the mean squared error to 1e-3
+    # in practice: the means agree to 1e-5 of the error's RMS, the mean squared error to 1e-3
     d_rms = np.sqrt(ref_s[0] / ref_s[3])
-    assert np.abs(got_me - ref_me).max() <= 1e-6 * d_rms
+    assert np.abs(got_me - ref_me).max() <= 1e-5 * d_rms
     assert abs(got_s[0] - ref_s[0]) <= 1e-3 * ref_s[0]
     if correct:
         assert np.abs(ref_me).max() < 1e-3 * np.abs(lin["delta"]).max() + 1e-7      # Eq. 15 removed the mean error
