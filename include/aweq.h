@@ -12,8 +12,8 @@
  *   6. 8-bit quantisation of the equalised inputs (W8A8)     aweq_quant_act
  * aweq_layer_pass runs all six for one input and the matrices it feeds.
  * Around the pass: aweq_fold_scale folds diag(s)^-1 into the producer of an input
- * (Section 3.1) and aweq_forward_check measures what Eq. 11 names, E[y~ - y], for a
- * calibrated W8A8 layer on the tensor cores.
+ * (Section 3.1); aweq_forward_check (W8A8) and aweq_forward_check_weights (weight-only)
+ * measure what Eq. 11 names, E[y~ - y], for a calibrated layer on the tensor cores.
  *
  * General rules
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned
