@@ -75,7 +75,8 @@ __global__ void __launch_bounds__(256) fc_rowsum_kernel(const unsigned char *__r
 // Comparison of one token chunk.  A CTA covers kFcRowBlock tokens x 128 output channels: a lane
 // owns four adjacent channels (16-byte loads of S and Y), the eight warps take the tokens
 // round-robin, and the per-warp sums are added in warp order through shared memory, so the
-// result does not depend on scheduling.  The integer part is formed in 64-bit integers:
+// result does not depend on scheduling.  The integer part is formed in binary64, where it is
+// exact (every term is an integer below 2^53):
 //   acc = S - Z^x cw_o + Z^w (K Z^x - rx_n)
 // The CTA's sums of d = y~ - y, d^2 and y^2 go to partial[block][channel]; chunk after chunk
 // adds into the same slots in stream order.
@@ -94,8 +95,7 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long o0 = (long long)blockIdx.x * 128 + lane * 4;
     const long long r0 = (long long)blockIdx.y * kFcRowBlock, r1 = min(rows, r0 + (long long)kFcRowBlock);
-    double sw[4], bq[4], b[4];
-    int zw[4], cwi[4];
+    double sw[4], zw[4], cwd[4], bq[4], b[4];
     double sd[4] = {0, 0, 0, 0}, sd2[4] = {0, 0, 0, 0}, sy2[4] = {0, 0, 0, 0};
     const bool live = o0 < C_out;                    // C_out is a multiple of 8: a lane's four channels are all in or all out
     if (live) {
@@ -103,8 +103,8 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
         for (int c = 0; c < 4; ++c) {
             if (!WO) {
                 sw[c] = (double)w_step[o0 + c];
-                zw[c] = w_zp[o0 + c];
-                cwi[c] = cw[o0 + c];
+                zw[c] = (double)w_zp[o0 + c];
+                cwd[c] = (double)cw[o0 + c];
             }
             b[c] = bias ? (double)D::one(bias[o0 + c]) : 0.0;
             bq[c] = bias_q ? (double)bias_q[o0 + c] : b[c];      // no corrected bias: the layer keeps its own
@@ -115,8 +115,7 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
             const float yv[4] = {y4.x, y4.y, y4.z, y4.w};
             int sv[4] = {0, 0, 0, 0}, tv[4] = {0, 0, 0, 0};
             float dv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-            long long zx = 0, u = 0;
-            double sx = 0.0;
+            double zx = 0.0, u = 0.0, sx = 0.0;
             if (WO) {
                 const float4 d4 = __ldg(reinterpret_cast<const float4 *>(Dm + n * C_out + o0));
                 dv[0] = d4.x; dv[1] = d4.y; dv[2] = d4.z; dv[3] = d4.w;
@@ -127,8 +126,8 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
                     const int4 t4 = __ldg(reinterpret_cast<const int4 *>(S2 + n * C_out + o0));
                     tv[0] = t4.x; tv[1] = t4.y; tv[2] = t4.z; tv[3] = t4.w;
                 }
-                zx = act_zp[n];
-                u = K * zx - (long long)rx[n];
+                zx = (double)act_zp[n];
+                u = (double)K * zx - (double)rx[n];
                 sx = (double)act_step[n];
             }
 #pragma unroll
@@ -138,9 +137,8 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
                 if (WO) {
                     d = (double)dv[c] + (bq[c] - b[c]);
                 } else {
-                    // the integer part in 64-bit integers (one conversion to binary64 instead of three)
-                    const long long acc = (long long)sv[c] + tv[c] - zx * cwi[c] + (long long)zw[c] * u;
-                    d = (sx * sw[c] * (double)acc + bq[c]) - y;
+                    const double acc = ((double)sv[c] + (double)tv[c]) - zx * cwd[c] + zw[c] * u;
+                    d = (sx * sw[c] * acc + bq[c]) - y;
                 }
                 sd[c] += d;
                 sd2[c] += d * d;
