@@ -35,7 +35,7 @@ sys.path.insert(0, ROOT)
 from paper_2311_01305_b200 import synth  # noqa: E402
 
 DEFAULT_WORKLOAD = "llama7b_layer_w4w3_g128"
-NORTH_STAR_PEAK_GBS = 8000.0
+NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0
 
@@ -367,7 +367,7 @@ def main():
                    "algorithmic_bytes_per_gpu": nbytes, "cache": "inputs (GBs) far larger than the 126 MB L2",
                    "parallelism": "token shards, one per GPU" if world > 1 else "single GPU"},
         "tokens_per_s": world * tokens / (ms / 1e3),
-        "pct_of_8000_gbs": 100.0 * gbs / world / NORTH_STAR_PEAK_GBS,
+        "pct_of_8000_gbs": 100.0 * gbs / world / NOMINAL_HBM_GBS,
         "pct_of_measured_copy": 100.0 * gbs / world / peak,
         "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "device_status": status,
     }
