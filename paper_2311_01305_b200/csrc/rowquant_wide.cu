@@ -24,7 +24,7 @@ constexpr int kRwHeader = 4096;
 
 struct RwSmem {
     RqSmem ring;                       // full / empty barriers, abort flag
-    float2 red[2][32][kRwMaxR];        // per-warp (lo, hi) of each row of the tile, by tile parity
+    float2 red[32][kRwMaxR];           // per-warp (lo, hi) of each row of the tile
     float4 q[kRwMaxR];                 // Step, 1/Step, Z (bits), flags (bits)
 };
 static_assert(sizeof(RwSmem) <= kRwHeader, "header");
@@ -143,54 +143,30 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
         for (int r = 0; r < kRwMaxR; ++r) {
             if (r < rows) {
                 const float l = redux_min(lo[r], 0xffffffffu), h = redux_max(hi[r], 0xffffffffu);
-                if (lane == 0) sm->red[k & 1][warp][r] = make_float2(l, h);
+                if (lane == 0) sm->red[warp][r] = make_float2(l, h);
             }
         }
         // the barrier doubles as the agreement on a timed-out wait: everybody leaves or nobody
         ok = __syncthreads_and(ok);
         if (!ok) break;
-        // 512 threads: warp r finishes row r and a second barrier publishes Step / Z.  1024 threads
-        // (one or two rows per tile): every warp finishes the rows itself from the partials, which
-        // costs ~50 instructions per warp and row and saves the second barrier, the larger cost there.
-        // The partials alternate between two buffers, so a warp that runs ahead into the next tile
-        // cannot overwrite what a slower warp still reads.
-        constexpr bool kOneBarrier = NT == 1024;
-        float4 qown[kOneBarrier ? kRwMaxR : 1];
-        if (kOneBarrier) {
-#pragma unroll
-            for (int r = 0; r < kRwMaxR; ++r) {
-                if (r < rows) {
-                    const float2 o = sm->red[k & 1][lane][r];          // NW == 32: one partial per lane
-                    const float l = redux_min(o.x, 0xffffffffu), h = redux_max(o.y, 0xffffffffu);
-                    const QParams q = make_qparams(l, h, qmax);
-                    const int fl = qflags(q, h, qmax);
-                    qown[r] = make_float4(q.step, q.inv, __int_as_float(q.zp), __int_as_float(fl));
-                    if (threadIdx.x == 0) {
-                        p.step[row0 + r] = q.step;
-                        p.zp[row0 + r] = q.zp;
-                    }
-                }
+        if (warp < rows) {
+            const float2 o = lane < NW ? sm->red[lane][warp] : make_float2(INFINITY, -INFINITY);
+            const float l = redux_min(o.x, 0xffffffffu), h = redux_max(o.y, 0xffffffffu);
+            const QParams q = make_qparams(l, h, qmax);
+            const int fl = qflags(q, h, qmax);
+            if (lane == 0) {
+                sm->q[warp] = make_float4(q.step, q.inv, __int_as_float(q.zp), __int_as_float(fl));
+                p.step[row0 + warp] = q.step;
+                p.zp[row0 + warp] = q.zp;
             }
-        } else {
-            if (warp < rows) {
-                const float2 o = lane < NW ? sm->red[k & 1][lane][warp] : make_float2(INFINITY, -INFINITY);
-                const float l = redux_min(o.x, 0xffffffffu), h = redux_max(o.y, 0xffffffffu);
-                const QParams q = make_qparams(l, h, qmax);
-                const int fl = qflags(q, h, qmax);
-                if (lane == 0) {
-                    sm->q[warp] = make_float4(q.step, q.inv, __int_as_float(q.zp), __int_as_float(fl));
-                    p.step[row0 + warp] = q.step;
-                    p.zp[row0 + warp] = q.zp;
-                }
-            }
-            __syncthreads();
         }
+        __syncthreads();
 
         // ---- pass 2: codes
 #pragma unroll
         for (int r = 0; r < kRwMaxR; ++r) {
             if (r < rows) {
-                const float4 qv = kOneBarrier ? qown[kOneBarrier ? r : 0] : sm->q[r];
+                const float4 qv = sm->q[r];
                 const float inv = qv.y;
                 const int zp = __float_as_int(qv.z), fl = __float_as_int(qv.w);
                 const uint4 *rowp = tile + (size_t)r * p.nvec;
