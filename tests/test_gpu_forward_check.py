@@ -233,3 +233,34 @@ def test_forward_check_weights_of_a_calibrated_layer(dtype, bits, gran, group, c
     assert abs(got_s[0] - ref_s[0]) <= 1e-3 * ref_s[0]
     if correct:
         assert np.abs(ref_me).max() < 1e-3 * np.abs(lin["delta"]).max() + 1e-7      # Eq. 15 removed the mean error
+
+
+def test_forward_check_layer_sized_sampled_channels():
+    """A LLaMA-13B-sized projection (5120 x 5120) on four token chunks, calibrated by the oracle; the
+    oracle then evaluates a sample of output channels (a forward check of those rows of W alone),
+    which must match the same channels of the full GPU check."""
+    N, C = 3 * 16384 + 24, 5120
+    Xc = util.rand16((N, C), torch.float16, 71, scale=1.0, offset=0.5, outlier_cols=26, outlier_scale=80.0)
+    Wc = util.rand16((C, C), torch.float16, 72, scale=0.015)
+    cal = util.oracle_layer(Xc, [Wc], 8, orc.PER_ROW, 0)
+    lin, (Xq, act_step, act_zp) = cal["linears"][0], cal["act"]
+    got_me, got_s = _run(Xq, act_step, act_zp, lin["codes"], lin["step"], lin["zp"], lin["bias_f32"], Xc, Wc, None)
+    rows = np.array([0, 1234, 2559, 5119])
+    ref_me, ref_s = orc.forward_check(Xq, act_step, act_zp, lin["codes"][rows], lin["step"][rows], lin["zp"][rows],
+                                      lin["bias_f32"][rows], util.bits(Xc), util.bits(Wc[rows].contiguous()), orc.F16)
+    y_rms = np.sqrt(ref_s[1] / ref_s[3])
+    assert np.abs(got_me[rows] - ref_me).max() <= 1e-5 * y_rms
+    assert got_s[3] == N * C
+    # the sampled channels carry their share of the sums (the layer is statistically uniform over channels)
+    assert 0.5 < (got_s[0] / C) / (ref_s[0] / len(rows)) < 2.0
+    # weight-only check of the same layer at 4 bits, same sample
+    cal4 = util.oracle_layer(Xc, [Wc], 4, orc.PER_GROUP, 128, act_quant=False)
+    l4, f4 = cal4["linears"][0], cal4["factors"]
+    got4, s4 = _run_weights(l4["codes"], l4["step"], l4["zp"], 4, orc.PER_GROUP, 128, f4["rinv"], l4["bias_f32"], Xc, Wc, None)
+    ng = C // 128
+    pick = (rows[:, None] * ng + np.arange(ng)[None, :]).reshape(-1)
+    ref4, r4 = orc.forward_check_weights(l4["codes"][rows], l4["step"][pick], l4["zp"][pick], 4, orc.PER_GROUP, 128, f4["rinv"],
+                                         l4["bias_f32"][rows], util.bits(Xc), util.bits(Wc[rows].contiguous()), orc.F16)
+    d_rms = np.sqrt(r4[0] / r4[3])
+    assert np.abs(got4[rows] - ref4).max() <= 1e-5 * d_rms
+    assert 0.5 < (s4[0] / C) / (r4[0] / len(rows)) < 2.0
