@@ -252,6 +252,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="issue every input's pass on one stream (default: two alternating streams)")
     ap.add_argument("--op", default="layer_pass", choices=["layer_pass", "forward_check"],
                     help="forward_check: time the W8A8 forward check of the calibrated layer instead (1 GPU)")
     args = ap.parse_args()
@@ -278,7 +280,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     X, W = generate(wl, dev, rank)
-    cal = calibrate.ShardedLayerCalibrator(wl, bits, X, W, None) if world > 1 else calibrate.LayerCalibrator(wl, bits, X, W, None)
+    cal = (calibrate.ShardedLayerCalibrator(wl, bits, X, W, None) if world > 1
+           else calibrate.LayerCalibrator(wl, bits, X, W, None, overlap=not args.no_overlap))
     nbytes = calibrate.algorithmic_bytes(wl, bits)
     tokens = wl.inputs[0].n_tokens
 
@@ -313,7 +316,7 @@ def main():
         else:
             for lp, (es, ea) in zip(cal.passes, hooks[k]):
                 lp.set_events(es, ea)
-                lp(cal.ws, cal.status)
+            cal.run()
     t_end.record()
     barrier()
     launches = aweq.launch_count() - n0

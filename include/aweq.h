@@ -254,6 +254,16 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
  */
 #define AWEQ_FLAG_NO_EQUALIZE 1      /* s = 1: plain round-to-nearest */
 #define AWEQ_FLAG_NO_BIAS_CORRECT 2  /* skip step 5 */
+/* Run only part of the pass (any combination; none of the three = the whole pass).  The parts
+ * communicate through the per-channel arrays of the argument block, so a caller can put them
+ * on different streams -- the HBM-bound sweeps over X on one, the short weight kernels on
+ * another -- ordering them with its own events and giving each stream its own `ws`:
+ *   STATS   step 1 (writes xmin, xmax, xmean)
+ *   WEIGHTS steps 2-5 (reads them; writes wmin, wmax, s, rinv, mu_hat, codes, Step, Z, biases)
+ *   ACT     step 6 (reads rinv; writes Xq, act_step, act_zp) */
+#define AWEQ_FLAG_PHASE_STATS 4
+#define AWEQ_FLAG_PHASE_WEIGHTS 8
+#define AWEQ_FLAG_PHASE_ACT 16
 
 typedef struct {
     /* input */

@@ -37,7 +37,13 @@ def algorithmic_bytes(wl: synth.Workload, bits: int) -> int:
 
 class LayerCalibrator:
     def __init__(self, wl: synth.Workload, bits: int, X: Dict[str, torch.Tensor], W: Dict[str, torch.Tensor],
-                 bias: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0, diagnostics: bool = True):
+                 bias: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0, diagnostics: bool = True,
+                 overlap: bool = False):
+        """``overlap``: split every pass into its parts (``FLAG_PHASE_*``) and issue the HBM-bound
+        sweeps over X (steps 1 and 6) on one CUDA stream and the short, issue-bound weight
+        kernels (steps 2-5) on another, each with its own scratch and ordered by events, so that
+        the weight kernels of one input run under the statistics sweep of the next; ``run()``
+        forks from and joins back into the current stream."""
         self.wl, self.bits = wl, bits
         dev = next(iter(X.values())).device
         td = synth.torch_dtype(wl.dtype)
@@ -86,13 +92,49 @@ class LayerCalibrator:
             self.passes.append(lp)
         self.ws = aweq.workspace(ws_bytes, dev)
         self.status = aweq.new_status(dev)
+        self.overlap = bool(overlap) and len(self.passes) > 1 and dev.type == "cuda"
+        if self.overlap:
+            self._streams = (torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev))
+            self._ws2 = (self.ws, aweq.workspace(ws_bytes, dev))
+            self._fork = torch.cuda.Event()
+            self._ev_stats = [torch.cuda.Event() for _ in self.passes]
+            self._ev_weights = [torch.cuda.Event() for _ in self.passes]
         self._fc_ws, self._fc_out = None, {}
         self.equalized = not (flags & aweq.FLAG_NO_EQUALIZE)
 
     def run(self) -> None:
         """One calibration pass of the whole layer: one library call per input."""
-        for lp in self.passes:
-            lp(self.ws, self.status)
+        if not self.overlap:
+            for lp in self.passes:
+                lp(self.ws, self.status)
+            return
+        cur = torch.cuda.current_stream()
+        big, small = self._streams
+        ws_big, ws_small = self._ws2
+        self._fork.record(cur)
+        big.wait_event(self._fork)
+        small.wait_event(self._fork)
+        n = len(self.passes)
+
+        def stats(i):
+            with torch.cuda.stream(big):
+                self.passes[i](ws_big, self.status, aweq.FLAG_PHASE_STATS)
+                self._ev_stats[i].record(big)
+
+        stats(0)
+        for i, lp in enumerate(self.passes):
+            with torch.cuda.stream(small):
+                small.wait_event(self._ev_stats[i])
+                lp(ws_small, self.status, aweq.FLAG_PHASE_WEIGHTS)
+                self._ev_weights[i].record(small)
+            if i + 1 < n:
+                stats(i + 1)                       # the next sweep goes ahead of this input's step 6
+            if self.wl.act_quant:
+                with torch.cuda.stream(big):
+                    big.wait_event(self._ev_weights[i])
+                    lp(ws_big, self.status, aweq.FLAG_PHASE_ACT)
+        cur.wait_stream(big)
+        cur.wait_stream(small)
 
     def forward_check(self, X, W, bias=None, corrected: bool = True):
         """The forward check of every linear after ``run()``: {linear name: (mean_err[C_out],

@@ -313,12 +313,23 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     const size_t ws_eq_bytes = need - col_part;
 
     cudaStream_t cs = (cudaStream_t)stream;
-    // steps 1-2
-    if (a->ev_stats_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_begin, cs));
-    rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
-                    col_part, st, stream);
-    if (rc != AWEQ_OK) return rc;
-    if (a->ev_stats_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_end, cs));
+    const int kAllPhases = AWEQ_FLAG_PHASE_STATS | AWEQ_FLAG_PHASE_WEIGHTS | AWEQ_FLAG_PHASE_ACT;
+    const int phases = (a->flags & kAllPhases) ? (a->flags & kAllPhases) : kAllPhases;
+    // step 1
+    if (phases & AWEQ_FLAG_PHASE_STATS) {
+        if (a->ev_stats_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_begin, cs));
+        rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
+                        col_part, st, stream);
+        if (rc != AWEQ_OK) return rc;
+        if (a->ev_stats_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_end, cs));
+    }
+    const bool eq = !(a->flags & AWEQ_FLAG_NO_EQUALIZE);
+    // without equalisation the layer sees x itself, so E[x^] = E[x]
+    const float *s_used = eq ? a->s : nullptr;
+    const float *rinv_used = eq ? a->rinv : nullptr;
+    const float *mu_used = eq ? a->mu_hat : a->xmean;
+    if (phases & AWEQ_FLAG_PHASE_WEIGHTS) {
+    // step 2
     for (int i = 0; i < a->n_w; ++i) {
         rc = aweq_wrange(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], a->wmin, a->wmax, i > 0, ws_col, col_part,
                          st, stream);
@@ -328,11 +339,6 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     rc = aweq_factors(a->xmin, a->xmax, a->xmean, a->wmin, a->wmax, a->C_in, a->s, a->rinv, a->mu_hat, a->pX, a->pW,
                       a->scalars, st, stream);
     if (rc != AWEQ_OK) return rc;
-    const bool eq = !(a->flags & AWEQ_FLAG_NO_EQUALIZE);
-    // without equalisation the layer sees x itself, so E[x^] = E[x]
-    const float *s_used = eq ? a->s : nullptr;
-    const float *rinv_used = eq ? a->rinv : nullptr;
-    const float *mu_used = eq ? a->mu_hat : a->xmean;
     // steps 4-5 per matrix: the corrected bias is written by the quantiser itself
     for (int i = 0; i < a->n_w; ++i) {
         float *em = bc ? a->epsmu[i] : nullptr;
@@ -347,8 +353,9 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
                                     ws_eq_bytes, st, stream);
         if (rc != AWEQ_OK) return rc;
     }
+    }
     // step 6
-    if (a->Xq) {
+    if (a->Xq && (phases & AWEQ_FLAG_PHASE_ACT)) {
         if (a->ev_act_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_act_begin, cs));
         rc = aweq_quant_act(a->X, a->dt, a->N, a->C_in, a->ldx, rinv_used, a->act_bits ? a->act_bits : 8, AWEQ_PER_ROW,
                             nullptr, a->Xq, a->act_step, a->act_zp, st, stream);
