@@ -99,9 +99,6 @@ class LayerCalibrator:
             self._fork = torch.cuda.Event()
             self._ev_stats = [torch.cuda.Event() for _ in self.passes]
             self._ev_weights = [torch.cuda.Event() for _ in self.passes]
-            names = [i.name for i in wl.inputs if i.name in self.out]
-            volume = [sum(l.c_out * l.c_in for l in wl.linears if l.input == nm) for nm in names]
-            self._overlap_order = sorted(range(len(names)), key=lambda i: -volume[i])
         self._fc_ws, self._fc_out = None, {}
         self.equalized = not (flags & aweq.FLAG_NO_EQUALIZE)
 
@@ -117,26 +114,21 @@ class LayerCalibrator:
         self._fork.record(cur)
         big.wait_event(self._fork)
         small.wait_event(self._fork)
-        # the last input's weight kernels have no sweep to hide under: take the inputs in order of
-        # decreasing weight volume (the passes are independent of one another)
-        order = self._overlap_order
-        n = len(order)
+        n = len(self.passes)
 
-        def stats(k):
-            i = order[k]
+        def stats(i):
             with torch.cuda.stream(big):
                 self.passes[i](ws_big, self.status, aweq.FLAG_PHASE_STATS)
                 self._ev_stats[i].record(big)
 
         stats(0)
-        for k, i in enumerate(order):
-            lp = self.passes[i]
+        for i, lp in enumerate(self.passes):
             with torch.cuda.stream(small):
                 small.wait_event(self._ev_stats[i])
                 lp(ws_small, self.status, aweq.FLAG_PHASE_WEIGHTS)
                 self._ev_weights[i].record(small)
-            if k + 1 < n:
-                stats(k + 1)                       # the next sweep goes ahead of this input's step 6
+            if i + 1 < n:
+                stats(i + 1)                       # the next sweep goes ahead of this input's step 6
             if self.wl.act_quant:
                 with torch.cuda.stream(big):
                     big.wait_event(self._ev_weights[i])
