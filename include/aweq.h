@@ -256,13 +256,14 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
 #define AWEQ_FLAG_NO_BIAS_CORRECT 2  /* skip step 5 */
 /* Run only part of the pass (any combination; none of the three = the whole pass).  The parts
  * communicate through the per-channel arrays of the argument block, so a caller can put them
- * on different streams -- the HBM-bound sweeps over X on one, the short weight kernels on
- * another -- ordering them with its own events and giving each stream its own `ws`:
- *   STATS   step 1 (writes xmin, xmax, xmean)
- *   WEIGHTS steps 2-5 (reads them; writes wmin, wmax, s, rinv, mu_hat, codes, Step, Z, biases)
+ * on different streams -- the shared-memory-staged, HBM-bound sweeps on one, the short
+ * issue-bound weight kernels on another, where they fit beside a running sweep -- ordering
+ * them with its own events and giving each stream its own `ws`:
+ *   REDUCE  steps 1-2 (column reductions: writes xmin, xmax, xmean, wmin, wmax)
+ *   QUANT   steps 3-5 (reads them; writes s, rinv, mu_hat, codes, Step, Z, biases)
  *   ACT     step 6 (reads rinv; writes Xq, act_step, act_zp) */
-#define AWEQ_FLAG_PHASE_STATS 4
-#define AWEQ_FLAG_PHASE_WEIGHTS 8
+#define AWEQ_FLAG_PHASE_REDUCE 4
+#define AWEQ_FLAG_PHASE_QUANT 8
 #define AWEQ_FLAG_PHASE_ACT 16
 
 typedef struct {

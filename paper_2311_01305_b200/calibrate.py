@@ -39,11 +39,12 @@ class LayerCalibrator:
     def __init__(self, wl: synth.Workload, bits: int, X: Dict[str, torch.Tensor], W: Dict[str, torch.Tensor],
                  bias: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0, diagnostics: bool = True,
                  overlap: bool = False):
-        """``overlap``: split every pass into its parts (``FLAG_PHASE_*``) and issue the HBM-bound
-        sweeps over X (steps 1 and 6) on one CUDA stream and the short, issue-bound weight
-        kernels (steps 2-5) on another, each with its own scratch and ordered by events, so that
-        the weight kernels of one input run under the statistics sweep of the next; ``run()``
-        forks from and joins back into the current stream."""
+        """``overlap``: split every pass into its parts (``FLAG_PHASE_*``) and issue the
+        shared-memory-staged, HBM-bound kernels (the column reductions of steps 1-2 and step 6) on
+        one CUDA stream and the short, issue-bound kernels that need no shared memory (factors,
+        weight quantiser: steps 3-5) on another, each with its own scratch and ordered by events,
+        so that the weight kernels of one input run beside the statistics sweep of the next;
+        ``run()`` forks from and joins back into the current stream."""
         self.wl, self.bits = wl, bits
         dev = next(iter(X.values())).device
         td = synth.torch_dtype(wl.dtype)
@@ -118,14 +119,14 @@ class LayerCalibrator:
 
         def stats(i):
             with torch.cuda.stream(big):
-                self.passes[i](ws_big, self.status, aweq.FLAG_PHASE_STATS)
+                self.passes[i](ws_big, self.status, aweq.FLAG_PHASE_REDUCE)
                 self._ev_stats[i].record(big)
 
         stats(0)
         for i, lp in enumerate(self.passes):
             with torch.cuda.stream(small):
                 small.wait_event(self._ev_stats[i])
-                lp(ws_small, self.status, aweq.FLAG_PHASE_WEIGHTS)
+                lp(ws_small, self.status, aweq.FLAG_PHASE_QUANT)
                 self._ev_weights[i].record(small)
             if i + 1 < n:
                 stats(i + 1)                       # the next sweep goes ahead of this input's step 6

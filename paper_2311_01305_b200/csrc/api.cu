@@ -313,28 +313,27 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     const size_t ws_eq_bytes = need - col_part;
 
     cudaStream_t cs = (cudaStream_t)stream;
-    const int kAllPhases = AWEQ_FLAG_PHASE_STATS | AWEQ_FLAG_PHASE_WEIGHTS | AWEQ_FLAG_PHASE_ACT;
+    const int kAllPhases = AWEQ_FLAG_PHASE_REDUCE | AWEQ_FLAG_PHASE_QUANT | AWEQ_FLAG_PHASE_ACT;
     const int phases = (a->flags & kAllPhases) ? (a->flags & kAllPhases) : kAllPhases;
-    // step 1
-    if (phases & AWEQ_FLAG_PHASE_STATS) {
+    // steps 1-2
+    if (phases & AWEQ_FLAG_PHASE_REDUCE) {
         if (a->ev_stats_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_begin, cs));
         rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
                         col_part, st, stream);
         if (rc != AWEQ_OK) return rc;
         if (a->ev_stats_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_end, cs));
+        for (int i = 0; i < a->n_w; ++i) {
+            rc = aweq_wrange(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], a->wmin, a->wmax, i > 0, ws_col, col_part,
+                             st, stream);
+            if (rc != AWEQ_OK) return rc;
+        }
     }
     const bool eq = !(a->flags & AWEQ_FLAG_NO_EQUALIZE);
     // without equalisation the layer sees x itself, so E[x^] = E[x]
     const float *s_used = eq ? a->s : nullptr;
     const float *rinv_used = eq ? a->rinv : nullptr;
     const float *mu_used = eq ? a->mu_hat : a->xmean;
-    if (phases & AWEQ_FLAG_PHASE_WEIGHTS) {
-    // step 2
-    for (int i = 0; i < a->n_w; ++i) {
-        rc = aweq_wrange(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], a->wmin, a->wmax, i > 0, ws_col, col_part,
-                         st, stream);
-        if (rc != AWEQ_OK) return rc;
-    }
+    if (phases & AWEQ_FLAG_PHASE_QUANT) {
     // step 3
     rc = aweq_factors(a->xmin, a->xmax, a->xmean, a->wmin, a->wmax, a->C_in, a->s, a->rinv, a->mu_hat, a->pX, a->pW,
                       a->scalars, st, stream);

@@ -133,8 +133,8 @@ def test_sharded_path_with_one_rank_equals_fused_layer_pass():
 
 @pytest.mark.parametrize("name,scale,bits", [("opt125m_model_w8a8", 1.0 / 64, 8), ("llama7b_layer_w4w3_g128", 1.0 / 256, 4)])
 def test_two_stream_schedule_equals_single_stream(name, scale, bits):
-    """The pass split into its parts (statistics and step 6 on one stream, the weight kernels on
-    another, ordered by events) writes exactly what the single-stream pass writes, run after run."""
+    """The pass split into its parts (column reductions and step 6 on one stream, factors and the
+    weight quantiser on another, ordered by events) writes exactly what the single-stream pass writes, run after run."""
     from paper_2311_01305_b200 import aweq, calibrate
     wl = synth.workloads(n_tokens_scale=scale)[name]
     Xc, Wc = make_workload_tensors(wl, offset=1.0)
@@ -154,10 +154,10 @@ def test_two_stream_schedule_equals_single_stream(name, scale, bits):
     for nm, outs in a.out.items():
         for k, v in outs.items():
             assert torch.equal(v.view(torch.uint8), b.out[nm][k].view(torch.uint8)), (nm, k)
-    # a single part on its own: the statistics phase leaves the other outputs alone
+    # a single part on its own: the reduction phase leaves the other outputs alone
     lp = b.passes[0]
     first = wl.inputs[0].name
     b.out[first]["s"].fill_(-1.0)
-    lp(b.ws, b.status, aweq.FLAG_PHASE_STATS)
+    lp(b.ws, b.status, aweq.FLAG_PHASE_REDUCE)
     torch.cuda.synchronize()
     assert bool((b.out[first]["s"] == -1.0).all()) and torch.equal(b.out[first]["xmin"], a.out[first]["xmin"])
