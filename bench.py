@@ -368,7 +368,9 @@ def main():
         "config": {"workload": wl.name, "w_bits": bits, "w_gran": wl.w_gran, "group": wl.group,
                    "act_quant": wl.act_quant, "storage": wl.dtype, "tokens_per_gpu": tokens,
                    "algorithmic_bytes_per_gpu": nbytes, "cache": "inputs (GBs) far larger than the 126 MB L2",
-                   "parallelism": "token shards, one per GPU" if world > 1 else "single GPU"},
+                   "parallelism": "token shards, one per GPU" if world > 1 else "single GPU",
+                   "schedule": ("two streams: column reductions and step 6 on one, factors and weight quantiser on the other"
+                                if getattr(cal, "overlap", False) else "one stream")},
         "tokens_per_s": world * tokens / (ms / 1e3),
         "pct_of_8000_gbs": 100.0 * gbs / world / NOMINAL_HBM_GBS,
         "pct_of_measured_copy": 100.0 * gbs / world / peak,
