@@ -137,6 +137,21 @@ class LayerCalibrator:
         cur.wait_stream(big)
         cur.wait_stream(small)
 
+    def capture(self) -> "torch.cuda.CUDAGraph":
+        """Record one ``run()`` (both streams and their events when ``overlap`` is on) into a CUDA
+        graph; ``graph.replay()`` then re-issues the whole pass with one launch.  The library's
+        calls are capture-safe (no allocation, no synchronisation); the profiling event hooks of
+        ``LayerPass.set_events`` must be unset, and one ordinary ``run()`` must have happened before
+        (it sets the kernels' shared-memory attributes outside the capture)."""
+        for lp in self.passes:
+            lp.set_events(None, None)
+        self.run()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run()
+        return graph
+
     def forward_check(self, X, W, bias=None, corrected: bool = True):
         """The forward check of every linear after ``run()``: {linear name: (mean_err[C_out],
         sums[4])} as binary64 device tensors.  W8A8 workloads with row-wise 8-bit weights go

@@ -161,3 +161,30 @@ def test_two_stream_schedule_equals_single_stream(name, scale, bits):
     lp(b.ws, b.status, aweq.FLAG_PHASE_REDUCE)
     torch.cuda.synchronize()
     assert bool((b.out[first]["s"] == -1.0).all()) and torch.equal(b.out[first]["xmin"], a.out[first]["xmin"])
+
+
+@pytest.mark.parametrize("overlap", [False, True])
+def test_graph_replay_equals_eager(overlap):
+    """One pass captured into a CUDA graph (with both streams when the two-stream schedule is on)
+    writes, on replay, exactly what the eager pass writes."""
+    from paper_2311_01305_b200 import aweq, calibrate
+    wl = synth.workloads(n_tokens_scale=1.0 / 64)["opt125m_model_w8a8"]
+    Xc, Wc = make_workload_tensors(wl, offset=1.0)
+    Xd = {k: v.to(DEV) for k, v in Xc.items()}
+    Wd = {k: v.to(DEV) for k, v in Wc.items()}
+    a = calibrate.LayerCalibrator(wl, 8, Xd, Wd, None)
+    b = calibrate.LayerCalibrator(wl, 8, Xd, Wd, None, overlap=overlap)
+    a.run()
+    graph = b.capture()
+    n0 = aweq.launch_count()
+    for _ in range(2):
+        for outs in b.out.values():
+            for v in outs.values():
+                v.view(torch.uint8).fill_(0x5A)
+        graph.replay()
+    torch.cuda.synchronize()
+    assert aweq.launch_count() == n0                      # replays go through no library call
+    assert aweq.read_status(b.status)["wait_timeout"] == 0
+    for nm, outs in a.out.items():
+        for k, v in outs.items():
+            assert torch.equal(v.view(torch.uint8), b.out[nm][k].view(torch.uint8)), (nm, k)
