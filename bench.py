@@ -191,6 +191,16 @@ def run_forward_check(args, wl, bits):
     torch.cuda.synchronize()
     launches = aweq.launch_count() - n0
     clocks = sampler.stop()
+    if graph is not None:
+        # the kernels of a replay are the ones one eager pass launches; time the dominant one eagerly
+        torch.cuda.synchronize()
+        n1 = aweq.launch_count()
+        for k in range(args.steps):
+            for lp, (es, ea) in zip(cal.passes, hooks[k]):
+                lp.set_events(es, ea)
+            cal.run()
+        torch.cuda.synchronize()
+        launches = aweq.launch_count() - n1
     ms = a.elapsed_time(b) / args.steps
     tokens = {i.name: i.n_tokens for i in wl.inputs}
     flops = sum(4.0 * tokens[l.input] * l.c_in * l.c_out for l in wl.linears)
@@ -254,6 +264,9 @@ def main():
     ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
     ap.add_argument("--no-overlap", action="store_true",
                     help="issue every input's pass on one stream (default: two alternating streams)")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the pass as one CUDA graph in the timed region (1 GPU; the dominant kernel is then "
+                         "timed in separate eager steps, because event hooks cannot be read back from a graph)")
     ap.add_argument("--op", default="layer_pass", choices=["layer_pass", "forward_check"],
                     help="forward_check: time the W8A8 forward check of the calibrated layer instead (1 GPU)")
     args = ap.parse_args()
@@ -300,6 +313,11 @@ def main():
 
     for _ in range(args.warmup):
         cal.run()
+    graph = None
+    if args.graph and world == 1:
+        graph = cal.capture()
+        for _ in range(args.warmup):
+            graph.replay()
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
@@ -313,6 +331,8 @@ def main():
             names = [i.name for i in wl.inputs if i.name in cal.out]
             cal.events = {n: h for n, h in zip(names, hooks[k])}
             cal.run()                       # statistics merged over the ranks inside the step
+        elif graph is not None:
+            graph.replay()
         else:
             for lp, (es, ea) in zip(cal.passes, hooks[k]):
                 lp.set_events(es, ea)
@@ -321,6 +341,16 @@ def main():
     barrier()
     launches = aweq.launch_count() - n0
     clocks = sampler.stop()
+    if graph is not None:
+        # the kernels of a replay are the ones one eager pass launches; time the dominant one eagerly
+        torch.cuda.synchronize()
+        n1 = aweq.launch_count()
+        for k in range(args.steps):
+            for lp, (es, ea) in zip(cal.passes, hooks[k]):
+                lp.set_events(es, ea)
+            cal.run()
+        torch.cuda.synchronize()
+        launches = aweq.launch_count() - n1
     for lp in cal.passes:
         lp.set_events(None, None)
     if world > 1:
@@ -369,6 +399,7 @@ def main():
                    "act_quant": wl.act_quant, "storage": wl.dtype, "tokens_per_gpu": tokens,
                    "algorithmic_bytes_per_gpu": nbytes, "cache": "inputs (GBs) far larger than the 126 MB L2",
                    "parallelism": "token shards, one per GPU" if world > 1 else "single GPU",
+                   "launch": "one CUDA graph replay per step" if graph is not None else "eager",
                    "schedule": ("two streams: column reductions and step 6 on one, factors and weight quantiser on the other"
                                 if getattr(cal, "overlap", False) else "one stream")},
         "tokens_per_s": world * tokens / (ms / 1e3),
