@@ -265,9 +265,6 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
 #define AWEQ_FLAG_PHASE_REDUCE 4
 #define AWEQ_FLAG_PHASE_QUANT 8
 #define AWEQ_FLAG_PHASE_ACT 16
-/* Launch the group-wise weight quantiser of steps 4-5 with one CTA per SM: slower on its own,
- * but it then takes few issue slots from a sweep it runs beside on another stream. */
-#define AWEQ_FLAG_BACKGROUND 32
 
 typedef struct {
     /* input */

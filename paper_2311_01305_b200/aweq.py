@@ -30,7 +30,6 @@ PER_TENSOR, PER_ROW, PER_GROUP = 0, 1, 2
 OP_STATS, OP_WRANGE, OP_EQUALIZE_QUANTIZE, OP_BIAS_CORRECT, OP_QUANT_ACT = 1, 2, 4, 5, 6
 FLAG_NO_EQUALIZE, FLAG_NO_BIAS_CORRECT = 1, 2
 FLAG_PHASE_REDUCE, FLAG_PHASE_QUANT, FLAG_PHASE_ACT = 4, 8, 16
-FLAG_BACKGROUND = 32
 
 _vp, _ll, _i, _sz = ctypes.c_void_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_size_t
 
@@ -315,7 +314,7 @@ class LayerPass:
 
     def __call__(self, ws: torch.Tensor, st: Optional[torch.Tensor] = None, phases: int = 0) -> None:
         """``phases``: 0 = the whole pass, or a mask of ``FLAG_PHASE_*`` (see ``include/aweq.h``)."""
-        base = self.args.flags & ~(FLAG_PHASE_REDUCE | FLAG_PHASE_QUANT | FLAG_PHASE_ACT | FLAG_BACKGROUND)
+        base = self.args.flags & ~(FLAG_PHASE_REDUCE | FLAG_PHASE_QUANT | FLAG_PHASE_ACT)
         self.args.flags = base | phases
         try:
             _check(_lib.aweq_layer_pass(ctypes.byref(self.args), _ptr(ws), ws.numel(), _ptr(st), _stream()))

@@ -38,7 +38,7 @@ def algorithmic_bytes(wl: synth.Workload, bits: int) -> int:
 class LayerCalibrator:
     def __init__(self, wl: synth.Workload, bits: int, X: Dict[str, torch.Tensor], W: Dict[str, torch.Tensor],
                  bias: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0, diagnostics: bool = True,
-                 overlap: bool = False, background: bool = True):
+                 overlap: bool = False):
         """``overlap``: split every pass into its parts (``FLAG_PHASE_*``) and issue the
         shared-memory-staged, HBM-bound kernels (the column reductions of steps 1-2 and step 6) on
         one CUDA stream and the short, issue-bound kernels that need no shared memory (factors,
@@ -98,7 +98,6 @@ class LayerCalibrator:
             self._streams = (torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev))
             self._ws2 = (self.ws, aweq.workspace(ws_bytes, dev))
             self._fork = torch.cuda.Event()
-            self._quant_extra = aweq.FLAG_BACKGROUND if background else 0
             self._ev_stats = [torch.cuda.Event() for _ in self.passes]
             self._ev_weights = [torch.cuda.Event() for _ in self.passes]
         self._fc_ws, self._fc_out = None, {}
@@ -127,7 +126,7 @@ class LayerCalibrator:
         for i, lp in enumerate(self.passes):
             with torch.cuda.stream(small):
                 small.wait_event(self._ev_stats[i])
-                lp(ws_small, self.status, aweq.FLAG_PHASE_QUANT | self._quant_extra)
+                lp(ws_small, self.status, aweq.FLAG_PHASE_QUANT)
                 self._ev_weights[i].record(small)
             if i + 1 < n:
                 stats(i + 1)                       # the next sweep goes ahead of this input's step 6

@@ -169,7 +169,7 @@ static aweq_status equalize_quantize_impl(const void *W, aweq_dtype dt, long lon
                                           long long ldw, const float *s, const float *mu_hat, int bits,
                                           aweq_gran gran, int group, unsigned char *codes, float *step, int *zp,
                                           float *epsmu, const BiasIO &bias, void *ws, size_t ws_bytes,
-                                          aweq_dev_status *st, void *stream, int background = 0)
+                                          aweq_dev_status *st, void *stream)
 {
     aweq_status rc = check_matrix(W, dt, C_out, C_in, ldw, false);
     if (rc != AWEQ_OK) return rc;
@@ -188,7 +188,7 @@ static aweq_status equalize_quantize_impl(const void *W, aweq_dtype dt, long lon
     }
     if (gran == AWEQ_PER_GROUP)
         return run_warpquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, group, nullptr, codes, step, zp, epsmu,
-                             bias, st, cs, background);
+                             bias, st, cs);
     // per tensor: column extremes of W -> extremes of diag(s) W -> static-range quantiser
     char *base = reinterpret_cast<char *>(ws);
     float *cmin = reinterpret_cast<float *>(base);
@@ -349,7 +349,7 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
         }
         rc = equalize_quantize_impl(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], s_used, bc ? mu_used : nullptr,
                                     a->bits, a->gran, a->group, a->codes[i], a->step[i], a->zp[i], em, bias, ws_eq,
-                                    ws_eq_bytes, st, stream, (a->flags & AWEQ_FLAG_BACKGROUND) ? 1 : 0);
+                                    ws_eq_bytes, st, stream);
         if (rc != AWEQ_OK) return rc;
     }
     }

@@ -42,7 +42,6 @@ struct WarpQuantParams {
     int ngroups;                // groups per row (group mode)
     const float *lo_hi;         // static mode: device float[2]
     aweq_dev_status *st;
-    int background;             // launch one CTA per SM only
 };
 
 constexpr int kWqWarps = 8;
@@ -272,9 +271,7 @@ template <class D, int BITS, bool STATIC, bool MU, bool BYTES_OUT>
 static aweq_status launch_wq(const WarpQuantParams &p, cudaStream_t stream)
 {
     long long blocks = (p.nrows + kWqWarps - 1) / kWqWarps;
-    // a few waves; warps stride over the rows beyond that.  Background mode: one CTA per SM, so that
-    // the kernel takes few issue slots from whatever it runs beside
-    const long long cap = p.background ? (long long)kSmCount : (long long)kSmCount * 8 * 4;
+    const long long cap = (long long)kSmCount * 8 * 4;      // a few waves; warps stride over the rows beyond that
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     AWEQ_LAUNCH((warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT>), dim3((unsigned)blocks), dim3(kWqWarps * 32), 0,
@@ -297,10 +294,9 @@ static aweq_status launch_wq_bits(const WarpQuantParams &p, cudaStream_t stream)
 aweq_status run_warpquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
                           const float *scale, const float *mu, int bits, bool weights, int group,
                           const float *lo_hi, unsigned char *out, float *step, int *zp, float *epsmu,
-                          const BiasIO &bias, aweq_dev_status *st, cudaStream_t stream, int background)
+                          const BiasIO &bias, aweq_dev_status *st, cudaStream_t stream)
 {
     WarpQuantParams p;
-    p.background = background;
     p.X = reinterpret_cast<const uint16_t *>(X);
     p.nrows = nrows; p.ld = ld; p.nvec = (int)(cols / 8);
     p.scale = scale; p.mu = mu; p.out = out;
