@@ -95,7 +95,8 @@ __device__ __forceinline__ void store_vec(unsigned char *orow, int idx, const ui
     }
 }
 
-template <class D, int BITS, bool STATIC, bool MU, bool BYTES_OUT>
+// FULL: the row is a whole number of 32-vector steps, so no lane is ever past its end.
+template <class D, int BITS, bool STATIC, bool MU, bool BYTES_OUT, bool FULL>
 __global__ void __launch_bounds__(kWqWarps * 32, 4)
 warpquant_kernel(const WarpQuantParams p)
 {
@@ -129,10 +130,12 @@ warpquant_kernel(const WarpQuantParams p)
         float *step_row = STATIC ? p.step : p.step + row * p.ngroups;
         int *zp_row = STATIC ? p.zp : p.zp + row * p.ngroups;
         float2 eneg = make_float2(0.0f, 0.0f);                 // minus the running eps . mu sum
-        uint4 nxt = lane < p.nvec ? ldg_stream(xrow + (size_t)lane * 8) : make_uint4(0, 0, 0, 0);
+        uint4 nxt = (FULL || lane < p.nvec) ? ldg_stream(xrow + (size_t)lane * 8) : make_uint4(0, 0, 0, 0);
+        float buf_step = 0.0f;                                 // (Step, Z) of the group whose index in the current
+        int buf_zp = 0;                                        // window of 32 groups is this lane
         for (int it = 0; it < nsteps; ++it) {
             const int idx = it * 32 + lane;
-            const bool active = idx < p.nvec;
+            const bool active = FULL || idx < p.nvec;
             float w[8];
             widen8<D>(nxt, w);
             nxt = idx + 32 < p.nvec ? ldg_stream(xrow + (size_t)(idx + 32) * 8) : make_uint4(0, 0, 0, 0);
@@ -165,15 +168,41 @@ warpquant_kernel(const WarpQuantParams p)
                 a = fminf(fminf(a, w2[1].y), w2[2].x); b = fmaxf(fmaxf(b, w2[1].y), w2[2].x);
                 a = fminf(fminf(a, w2[2].y), w2[3].x); b = fmaxf(fmaxf(b, w2[2].y), w2[3].x);
                 a = fminf(a, w2[3].y); b = fmaxf(b, w2[3].y);
-                if (L > 1) {
+                if (L == 16) {
+                    // two groups per warp: a full-mask reduction per group with the other half's lanes
+                    // neutral costs a third of what one reduction over a 16-lane sub-mask does (the two
+                    // halves name different masks, which the hardware does not take in one go)
+                    const bool upper = lane >= 16;
+                    const float a0 = redux_min(upper ? INFINITY : a, 0xffffffffu);
+                    const float a1 = redux_min(upper ? a : INFINITY, 0xffffffffu);
+                    const float b0 = redux_max(upper ? -INFINITY : b, 0xffffffffu);
+                    const float b1 = redux_max(upper ? b : -INFINITY, 0xffffffffu);
+                    a = upper ? a1 : a0;
+                    b = upper ? b1 : b0;
+                } else if (L > 1) {
                     a = redux_min(a, gmask);
                     b = redux_max(b, gmask);
                 }
                 q = make_qparams(a, b, qmax);
                 fl = qflags(q, b, qmax);
-                if (active && (lane & (L - 1)) == 0) {
-                    step_row[idx >> p.log2_lanes] = q.step;
-                    zp_row[idx >> p.log2_lanes] = q.zp;
+                // (Step, Z) pairs are collected in registers -- lane l keeps group l of the current window
+                // of 32 groups, fetched from the first lane of that group in the step that formed it --
+                // and leave as one coalesced store per window instead of a scattered one per step
+                const int gps = 32 >> p.log2_lanes;                       // groups per step
+                const int wpos = it & (L - 1);                            // step within the window (L steps)
+                const int src = (lane & (gps - 1)) << p.log2_lanes;       // first lane of "my" group in its step
+                const float sh_step = __shfl_sync(0xffffffffu, q.step, src);
+                const int sh_zp = __shfl_sync(0xffffffffu, q.zp, src);
+                if ((lane >> (5 - p.log2_lanes)) == wpos) {
+                    buf_step = sh_step;
+                    buf_zp = sh_zp;
+                }
+                if (wpos == L - 1 || it == nsteps - 1) {
+                    const int g0 = (it - wpos) * gps;                     // first group of the window
+                    if (g0 + lane < p.ngroups) {
+                        step_row[g0 + lane] = buf_step;
+                        zp_row[g0 + lane] = buf_zp;
+                    }
                 }
             }
             const bool all_lean = __all_sync(0xffffffffu, !active || fl == (kQFast | kQNoClamp));
@@ -274,8 +303,12 @@ static aweq_status launch_wq(const WarpQuantParams &p, cudaStream_t stream)
     const long long cap = (long long)kSmCount * 8 * 4;      // a few waves; warps stride over the rows beyond that
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    AWEQ_LAUNCH((warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT>), dim3((unsigned)blocks), dim3(kWqWarps * 32), 0,
-                stream, p);
+    if (p.nvec % 32 == 0)
+        AWEQ_LAUNCH((warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT, true>), dim3((unsigned)blocks), dim3(kWqWarps * 32),
+                    0, stream, p);
+    else
+        AWEQ_LAUNCH((warpquant_kernel<D, BITS, STATIC, MU, BYTES_OUT, false>), dim3((unsigned)blocks),
+                    dim3(kWqWarps * 32), 0, stream, p);
     return AWEQ_OK;
 }
 
