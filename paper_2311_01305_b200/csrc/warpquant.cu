@@ -169,13 +169,16 @@ warpquant_kernel(const WarpQuantParams p)
                 a = fminf(fminf(a, w2[2].y), w2[3].x); b = fmaxf(fmaxf(b, w2[2].y), w2[3].x);
                 a = fminf(a, w2[3].y); b = fmaxf(b, w2[3].y);
                 if (L == 16) {
-                    // two groups per warp: a shuffle butterfly inside each half (a reduction instruction over
-                    // a 16-lane sub-mask costs about twice as much: the halves name different masks)
-#pragma unroll
-                    for (int o = 8; o > 0; o >>= 1) {
-                        a = fminf(a, __shfl_xor_sync(0xffffffffu, a, o));
-                        b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, o));
-                    }
+                    // two groups per warp: a full-mask reduction per group with the other half's lanes
+                    // neutral costs a third of what one reduction over a 16-lane sub-mask does (the two
+                    // halves name different masks, which the hardware does not take in one go)
+                    const bool upper = lane >= 16;
+                    const float a0 = redux_min(upper ? INFINITY : a, 0xffffffffu);
+                    const float a1 = redux_min(upper ? a : INFINITY, 0xffffffffu);
+                    const float b0 = redux_max(upper ? -INFINITY : b, 0xffffffffu);
+                    const float b1 = redux_max(upper ? b : -INFINITY, 0xffffffffu);
+                    a = upper ? a1 : a0;
+                    b = upper ? b1 : b0;
                 } else if (L > 1) {
                     a = redux_min(a, gmask);
                     b = redux_max(b, gmask);
