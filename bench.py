@@ -217,14 +217,18 @@ def run_forward_check(args, wl, bits):
     # ablation (outside the timed region): equalisation and bias correction switched on and off
     del cal
     ablation = {}
-    for eq in (True, False):
+    for eq in (True, "absmax", False):
         for bc in (True, False):
+            if eq == "absmax" and not bc:
+                continue
             flags = (0 if eq else aweq.FLAG_NO_EQUALIZE) | (0 if bc else aweq.FLAG_NO_BIAS_CORRECT)
+            flags |= aweq.FLAG_ABSMAX_CRITERION if eq == "absmax" else 0
             c = calibrate.LayerCalibrator(wl, bits, X, W, None, flags=flags)
             c.run()
             r = c.forward_check(X, W, corrected=bc)
             torch.cuda.synchronize()
-            ablation[("AWE" if eq else "no AWE") + (" + BC" if bc else "")] = {
+            name = "abs-max criterion" if eq == "absmax" else ("AWE" if eq else "no AWE")
+            ablation[name + (" + BC" if bc else "")] = {
                 "output_sqnr_db": {n: round(float(10.0 * torch.log10(s4[1] / s4[0]).item()), 3)
                                    for n, (me, s4) in r.items()},
                 "rms_mean_err_over_output_rms": {n: float(((s4[2] / me.numel()) / (s4[1] / s4[3])).sqrt().item())

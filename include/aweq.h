@@ -186,6 +186,20 @@ aweq_status aweq_factors(const float *xmin, const float *xmax, const float *xmea
                          aweq_dev_status *st, void *stream);
 
 /*
+ * Step 3 with the criterion AWEQ argues against, for comparison.  Section 3.1 starts from the
+ * per-channel equalisation that balances the LARGEST MAGNITUDES of activations and weights;
+ * the paper's point is that balancing the channel RANGES (Eq. 4-10) does better.  This entry
+ * feeds Eq. 10 with max|x_j| and max|w_j| instead of the ranges,
+ *   s_j = (1 / max|w_j|) sqrt(max|x_j| max|w_j|)   ( = sqrt(max|x_j| / max|w_j|) ),
+ * everything else (rinv, mu_hat, the range-based diagnostics, dead channels, rounding) as in
+ * aweq_factors, so that the two criteria can be put through the same quantiser and forward check.
+ */
+aweq_status aweq_factors_absmax(const float *xmin, const float *xmax, const float *xmean,
+                                const float *wmin, const float *wmax, long long C_in,
+                                float *s, float *rinv, float *mu_hat, float *pX, float *pW, double *scalars,
+                                aweq_dev_status *st, void *stream);
+
+/*
  * Step 4 -- fold s into W and quantise (Eq. 3: W^ = diag(s) W, so input
  * channel j of every row is multiplied by s_j; Eq. 1-2 on every row or group).
  * One pass over W: rescale, range, quantise and pack are fused.
@@ -265,6 +279,7 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
 #define AWEQ_FLAG_PHASE_REDUCE 4
 #define AWEQ_FLAG_PHASE_QUANT 8
 #define AWEQ_FLAG_PHASE_ACT 16
+#define AWEQ_FLAG_ABSMAX_CRITERION 32   /* step 3 through aweq_factors_absmax (comparison criterion) */
 
 typedef struct {
     /* input */

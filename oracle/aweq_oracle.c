@@ -217,7 +217,7 @@ void oracle_wrange(const uint16_t *W, int dtype, int64_t C_out, int64_t C_in, in
 int64_t oracle_factors(const float *xmin, const float *xmax, const float *xmean,
                        const float *wmin, const float *wmax, int64_t C,
                        float *s, float *rinv, float *mu_hat, float *pX, float *pW,
-                       double *scalars)
+                       double *scalars, int criterion)
 {
     int64_t dead = 0;
     double gxlo = INFINITY, gxhi = -INFINITY, gwlo = INFINITY, gwhi = -INFINITY;
@@ -227,9 +227,13 @@ int64_t oracle_factors(const float *xmin, const float *xmax, const float *xmean,
         float rx = xmax[i] - xmin[i];
         float rw = wmax[i] - wmin[i];
         float si = 1.0f;
-        int ok = isfinite(rx) && isfinite(rw) && rx > 0.0f && rw > 0.0f;
+        /* criterion 0: the channel ranges (Eq. 4-10).  criterion 1, for comparison: the largest
+         * magnitudes, which is what the per-channel equalisation of Section 3.1 balances. */
+        float cx = criterion ? fmaxf(fabsf(xmin[i]), fabsf(xmax[i])) : rx;
+        float cw = criterion ? fmaxf(fabsf(wmin[i]), fabsf(wmax[i])) : rw;
+        int ok = isfinite(rx) && isfinite(rw) && cx > 0.0f && cw > 0.0f && isfinite(cx) && isfinite(cw);
         if (ok) {
-            double sd = (1.0 / (double)rw) * sqrt((double)rx * (double)rw);
+            double sd = (1.0 / (double)cw) * sqrt((double)cx * (double)cw);
             si = (float)sd;
             if (!(isfinite(si) && si > 0.0f) || !isfinite(1.0f / si)) {
                 si = 1.0f;

@@ -112,15 +112,19 @@ def wrange(W: np.ndarray, dtype: int, prev=None):
     return wmin, wmax
 
 
-def factors(xmin, xmax, xmean, wmin, wmax):
-    """Step 3 -> dict(s, rinv, mu_hat, pX, pW, scalars[8], dead)."""
+RANGE, ABSMAX = 0, 1
+
+
+def factors(xmin, xmax, xmean, wmin, wmax, criterion=RANGE):
+    """Step 3 -> dict(s, rinv, mu_hat, pX, pW, scalars[8], dead).  ``criterion``: RANGE is the paper's
+    (Eq. 4-10); ABSMAX feeds Eq. 10 with the largest magnitudes instead (the comparison criterion)."""
     xmin, xmax, xmean, wmin, wmax = map(_f32, (xmin, xmax, xmean, wmin, wmax))
     C = xmin.size
     out = {k: np.empty(C, np.float32) for k in ("s", "rinv", "mu_hat", "pX", "pW")}
     scalars = np.empty(8, np.float64)
     dead = _load().oracle_factors(_p(xmin), _p(xmax), _p(xmean), _p(wmin), _p(wmax), i64(C),
                                   _p(out["s"]), _p(out["rinv"]), _p(out["mu_hat"]), _p(out["pX"]),
-                                  _p(out["pW"]), _p(scalars))
+                                  _p(out["pW"]), _p(scalars), ci(criterion))
     out["scalars"] = scalars
     out["dead"] = int(dead)
     return out

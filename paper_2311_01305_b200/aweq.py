@@ -30,6 +30,7 @@ PER_TENSOR, PER_ROW, PER_GROUP = 0, 1, 2
 OP_STATS, OP_WRANGE, OP_EQUALIZE_QUANTIZE, OP_BIAS_CORRECT, OP_QUANT_ACT = 1, 2, 4, 5, 6
 FLAG_NO_EQUALIZE, FLAG_NO_BIAS_CORRECT = 1, 2
 FLAG_PHASE_REDUCE, FLAG_PHASE_QUANT, FLAG_PHASE_ACT = 4, 8, 16
+FLAG_ABSMAX_CRITERION = 32
 
 _vp, _ll, _i, _sz = ctypes.c_void_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_size_t
 
@@ -66,6 +67,8 @@ _lib.aweq_stats_static.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _vp, _vp, _
 _lib.aweq_stats_static.restype = _i
 _lib.aweq_wrange.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _i, _vp, _sz, _vp, _vp]
 _lib.aweq_factors.argtypes = [_vp, _vp, _vp, _vp, _vp, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.aweq_factors_absmax.argtypes = [_vp, _vp, _vp, _vp, _vp, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.aweq_factors_absmax.restype = _i
 _lib.aweq_equalize_quantize.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _sz,
                                         _vp, _vp]
 _lib.aweq_bias_correct.argtypes = [_vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _ll, _ll, _ll, _i, _i, _i, _vp, _vp, _vp,
@@ -185,6 +188,11 @@ def aweq_wrange(W, wmin, wmax, accumulate=False, ws=None, st=None):
 def aweq_factors(xmin, xmax, xmean, wmin, wmax, s, rinv, mu_hat, pX=None, pW=None, scalars=None, st=None):
     _check(_lib.aweq_factors(_ptr(xmin), _ptr(xmax), _ptr(xmean), _ptr(wmin), _ptr(wmax), xmin.numel(), _ptr(s),
                              _ptr(rinv), _ptr(mu_hat), _ptr(pX), _ptr(pW), _ptr(scalars), _ptr(st), _stream()))
+
+
+def aweq_factors_absmax(xmin, xmax, xmean, wmin, wmax, s, rinv, mu_hat, pX=None, pW=None, scalars=None, st=None):
+    _check(_lib.aweq_factors_absmax(_ptr(xmin), _ptr(xmax), _ptr(xmean), _ptr(wmin), _ptr(wmax), xmin.numel(), _ptr(s),
+                                    _ptr(rinv), _ptr(mu_hat), _ptr(pX), _ptr(pW), _ptr(scalars), _ptr(st), _stream()))
 
 
 def aweq_equalize_quantize(W, s, mu_hat, bits, gran, group, codes, step, zp, epsmu=None, ws=None, st=None):

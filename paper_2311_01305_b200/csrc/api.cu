@@ -165,6 +165,16 @@ aweq_status aweq_factors(const float *xmin, const float *xmax, const float *xmea
                        (cudaStream_t)stream);
 }
 
+aweq_status aweq_factors_absmax(const float *xmin, const float *xmax, const float *xmean, const float *wmin,
+                                const float *wmax, long long C_in, float *s, float *rinv, float *mu_hat, float *pX,
+                                float *pW, double *scalars, aweq_dev_status *st, void *stream)
+{
+    if (!xmin || !xmax || !xmean || !wmin || !wmax || !s || !rinv || !mu_hat) return AWEQ_ERR_NULL;
+    if (C_in <= 0 || C_in > (1ll << 20)) return AWEQ_ERR_SHAPE;
+    return run_factors(xmin, xmax, xmean, wmin, wmax, C_in, s, rinv, mu_hat, pX, pW, scalars, st,
+                       (cudaStream_t)stream, 1);
+}
+
 static aweq_status equalize_quantize_impl(const void *W, aweq_dtype dt, long long C_out, long long C_in,
                                           long long ldw, const float *s, const float *mu_hat, int bits,
                                           aweq_gran gran, int group, unsigned char *codes, float *step, int *zp,
@@ -335,8 +345,9 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     const float *mu_used = eq ? a->mu_hat : a->xmean;
     if (phases & AWEQ_FLAG_PHASE_QUANT) {
     // step 3
-    rc = aweq_factors(a->xmin, a->xmax, a->xmean, a->wmin, a->wmax, a->C_in, a->s, a->rinv, a->mu_hat, a->pX, a->pW,
-                      a->scalars, st, stream);
+    rc = ((a->flags & AWEQ_FLAG_ABSMAX_CRITERION) ? aweq_factors_absmax : aweq_factors)(
+        a->xmin, a->xmax, a->xmean, a->wmin, a->wmax, a->C_in, a->s, a->rinv, a->mu_hat, a->pX, a->pW, a->scalars, st,
+        stream);
     if (rc != AWEQ_OK) return rc;
     // steps 4-5 per matrix: the corrected bias is written by the quantiser itself
     for (int i = 0; i < a->n_w; ++i) {

@@ -33,14 +33,18 @@ struct FacOut {
 
 // one channel of pass 1: the factor, its reciprocal, E[x^], and the running extremes
 __device__ __forceinline__ FacOut fac_channel(float lo, float hi, float mean, float wl, float wh, FacRed &a,
-                                              unsigned int &dead)
+                                              unsigned int &dead, int criterion)
 {
     const float rx = __fsub_rn(hi, lo), rw = __fsub_rn(wh, wl);
+    // what Eq. 10 is fed: the channel ranges (the paper's criterion), or the largest magnitudes (the
+    // criterion of the per-channel equalisation it starts from, Section 3.1) for comparison
+    const float cx = criterion ? fmaxf(fabsf(lo), fabsf(hi)) : rx;
+    const float cw = criterion ? fmaxf(fabsf(wl), fabsf(wh)) : rw;
     float sj = 1.0f;
-    bool ok = isfinite(rx) && isfinite(rw) && rx > 0.0f && rw > 0.0f;
+    bool ok = isfinite(rx) && isfinite(rw) && cx > 0.0f && cw > 0.0f && isfinite(cx) && isfinite(cw);
     if (ok) {
         // Eq. 10 as printed, in binary64, rounded once to binary32
-        sj = (float)__dmul_rn(__ddiv_rn(1.0, (double)rw), __dsqrt_rn(__dmul_rn((double)rx, (double)rw)));
+        sj = (float)__dmul_rn(__ddiv_rn(1.0, (double)cw), __dsqrt_rn(__dmul_rn((double)cx, (double)cw)));
         if (!(isfinite(sj) && sj > 0.0f) || !isfinite(__fdiv_rn(1.0f, sj))) {
             sj = 1.0f;
             ok = false;
@@ -80,7 +84,7 @@ __global__ void __launch_bounds__(kFacThreads)
 factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, const float *__restrict__ xmean,
                const float *__restrict__ wmin, const float *__restrict__ wmax, int C, float *__restrict__ s,
                float *__restrict__ rinv, float *__restrict__ mu_hat, float *__restrict__ pX, float *__restrict__ pW,
-               double *__restrict__ scalars, aweq_dev_status *st)
+               double *__restrict__ scalars, aweq_dev_status *st, int criterion)
 {
     __shared__ FacRed red[kFacThreads / 32];
     __shared__ FacRed total;
@@ -106,16 +110,16 @@ factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, c
     for (int q = threadIdx.x; q < nquad; q += kFacThreads) {
         const float4 lo = ldg_f4(xmin + 4 * q), hi = ldg_f4(xmax + 4 * q), me = ldg_f4(xmean + 4 * q);
         const float4 wl = ldg_f4(wmin + 4 * q), wh = ldg_f4(wmax + 4 * q);
-        const FacOut o0 = fac_channel(lo.x, hi.x, me.x, wl.x, wh.x, a, dead);
-        const FacOut o1 = fac_channel(lo.y, hi.y, me.y, wl.y, wh.y, a, dead);
-        const FacOut o2 = fac_channel(lo.z, hi.z, me.z, wl.z, wh.z, a, dead);
-        const FacOut o3 = fac_channel(lo.w, hi.w, me.w, wl.w, wh.w, a, dead);
+        const FacOut o0 = fac_channel(lo.x, hi.x, me.x, wl.x, wh.x, a, dead, criterion);
+        const FacOut o1 = fac_channel(lo.y, hi.y, me.y, wl.y, wh.y, a, dead, criterion);
+        const FacOut o2 = fac_channel(lo.z, hi.z, me.z, wl.z, wh.z, a, dead, criterion);
+        const FacOut o3 = fac_channel(lo.w, hi.w, me.w, wl.w, wh.w, a, dead, criterion);
         *reinterpret_cast<float4 *>(s + 4 * q) = make_float4(o0.s, o1.s, o2.s, o3.s);
         *reinterpret_cast<float4 *>(rinv + 4 * q) = make_float4(o0.rinv, o1.rinv, o2.rinv, o3.rinv);
         *reinterpret_cast<float4 *>(mu_hat + 4 * q) = make_float4(o0.mu, o1.mu, o2.mu, o3.mu);
     }
     for (int j = 4 * nquad + threadIdx.x; j < C; j += kFacThreads) {
-        const FacOut o = fac_channel(xmin[j], xmax[j], xmean[j], wmin[j], wmax[j], a, dead);
+        const FacOut o = fac_channel(xmin[j], xmax[j], xmean[j], wmin[j], wmax[j], a, dead, criterion);
         s[j] = o.s;
         rinv[j] = o.rinv;
         mu_hat[j] = o.mu;
@@ -190,10 +194,10 @@ factors_kernel(const float *__restrict__ xmin, const float *__restrict__ xmax, c
 
 aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean, const float *wmin,
                         const float *wmax, long long C, float *s, float *rinv, float *mu_hat, float *pX, float *pW,
-                        double *scalars, aweq_dev_status *st, cudaStream_t stream)
+                        double *scalars, aweq_dev_status *st, cudaStream_t stream, int criterion)
 {
     AWEQ_LAUNCH(factors_kernel, dim3(1), dim3(kFacThreads), 0, stream, xmin, xmax, xmean, wmin, wmax, (int)C, s, rinv,
-                mu_hat, pX, pW, scalars, st);
+                mu_hat, pX, pW, scalars, st, criterion);
     return AWEQ_OK;
 }
 

@@ -19,7 +19,7 @@ aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long 
                        float *wmax, int accumulate, void *ws, aweq_dev_status *st, cudaStream_t stream);
 aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean, const float *wmin,
                         const float *wmax, long long C, float *s, float *rinv, float *mu_hat, float *pX, float *pW,
-                        double *scalars, aweq_dev_status *st, cudaStream_t stream);
+                        double *scalars, aweq_dev_status *st, cudaStream_t stream, int criterion = 0);
 bool rowquant_supported(long long nrows, long long cols);
 aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long long cols, long long ld,
                          const float *scale, const float *mu, int bits, bool weights, unsigned char *out,

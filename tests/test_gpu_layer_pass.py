@@ -43,7 +43,8 @@ def compare_layer(wl, bits, Xc, Wc, bias_c=None, flags=0):
         lins = [l for l in wl.linears if l.input == inp.name]
         ref = util.oracle_layer(Xc[inp.name], [Wc[l.name] for l in lins], bits, gran, wl.group,
                                 None if bias_c is None else [bias_c.get(l.name) for l in lins],
-                                act_quant=wl.act_quant, equalize=eq, bias_correct=bc)
+                                act_quant=wl.act_quant, equalize=eq, bias_correct=bc,
+                                criterion=1 if flags & aweq.FLAG_ABSMAX_CRITERION else 0)
         o = {k: v.cpu().numpy() for k, v in cal.out[inp.name].items()}
         util.assert_same_values(o["xmin"], ref["stats"][0])
         util.assert_same_values(o["xmax"], ref["stats"][1])
@@ -101,7 +102,8 @@ def test_ablation_switches():
     from paper_2311_01305_b200 import aweq
     wl = synth.workloads(n_tokens_scale=1.0 / 8)["opt125m_linear_w8a8"]
     Xc, Wc = make_workload_tensors(wl, offset=2.0)
-    for flags in (aweq.FLAG_NO_EQUALIZE, aweq.FLAG_NO_BIAS_CORRECT, aweq.FLAG_NO_EQUALIZE | aweq.FLAG_NO_BIAS_CORRECT):
+    for flags in (aweq.FLAG_NO_EQUALIZE, aweq.FLAG_NO_BIAS_CORRECT, aweq.FLAG_NO_EQUALIZE | aweq.FLAG_NO_BIAS_CORRECT,
+                  aweq.FLAG_ABSMAX_CRITERION):
         compare_layer(wl, 8, Xc, Wc, None, flags=flags)
 
 

@@ -420,3 +420,23 @@ def test_bad_arguments_are_error_codes():
     with pytest.raises(aweq.AweqError) as e:
         aweq.aweq_quant_act(X, None, 8, aweq.PER_TENSOR, None, codes, step, zp)
     assert e.value.code == 1
+
+
+def test_factors_absmax_criterion_matches_oracle():
+    Xc = util.rand16((300, 1032), torch.float16, seed=21, offset=2.0, outlier_cols=5)
+    Wc = util.rand16((64, 1032), torch.float16, seed=22, scale=0.02)
+    xs = orc.stats(util.bits(Xc), orc.F16)
+    wr = orc.wrange(util.bits(Wc), orc.F16)
+    f = orc.factors(xs[0], xs[1], xs[2], wr[0], wr[1], orc.ABSMAX)
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(DEV)
+    C = 1032
+    o = {k: torch.empty(C, device=DEV) for k in ("s", "rinv", "mu", "pX", "pW")}
+    sc = torch.empty(8, dtype=torch.float64, device=DEV)
+    aweq.aweq_factors_absmax(t(xs[0]), t(xs[1]), t(xs[2]), t(wr[0]), t(wr[1]), o["s"], o["rinv"], o["mu"], o["pX"], o["pW"], sc)
+    torch.cuda.synchronize()
+    util.assert_same_values(o["s"].cpu().numpy(), f["s"], "s")
+    util.assert_same_values(o["rinv"].cpu().numpy(), f["rinv"], "rinv")
+    assert np.allclose(o["mu"].cpu().numpy(), f["mu_hat"], rtol=1e-6, atol=1e-12)
+    assert np.allclose(o["pX"].cpu().numpy(), f["pX"], rtol=1e-6) and np.allclose(sc.cpu().numpy(), f["scalars"], rtol=1e-6)
+    g = orc.factors(xs[0], xs[1], xs[2], wr[0], wr[1])
+    assert not np.array_equal(f["s"], g["s"])                 # offset data: the two criteria differ

@@ -57,6 +57,8 @@ def test_validation_rejects_null_before_any_cuda_call(lib):
     assert lib.aweq_stats(None, 0, 16, 64, 64, None, None, None, None, None, 0, None, 0, None, None) == 1
     lib.aweq_factors.argtypes = [vp] * 5 + [ll] + [vp] * 8
     assert lib.aweq_factors(None, None, None, None, None, 8, None, None, None, None, None, None, None, None) == 1
+    lib.aweq_factors_absmax.argtypes = [vp] * 5 + [ll] + [vp] * 8
+    assert lib.aweq_factors_absmax(None, None, None, None, None, 8, None, None, None, None, None, None, None, None) == 1
     lib.aweq_layer_pass.argtypes = [vp, vp, sz, vp, vp]
     assert lib.aweq_layer_pass(None, None, 0, None, None) == 1
     lib.aweq_fold_scale.argtypes = [vp, i, ll, ll, ll, vp, vp, ll, vp]

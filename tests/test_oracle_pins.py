@@ -669,3 +669,35 @@ def test_forward_check_weights_against_numpy_and_bias_correction(bits, gran, gro
     assert np.all(np.abs(raw - delta) <= 3e-6 * scale)
     assert np.all(np.abs(fixed) <= 3e-6 * scale + 2.0 ** -24 * np.abs(bf))
     assert np.abs(raw).max() > 20 * np.abs(fixed).max()
+
+
+# ---------------------------------------------------------------- the comparison criterion (Section 3.1)
+def test_absmax_criterion_closed_form_and_what_it_balances():
+    """Fed with the largest magnitudes, Eq. 10 is s = sqrt(max|x| / max|w|) and makes the largest
+    magnitudes of the equalised activations and weights equal per channel (what the per-channel
+    equalisation the paper starts from does); the range criterion makes the RANGES equal instead.
+    On channels with an offset the two differ; on symmetric channels they coincide."""
+    rng = np.random.default_rng(61)
+    C = 40
+    xmin = -rng.uniform(0.5, 3, C).astype(np.float32)
+    xmax = rng.uniform(0.5, 3, C).astype(np.float32)
+    xmin[:10] += 4.0                                        # offset channels: all positive
+    xmax[:10] += 4.0
+    xmean = ((xmin + xmax) / 2).astype(np.float32)
+    wmin = -rng.uniform(0.01, 0.1, C).astype(np.float32)
+    wmax = rng.uniform(0.01, 0.1, C).astype(np.float32)
+    xmin[20:30], wmin[20:30] = -xmax[20:30], -wmax[20:30]   # symmetric channels
+    f = orc.factors(xmin, xmax, xmean, wmin, wmax, orc.ABSMAX)
+    ax = np.maximum(np.abs(xmin), np.abs(xmax)).astype(np.float64)
+    aw = np.maximum(np.abs(wmin), np.abs(wmax)).astype(np.float64)
+    assert np.allclose(f["s"], np.sqrt(ax / aw), rtol=2e-7)
+    assert np.allclose(f["rinv"], 1.0 / f["s"], rtol=1e-7) and np.allclose(f["mu_hat"], xmean * f["rinv"], rtol=1e-7)
+    assert np.allclose(ax / f["s"], f["s"] * aw, rtol=3e-7)                      # equal largest magnitudes
+    g = orc.factors(xmin, xmax, xmean, wmin, wmax, orc.RANGE)
+    rx, rw = (xmax - xmin).astype(np.float64), (wmax - wmin).astype(np.float64)
+    assert np.allclose(rx / g["s"], g["s"] * rw, rtol=3e-7)                      # equal ranges
+    assert np.allclose(f["s"][20:30], g["s"][20:30], rtol=3e-7)                  # symmetric: the same factor
+    assert np.all(f["s"][:10] > 1.1 * g["s"][:10])                               # offset: abs-max overstates x
+    assert np.array_equal(g["s"], orc.factors(xmin, xmax, xmean, wmin, wmax)["s"])   # the default is the paper's
+    # the diagnostics stay range-based under either criterion
+    assert np.array_equal(f["pX"], g["pX"]) and np.array_equal(f["pW"], g["pW"])

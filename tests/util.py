@@ -63,14 +63,15 @@ def assert_same_values(a, b, what=""):
         what, int(bad.sum()), np.argwhere(bad)[0], a[bad][0], b[bad][0])
 
 
-def oracle_layer(Xc, Wcs, bits, gran, group, biases=None, act_quant=True, equalize=True, bias_correct=True):
+def oracle_layer(Xc, Wcs, bits, gran, group, biases=None, act_quant=True, equalize=True, bias_correct=True,
+                 criterion=0):
     """The six steps through the CPU oracle for one input and the matrices it feeds."""
     dt = odt(Xc)
     xs = orc.stats(bits_of(Xc), dt)
     wr = None
     for Wc in Wcs:
         wr = orc.wrange(bits_of(Wc), dt, prev=wr)
-    f = orc.factors(xs[0], xs[1], xs[2], wr[0], wr[1])
+    f = orc.factors(xs[0], xs[1], xs[2], wr[0], wr[1], criterion)
     s = f["s"] if equalize else None
     rinv = f["rinv"] if equalize else None
     mu = f["mu_hat"] if equalize else xs[2]
