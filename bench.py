@@ -191,16 +191,6 @@ def run_forward_check(args, wl, bits):
     torch.cuda.synchronize()
     launches = aweq.launch_count() - n0
     clocks = sampler.stop()
-    if graph is not None:
-        # the kernels of a replay are the ones one eager pass launches; time the dominant one eagerly
-        torch.cuda.synchronize()
-        n1 = aweq.launch_count()
-        for k in range(args.steps):
-            for lp, (es, ea) in zip(cal.passes, hooks[k]):
-                lp.set_events(es, ea)
-            cal.run()
-        torch.cuda.synchronize()
-        launches = aweq.launch_count() - n1
     ms = a.elapsed_time(b) / args.steps
     tokens = {i.name: i.n_tokens for i in wl.inputs}
     flops = sum(4.0 * tokens[l.input] * l.c_in * l.c_out for l in wl.linears)
