@@ -12,6 +12,15 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+def pytest_sessionstart(session):
+    """Build the CUDA library and the oracle when they are missing or stale (nvcc and gcc only; no
+    GPU needed), so that a fresh checkout can be tested without a separate build step."""
+    from paper_2311_01305_b200 import build
+    build.build()
+    from oracle import aweq_oracle
+    aweq_oracle.build()
+
+
 def pytest_collection_modifyitems(config, items):
     import torch
     if torch.cuda.is_available():
