@@ -270,6 +270,8 @@ def main():
     if args.impl == "reference":
         return run_reference(args, wl, bits)
 
+    from paper_2311_01305_b200 import build as _build
+    _build.build()                      # no-op when libaweq.so is up to date
     from paper_2311_01305_b200 import aweq, calibrate
 
     if args.op == "forward_check":

@@ -63,6 +63,19 @@ def _compile(src: str, obj: str, verbose: bool) -> str:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    """Build when the library is missing or older than a source; returns its path.  Serialised with
+    a file lock, so that several ranks starting together compile once."""
+    import fcntl
+    os.makedirs(OBJ, exist_ok=True)
+    with open(os.path.join(OBJ, ".lock"), "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            return _build_locked(force, verbose)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
+
+
+def _build_locked(force: bool, verbose: bool) -> str:
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     deps = srcs + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) + [
         os.path.join(os.path.dirname(HERE), "include", "aweq.h"), os.path.abspath(__file__)]
