@@ -332,11 +332,10 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
                         col_part, st, stream);
         if (rc != AWEQ_OK) return rc;
         if (a->ev_stats_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_end, cs));
-        for (int i = 0; i < a->n_w; ++i) {
-            rc = aweq_wrange(a->W[i], a->dt, a->C_out[i], a->C_in, a->ldw[i], a->wmin, a->wmax, i > 0, ws_col, col_part,
-                             st, stream);
-            if (rc != AWEQ_OK) return rc;
-        }
+        // step 2: the matrices share the input, hence one range per input channel over all of them
+        AWEQ_LOGF("aweq_wrange x%d C_in=%lld\n", a->n_w, a->C_in);
+        rc = run_wrange_multi(a->W, a->C_out, a->ldw, a->n_w, a->dt, a->C_in, a->wmin, a->wmax, 0, ws_col, st, cs);
+        if (rc != AWEQ_OK) return rc;
     }
     const bool eq = !(a->flags & AWEQ_FLAG_NO_EQUALIZE);
     // without equalisation the layer sees x itself, so E[x^] = E[x]

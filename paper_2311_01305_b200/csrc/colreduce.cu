@@ -158,6 +158,33 @@ __device__ __forceinline__ void two_sum_into(float &hi, float &lo, float a)
     hi = s;
 }
 
+// Up to four matrices with the same number of columns, reduced as if stacked on top of one
+// another (the weight matrices that share a layer input: q / k / v, gate / up).  A stage never
+// straddles two of them.
+constexpr int kColMaxSegs = 4;
+struct ColSegs {
+    const uint16_t *base[kColMaxSegs];
+    long long rows[kColMaxSegs];
+    long long ld[kColMaxSegs];
+    int n;
+};
+
+// the matrix that holds stacked row v, the row inside it, and the stacked index where it ends
+__device__ __forceinline__ void seg_locate(const ColSegs &sg, long long v, int &m, long long &local, long long &end)
+{
+    long long start = 0;
+    m = 0;
+#pragma unroll
+    for (int k = 0; k < kColMaxSegs - 1; ++k) {
+        if (m == k && k + 1 < sg.n && v >= start + sg.rows[k]) {
+            start += sg.rows[k];
+            m = k + 1;
+        }
+    }
+    local = v - start;
+    end = start + sg.rows[m];
+}
+
 struct ColSmem {
     uint64_t full[kColStages];
     uint64_t empty[kColStages];
@@ -166,7 +193,7 @@ struct ColSmem {
 
 template <class D, bool WITH_SUM>
 __global__ void __launch_bounds__(kColThreads + 32, kColCtasPerSm)
-colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, int nvec, int nslab, int slab_w,
+colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int slab_w,
                  int phases, int stage_rows, long long rows_per_split, long long cols, float *__restrict__ pmin,
                  float *__restrict__ pmax, double *__restrict__ psum, aweq_dev_status *st)
 {
@@ -180,7 +207,6 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
     const int w = min(slab_w, nvec - v0);                 // vectors in this slab (> 0)
     const long long r0 = (long long)split * rows_per_split;
     const long long r1 = min(nrows, r0 + rows_per_split);
-    const int ntiles = r1 > r0 ? (int)((r1 - r0 + stage_rows - 1) / stage_rows) : 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // phase p of the consumer threads takes rows [p, p + 1) * stage_rows / phases of every stage;
     // a phase is a whole number of warps
@@ -201,9 +227,9 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
 
     if (warp == kColThreads / 32) {
         // ---------------- producer warp
-        const bool contiguous = (nslab == 1) && (ld == cols);
         bool ok = true;
-        for (int t = 0; t < ntiles && ok; ++t) {
+        long long cur = r0;
+        for (int t = 0; cur < r1 && ok; ++t) {
             const int s = t % kColStages;
             const uint32_t use = t / kColStages;
             if (use > 0) {
@@ -211,18 +237,24 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
             }
-            const long long row0 = r0 + (long long)t * stage_rows;
-            const int rows = (int)min((long long)stage_rows, r1 - row0);
+            int m;
+            long long local, seg_end;
+            seg_locate(segs, cur, m, local, seg_end);
+            const long long ld = segs.ld[m];
+            const uint16_t *X = segs.base[m];
+            const int rows = (int)min((long long)stage_rows, min(r1, seg_end) - cur);
+            const bool contiguous = (nslab == 1) && (ld == cols);
             uint4 *dst = stage_base + (size_t)s * stage_vecs;
             if (lane == 0) mbar_arrive_expect_tx(&sm->full[s], (uint32_t)rows * w * 16u);
             __syncwarp();
             if (contiguous) {
-                if (lane == 0) bulk_g2s(dst, X + row0 * ld, (uint32_t)rows * w * 16u, &sm->full[s]);
+                if (lane == 0) bulk_g2s(dst, X + local * ld, (uint32_t)rows * w * 16u, &sm->full[s]);
             } else {
                 for (int r = lane; r < rows; r += 32)
-                    bulk_g2s(dst + (size_t)r * w, X + (row0 + r) * ld + (long long)v0 * 8, (uint32_t)w * 16u,
+                    bulk_g2s(dst + (size_t)r * w, X + (local + r) * ld + (long long)v0 * 8, (uint32_t)w * 16u,
                              &sm->full[s]);
             }
+            cur += rows;
         }
         if (!ok && lane == 0) {
             atomicExch(&sm->abort_flag, 1);
@@ -244,13 +276,17 @@ colreduce_kernel(const uint16_t *__restrict__ X, long long nrows, long long ld, 
 #pragma unroll
         for (int k = 0; k < 8; ++k) sum_hi[k] = sum_lo[k] = 0.0f;
         bool ok = true;
-        for (int t = 0; t < ntiles; ++t) {
+        long long cur = r0;
+        for (int t = 0; cur < r1; ++t) {
             const int s = t % kColStages;
             const uint32_t use = t / kColStages;
             ok = mbar_wait(&sm->full[s], use & 1);
             if (!ok || *reinterpret_cast<volatile int *>(&sm->abort_flag)) { ok = false; break; }
-            const long long row0 = r0 + (long long)t * stage_rows;
-            const int rows_in_stage = (int)min((long long)stage_rows, r1 - row0);
+            int m;
+            long long local, seg_end;
+            seg_locate(segs, cur, m, local, seg_end);
+            const int rows_in_stage = (int)min((long long)stage_rows, min(r1, seg_end) - cur);
+            cur += rows_in_stage;
             const int rows = min(rows_in_stage, (phase + 1) * rows_per_phase);      // end of my share
             const uint4 *src = stage_base + (size_t)s * stage_vecs + t_col;
             if (mine) {
@@ -387,10 +423,12 @@ static size_t colreduce_smem_bytes(int slab_w, int stage_rows)
 }
 
 template <class D, bool WITH_SUM>
-static aweq_status launch_colreduce(const void *X, long long rows, long long cols, long long ld, float *omin,
+static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *omin,
                                     float *omax, float *omean, double *osum, long long *count, int accumulate,
                                     void *ws, aweq_dev_status *st, cudaStream_t stream)
 {
+    long long rows = 0;
+    for (int k = 0; k < segs.n; ++k) rows += segs.rows[k];
     ColPlan p = plan_colreduce(rows, cols);
     char *base = reinterpret_cast<char *>(ws);
     float *pmin = reinterpret_cast<float *>(base);
@@ -405,8 +443,8 @@ static aweq_status launch_colreduce(const void *X, long long rows, long long col
     int nsplit_eff = rows > 0 ? (int)nparts : 0;
     if (rows > 0) {
         AWEQ_LAUNCH(kern, dim3(p.nslab * p.nsplit), dim3(kColThreads + 32), smem, stream,
-                    reinterpret_cast<const uint16_t *>(X), rows, ld, p.nvec, p.nslab, p.slab_w, p.phases, p.stage_rows,
-                    p.rows_per_split, cols, pmin, pmax, psum, st);
+                    segs, rows, p.nvec, p.nslab, p.slab_w, p.phases, p.stage_rows, p.rows_per_split, cols, pmin, pmax,
+                    psum, st);
     }
     AWEQ_LAUNCH(colreduce_finalize_kernel<WITH_SUM>, dim3((unsigned)((cols + kFinCols - 1) / kFinCols)),
                 dim3(kFinCols * kFinLanes), 0, stream, (const float *)pmin, (const float *)pmax, (const double *)psum,
@@ -434,19 +472,45 @@ aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, lo
                       float *xmean, double *xsum, long long *count, int accumulate, void *ws, aweq_dev_status *st,
                       cudaStream_t stream)
 {
+    ColSegs segs = {};
+    segs.base[0] = reinterpret_cast<const uint16_t *>(X);
+    segs.rows[0] = N;
+    segs.ld[0] = ld;
+    segs.n = 1;
     if (dt == AWEQ_F16)
-        return launch_colreduce<F16, true>(X, N, C, ld, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
-    return launch_colreduce<BF16, true>(X, N, C, ld, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
+        return launch_colreduce<F16, true>(segs, C, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
+    return launch_colreduce<BF16, true>(segs, C, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
 }
 
 aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld, float *wmin,
                        float *wmax, int accumulate, void *ws, aweq_dev_status *st, cudaStream_t stream)
 {
-    if (dt == AWEQ_F16)
-        return launch_colreduce<F16, false>(W, C_out, C_in, ld, wmin, wmax, nullptr, nullptr, nullptr, accumulate, ws,
-                                            st, stream);
-    return launch_colreduce<BF16, false>(W, C_out, C_in, ld, wmin, wmax, nullptr, nullptr, nullptr, accumulate, ws, st,
-                                         stream);
+    const void *Ws[1] = {W};
+    return run_wrange_multi(Ws, &C_out, &ld, 1, dt, C_in, wmin, wmax, accumulate, ws, st, stream);
+}
+
+// The common range of several matrices with the same C_in: stacks of up to four go through one
+// launch (one pipeline fill and one finalize instead of one per matrix).
+aweq_status run_wrange_multi(const void *const *W, const long long *C_out, const long long *ld, int n, aweq_dtype dt,
+                             long long C_in, float *wmin, float *wmax, int accumulate, void *ws, aweq_dev_status *st,
+                             cudaStream_t stream)
+{
+    for (int i0 = 0; i0 < n; i0 += kColMaxSegs) {
+        ColSegs segs = {};
+        segs.n = n - i0 < kColMaxSegs ? n - i0 : kColMaxSegs;
+        for (int k = 0; k < segs.n; ++k) {
+            segs.base[k] = reinterpret_cast<const uint16_t *>(W[i0 + k]);
+            segs.rows[k] = C_out[i0 + k];
+            segs.ld[k] = ld[i0 + k];
+        }
+        const int acc = accumulate || i0 > 0;
+        const aweq_status rc =
+            dt == AWEQ_F16 ? launch_colreduce<F16, false>(segs, C_in, wmin, wmax, nullptr, nullptr, nullptr, acc, ws, st, stream)
+                           : launch_colreduce<BF16, false>(segs, C_in, wmin, wmax, nullptr, nullptr, nullptr, acc, ws, st,
+                                                           stream);
+        if (rc != AWEQ_OK) return rc;
+    }
+    return AWEQ_OK;
 }
 
 }  // namespace aweq

@@ -17,6 +17,9 @@ aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, lo
                       cudaStream_t stream);
 aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld, float *wmin,
                        float *wmax, int accumulate, void *ws, aweq_dev_status *st, cudaStream_t stream);
+aweq_status run_wrange_multi(const void *const *W, const long long *C_out, const long long *ld, int n, aweq_dtype dt,
+                             long long C_in, float *wmin, float *wmax, int accumulate, void *ws, aweq_dev_status *st,
+                             cudaStream_t stream);
 aweq_status run_factors(const float *xmin, const float *xmax, const float *xmean, const float *wmin,
                         const float *wmax, long long C, float *s, float *rinv, float *mu_hat, float *pX, float *pW,
                         double *scalars, aweq_dev_status *st, cudaStream_t stream, int criterion = 0);
