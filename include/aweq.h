@@ -319,6 +319,15 @@ aweq_status aweq_layer_pass(const aweq_layer_args *args, void *ws, size_t ws_byt
 aweq_status aweq_fold_scale(const void *P, aweq_dtype dt, long long rows, long long cols, long long ld,
                             const float *rinv, void *out, long long ld_out, void *stream);
 
+/* ---- Signed relabelling of 8-bit codes ------------------------------------------------------
+ * Eq. 1 gives unsigned codes q in [0, 255] and a zero-point Z; consumers that take signed 8-bit
+ * operands use q' = q - 128 and Z' = Z - 128 (saturating), which de-quantise to the same values,
+ * Step (q' - Z') = Step (q - Z).  codes: n bytes, one 8-bit code each (step-6 activations or 8-bit
+ * step-4 weights); out: n bytes, may be codes itself (in place).  zp / zp_out: nz zero-points, or
+ * both NULL.  Device pointers; enqueued on `stream`. */
+aweq_status aweq_relabel_signed(const unsigned char *codes, long long n, signed char *out,
+                                const int *zp, long long nz, int *zp_out, void *stream);
+
 /* ---- Forward check of a calibrated W8A8 layer (Eq. 11; the quantity ablated in the AWE / BC
  * table) ------------------------------------------------------------------------------------
  * Compares, on the calibration tokens, the quantised layer

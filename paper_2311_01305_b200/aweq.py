@@ -79,6 +79,8 @@ _lib.aweq_layer_pass_workspace_bytes.argtypes = [ctypes.POINTER(LayerArgs)]
 _lib.aweq_layer_pass.argtypes = [ctypes.POINTER(LayerArgs), _vp, _sz, _vp, _vp]
 _lib.aweq_plan_query.argtypes = [_i, _ll, _ll, ctypes.POINTER(_ll * 8)]
 _lib.aweq_plan_query.restype = _i
+_lib.aweq_relabel_signed.argtypes = [_vp, _ll, _vp, _vp, _ll, _vp, _vp]
+_lib.aweq_relabel_signed.restype = _i
 _lib.aweq_fold_scale.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _vp, _ll, _vp]
 _lib.aweq_fold_scale.restype = _i
 _lib.aweq_forward_check_workspace_bytes.restype = _sz
@@ -223,6 +225,17 @@ def aweq_plan_query(op: int, rows: int, cols: int):
     plan = (_ll * 8)()
     _check(_lib.aweq_plan_query(op, rows, cols, ctypes.byref(plan)))
     return tuple(plan)
+
+
+def aweq_relabel_signed(codes, out=None, zp=None, zp_out=None):
+    """8-bit codes q -> q - 128 (an ``int8`` view of the result is the signed code) and zero-points
+    Z -> Z - 128; in place when ``out`` / ``zp_out`` are None."""
+    out = codes if out is None else out
+    if zp is not None and zp_out is None:
+        zp_out = zp
+    _check(_lib.aweq_relabel_signed(_ptr(codes), codes.numel(), _ptr(out), _ptr(zp), 0 if zp is None else zp.numel(),
+                                    _ptr(zp_out), _stream()))
+    return out, zp_out
 
 
 def aweq_fold_scale(P, rinv, out=None):

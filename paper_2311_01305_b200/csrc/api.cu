@@ -387,6 +387,16 @@ aweq_status aweq_fold_scale(const void *P, aweq_dtype dt, long long rows, long l
     return run_fold_scale(P, dt, rows, cols, ld, rinv, out, ld_out, (cudaStream_t)stream);
 }
 
+// ------------------------------------------------------------------ signed relabelling
+aweq_status aweq_relabel_signed(const unsigned char *codes, long long n, signed char *out, const int *zp, long long nz,
+                                int *zp_out, void *stream)
+{
+    if (!codes || !out) return AWEQ_ERR_NULL;
+    if ((zp == nullptr) != (zp_out == nullptr)) return AWEQ_ERR_NULL;
+    if (n <= 0 || nz < 0 || (zp && nz == 0)) return AWEQ_ERR_SHAPE;
+    return run_relabel_signed(codes, n, out, zp, zp ? nz : 0, zp_out, (cudaStream_t)stream);
+}
+
 // ------------------------------------------------------------------ forward check
 size_t aweq_forward_check_workspace_bytes(long long N, long long C_in, long long C_out)
 {

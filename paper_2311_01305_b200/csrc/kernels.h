@@ -44,6 +44,9 @@ aweq_status run_bias_gemv(const void *W, aweq_dtype dt, long long C_out, long lo
 aweq_status run_fold_scale(const void *P, aweq_dtype dt, long long rows, long long cols, long long ld,
                            const float *rinv, void *out, long long ld_out, cudaStream_t stream);
 
+aweq_status run_relabel_signed(const unsigned char *codes, long long n, signed char *out, const int *zp, long long nz,
+                               int *zp_out, cudaStream_t stream);
+
 // forward check (tensor-core GEMMs + comparison)
 size_t forward_check_ws_bytes(long long N, long long C_in, long long C_out);
 aweq_status run_forward_check(const unsigned char *Xq, const float *act_step, const int *act_zp,

@@ -137,3 +137,28 @@ def test_decoder_walk_matches_oracle_in_the_same_order(kind, dtype, act_quant, b
         changed = not torch.equal(walk.W[l.name].cpu(), Wc[l.name])
         assert changed == (l.name in {p for kd, p in prod.values() if kd == "linear"})
         assert np.array_equal(util.bits(walk.W[l.name]), Wb[l.name])
+
+
+@pytest.mark.parametrize("shape", [(300, 768), (7, 13), (1, 1)])
+def test_relabel_signed_keeps_the_dequantised_values(shape):
+    """q' = q - 128, Z' = Z - 128 (checked against NumPy integer arithmetic, the definition); the
+    de-quantised values Step (q' - Z') are those of the unsigned codes."""
+    from paper_2311_01305_b200 import aweq
+    rng = np.random.default_rng(shape[0])
+    q = rng.integers(0, 256, shape).astype(np.uint8)
+    zp = rng.integers(-300, 600, shape[0]).astype(np.int32)
+    out, check = util.guarded(shape, torch.uint8)
+    zp_out, check_z = util.guarded((shape[0],), torch.int32)
+    aweq.aweq_relabel_signed(torch.from_numpy(q).to(DEV), out, torch.from_numpy(zp).to(DEV), zp_out)
+    torch.cuda.synchronize()
+    check()
+    check_z()
+    qs = out.cpu().numpy().view(np.int8)
+    assert np.array_equal(qs.astype(np.int32), q.astype(np.int32) - 128)
+    assert np.array_equal(zp_out.cpu().numpy(), zp - 128)
+    assert np.array_equal(qs.astype(np.int64) - zp_out.cpu().numpy()[:, None], q.astype(np.int64) - zp[:, None])
+    # in place, codes only
+    t = torch.from_numpy(q).to(DEV)
+    aweq.aweq_relabel_signed(t)
+    torch.cuda.synchronize()
+    assert np.array_equal(t.cpu().numpy().view(np.int8).astype(np.int32), q.astype(np.int32) - 128)

@@ -63,6 +63,8 @@ def test_validation_rejects_null_before_any_cuda_call(lib):
     assert lib.aweq_layer_pass(None, None, 0, None, None) == 1
     lib.aweq_fold_scale.argtypes = [vp, i, ll, ll, ll, vp, vp, ll, vp]
     assert lib.aweq_fold_scale(None, 0, 8, 8, 8, None, None, 8, None) == 1
+    lib.aweq_relabel_signed.argtypes = [vp, ll, vp, vp, ll, vp, vp]
+    assert lib.aweq_relabel_signed(None, 16, None, None, 0, None, None) == 1
     lib.aweq_forward_check.argtypes = [vp] * 9 + [i, vp, ll, ll, ll, vp, vp, vp, sz, vp]
     assert lib.aweq_forward_check(*([None] * 9), 0, None, 64, 64, 64, None, None, None, 0, None) == 1
     lib.aweq_forward_check_workspace_bytes.restype = sz
