@@ -137,14 +137,18 @@ class LayerCalibrator:
         cur.wait_stream(big)
         cur.wait_stream(small)
 
-    def capture(self) -> "torch.cuda.CUDAGraph":
+    def capture(self, events=None) -> "torch.cuda.CUDAGraph":
         """Record one ``run()`` (both streams and their events when ``overlap`` is on) into a CUDA
         graph; ``graph.replay()`` then re-issues the whole pass with one launch.  The library's
-        calls are capture-safe (no allocation, no synchronisation); the profiling event hooks of
-        ``LayerPass.set_events`` must be unset, and one ordinary ``run()`` must have happened before
-        (it sets the kernels' shared-memory attributes outside the capture)."""
-        for lp in self.passes:
-            lp.set_events(None, None)
+        calls are capture-safe (no allocation, no synchronisation).  ``events``: one (stats pair,
+        act pair or None) of timing events per pass for the profiling hooks; inside a graph they
+        are recorded anew on every replay and hold the times of the latest one.  One ordinary
+        ``run()`` happens first (it sets the kernels' shared-memory attributes outside the capture)."""
+        for i, lp in enumerate(self.passes):
+            if events is None:
+                lp.set_events(None, None)
+            else:
+                lp.set_events(events[i][0], events[i][1])
         self.run()
         torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()

@@ -291,6 +291,18 @@ size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args)
     return layer_ws_parts(args, nullptr);
 }
 
+// A profiling hook.  While the stream is being captured into a CUDA graph an ordinary record would
+// only become an edge of the graph; as an external record it becomes a node of its own, so the
+// event is recorded anew on every replay and can be read back afterwards.
+static cudaError_t record_hook(void *ev, cudaStream_t cs)
+{
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    cudaError_t e = cudaStreamIsCapturing(cs, &cap);
+    if (e != cudaSuccess) return e;
+    return cudaEventRecordWithFlags((cudaEvent_t)ev, cs,
+                                    cap == cudaStreamCaptureStatusActive ? cudaEventRecordExternal : cudaEventRecordDefault);
+}
+
 aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes, aweq_dev_status *st, void *stream)
 {
     if (!a) return AWEQ_ERR_NULL;
@@ -327,11 +339,11 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     const int phases = (a->flags & kAllPhases) ? (a->flags & kAllPhases) : kAllPhases;
     // steps 1-2
     if (phases & AWEQ_FLAG_PHASE_REDUCE) {
-        if (a->ev_stats_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_begin, cs));
+        if (a->ev_stats_begin) AWEQ_CUDA_OK(record_hook(a->ev_stats_begin, cs));
         rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
                         col_part, st, stream);
         if (rc != AWEQ_OK) return rc;
-        if (a->ev_stats_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_stats_end, cs));
+        if (a->ev_stats_end) AWEQ_CUDA_OK(record_hook(a->ev_stats_end, cs));
         // step 2: the matrices share the input, hence one range per input channel over all of them
         AWEQ_LOGF("aweq_wrange x%d C_in=%lld\n", a->n_w, a->C_in);
         rc = run_wrange_multi(a->W, a->C_out, a->ldw, a->n_w, a->dt, a->C_in, a->wmin, a->wmax, 0, ws_col, st, cs);
@@ -365,11 +377,11 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     }
     // step 6
     if (a->Xq && (phases & AWEQ_FLAG_PHASE_ACT)) {
-        if (a->ev_act_begin) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_act_begin, cs));
+        if (a->ev_act_begin) AWEQ_CUDA_OK(record_hook(a->ev_act_begin, cs));
         rc = aweq_quant_act(a->X, a->dt, a->N, a->C_in, a->ldx, rinv_used, a->act_bits ? a->act_bits : 8, AWEQ_PER_ROW,
                             nullptr, a->Xq, a->act_step, a->act_zp, st, stream);
         if (rc != AWEQ_OK) return rc;
-        if (a->ev_act_end) AWEQ_CUDA_OK(cudaEventRecord((cudaEvent_t)a->ev_act_end, cs));
+        if (a->ev_act_end) AWEQ_CUDA_OK(record_hook(a->ev_act_end, cs));
     }
     return AWEQ_OK;
 }

@@ -177,7 +177,15 @@ def test_graph_replay_equals_eager(overlap):
     a = calibrate.LayerCalibrator(wl, 8, Xd, Wd, None)
     b = calibrate.LayerCalibrator(wl, 8, Xd, Wd, None, overlap=overlap)
     a.run()
-    graph = b.capture()
+    E = lambda: torch.cuda.Event(enable_timing=True)
+    hooks = []
+    for _ in b.passes:
+        pairs = ((E(), E()), (E(), E()))
+        for pr in pairs:
+            for e in pr:
+                e.record()                                # create the handles
+        hooks.append(pairs)
+    graph = b.capture(hooks)
     n0 = aweq.launch_count()
     for _ in range(2):
         for outs in b.out.values():
@@ -186,6 +194,10 @@ def test_graph_replay_equals_eager(overlap):
         graph.replay()
     torch.cuda.synchronize()
     assert aweq.launch_count() == n0                      # replays go through no library call
+    # the profiling hooks were recorded by the replay itself and can be read back
+    for stats_pair, act_pair in hooks:
+        assert 0.0 < stats_pair[0].elapsed_time(stats_pair[1]) < 50.0
+        assert 0.0 < act_pair[0].elapsed_time(act_pair[1]) < 50.0
     assert aweq.read_status(b.status)["wait_timeout"] == 0
     for nm, outs in a.out.items():
         for k, v in outs.items():
