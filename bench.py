@@ -258,6 +258,9 @@ def main():
     ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
     ap.add_argument("--no-overlap", action="store_true",
                     help="issue every input's pass on one stream (default: two alternating streams)")
+    ap.add_argument("--eager", action="store_true",
+                    help="launch every timed step eagerly (default at 1 GPU: the steps that carry the event hooks "
+                         "are eager, the others replay the pass from a CUDA graph)")
     ap.add_argument("--graph", action="store_true",
                     help="replay the pass as one CUDA graph in the timed region (1 GPU; the dominant kernel is then "
                          "timed in eager passes after it)")
@@ -313,10 +316,16 @@ def main():
     for _ in range(args.warmup):
         cal.run()
     graph = None
-    if args.graph and world == 1:
-        graph = cal.capture()               # without the event hooks: as graph nodes they cost 3 % of the pass
-        for _ in range(args.warmup):
-            graph.replay()
+    if world == 1 and not args.eager:
+        try:
+            graph = cal.capture()           # without the event hooks: as graph nodes they cost 3 % of the pass
+            for _ in range(args.warmup):
+                graph.replay()
+        except Exception as exc:            # a capture that fails leaves the eager pass as it was
+            sys.stderr.write("CUDA graph capture failed (%s); timing eager launches\n" % exc)
+            graph = None
+            torch.cuda.synchronize()
+    mixed = graph is not None and not args.graph
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
@@ -330,7 +339,7 @@ def main():
             names = [i.name for i in wl.inputs if i.name in cal.out]
             cal.events = {n: h for n, h in zip(names, hooks[k])} if k in hooks else None
             cal.run()                       # statistics merged over the ranks inside the step
-        elif graph is not None:
+        elif graph is not None and not (mixed and k in hooks):
             graph.replay()
         else:
             for i, lp in enumerate(cal.passes):
@@ -341,7 +350,10 @@ def main():
     barrier()
     launches = aweq.launch_count() - n0
     clocks = sampler.stop()
-    if graph is not None:
+    if mixed:
+        # replays go through no library call: a replay launches what an eager step launches
+        launches = launches // len(hooks) * args.steps
+    elif graph is not None:
         # replays go through no library call: a replay launches what one eager pass launches.  The
         # dominant kernel is timed in eager passes after the timed region (hooks inside the graph
         # would be recorded by every replay, but as graph nodes of their own they slow it down).
@@ -402,7 +414,8 @@ def main():
                    "act_quant": wl.act_quant, "storage": wl.dtype, "tokens_per_gpu": tokens,
                    "algorithmic_bytes_per_gpu": nbytes, "cache": "inputs (GBs) far larger than the 126 MB L2",
                    "parallelism": "token shards, one per GPU" if world > 1 else "single GPU",
-                   "launch": "one CUDA graph replay per step" if graph is not None else "eager",
+                   "launch": ("CUDA graph replay; every fourth step eager, with the event hooks" if mixed
+                              else "one CUDA graph replay per step" if graph is not None else "eager"),
                    "schedule": ("two streams: column reductions and step 6 on one, factors and weight quantiser on the other"
                                 if getattr(cal, "overlap", False) else "one stream")},
         "tokens_per_s": world * tokens / (ms / 1e3),
