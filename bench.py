@@ -13,7 +13,8 @@ with the shapes and value distributions of the named model layer; they are
 resident in HBM before the timed region and are far larger than L2.
 
 The metric is layer-pass HBM GB/s: algorithmic bytes of the pass divided by its
-device time (CUDA events, max over ranks).  With N > 1 every rank calibrates
+device time (CUDA events, max over ranks).  At one GPU the pass runs on two streams and the
+steps that carry no profiling hooks replay it from a CUDA graph (--eager, --no-overlap).  With N > 1 every rank calibrates
 its own token shard of the same layer (weak scaling, no data-path collective).
 """
 from __future__ import annotations
