@@ -72,7 +72,17 @@ struct F16 {
     static __device__ __forceinline__ T2 from_bits(uint32_t u) { return *reinterpret_cast<T2 *>(&u); }
     static __device__ __forceinline__ uint32_t pos_inf2() { return 0x7C007C00u; }
     static __device__ __forceinline__ uint32_t neg_inf2() { return 0xFC00FC00u; }
-    static __device__ __forceinline__ float2 to_float2(T2 v) { return __half22float2(v); }
+    // fp16 -> binary32 as "x + (-0)" with the mixed-precision add of sm_100 (exact, signed zeros
+    // included): it issues on the FMA pipe, whereas cvt.f32.f16 goes through the conversion unit,
+    // which the row quantisers saturated (16 conversions per 16 bytes of input)
+    static __device__ __forceinline__ float2 to_float2(T2 v)
+    {
+        float2 r;
+        asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\t"
+            "add.rn.f32.f16 %0, l, 0f80000000;\n\tadd.rn.f32.f16 %1, h, 0f80000000;\n\t}"
+            : "=f"(r.x), "=f"(r.y) : "r"(*reinterpret_cast<const uint32_t *>(&v)));
+        return r;
+    }
     static __device__ __forceinline__ float one(uint16_t b) { return __half2float(__ushort_as_half(b)); }
     static __device__ __forceinline__ uint16_t encode(float f) { return __half_as_ushort(__float2half_rn(f)); }
 };
