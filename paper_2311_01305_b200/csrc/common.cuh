@@ -206,6 +206,20 @@ __device__ __forceinline__ bool named_bar_and(int id, int threads, bool pred)
     return r != 0;
 }
 
+// three-input min / max (one instruction on sm_100)
+__device__ __forceinline__ float fmin3(float a, float b, float c)
+{
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // ------------------------------------------------------------------ warp reductions
 __device__ __forceinline__ float redux_min(float v, uint32_t mask)
 {

@@ -276,10 +276,10 @@ rowquant_kernel(const RowQuantParams p)
                             xh[v][2] = __fmul2_rn(xh[v][2], make_float2(s1.x, s1.y));
                             xh[v][3] = __fmul2_rn(xh[v][3], make_float2(s1.z, s1.w));
                         }
-                        lo = fminf(fminf(lo, xh[v][0].x), xh[v][0].y); hi = fmaxf(fmaxf(hi, xh[v][0].x), xh[v][0].y);
-                        lo = fminf(fminf(lo, xh[v][1].x), xh[v][1].y); hi = fmaxf(fmaxf(hi, xh[v][1].x), xh[v][1].y);
-                        lo = fminf(fminf(lo, xh[v][2].x), xh[v][2].y); hi = fmaxf(fmaxf(hi, xh[v][2].x), xh[v][2].y);
-                        lo = fminf(fminf(lo, xh[v][3].x), xh[v][3].y); hi = fmaxf(fmaxf(hi, xh[v][3].x), xh[v][3].y);
+                        lo = fmin3(lo, xh[v][0].x, xh[v][0].y); hi = fmax3(hi, xh[v][0].x, xh[v][0].y);
+                        lo = fmin3(lo, xh[v][1].x, xh[v][1].y); hi = fmax3(hi, xh[v][1].x, xh[v][1].y);
+                        lo = fmin3(lo, xh[v][2].x, xh[v][2].y); hi = fmax3(hi, xh[v][2].x, xh[v][2].y);
+                        lo = fmin3(lo, xh[v][3].x, xh[v][3].y); hi = fmax3(hi, xh[v][3].x, xh[v][3].y);
                     }
                 }
                 if (early && r + teams >= rows) {             // my last row of the tile is in registers

@@ -131,8 +131,8 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
 #pragma unroll
                             for (int c = 0; c < 4; ++c) {
                                 const float2 x = __fmul2_rn(D::to_float2(D::from_bits(w[c])), f[c]);
-                                lo[r] = fminf(fminf(lo[r], x.x), x.y);
-                                hi[r] = fmaxf(fmaxf(hi[r], x.x), x.y);
+                                lo[r] = fmin3(lo[r], x.x, x.y);
+                                hi[r] = fmax3(hi[r], x.x, x.y);
                             }
                         }
                     }

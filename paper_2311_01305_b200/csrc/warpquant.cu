@@ -164,9 +164,9 @@ warpquant_kernel(const WarpQuantParams p)
                 q = qs;
                 fl = qs_flags;
             } else {
-                float a = fminf(fminf(w2[0].x, w2[0].y), w2[1].x), b = fmaxf(fmaxf(w2[0].x, w2[0].y), w2[1].x);
-                a = fminf(fminf(a, w2[1].y), w2[2].x); b = fmaxf(fmaxf(b, w2[1].y), w2[2].x);
-                a = fminf(fminf(a, w2[2].y), w2[3].x); b = fmaxf(fmaxf(b, w2[2].y), w2[3].x);
+                float a = fmin3(w2[0].x, w2[0].y, w2[1].x), b = fmax3(w2[0].x, w2[0].y, w2[1].x);
+                a = fmin3(a, w2[1].y, w2[2].x); b = fmax3(b, w2[1].y, w2[2].x);
+                a = fmin3(a, w2[2].y, w2[3].x); b = fmax3(b, w2[2].y, w2[3].x);
                 a = fminf(a, w2[3].y); b = fmaxf(b, w2[3].y);
                 if (L == 16) {
                     // two groups per warp: a full-mask reduction per group with the other half's lanes
