@@ -15,7 +15,13 @@ resident in HBM before the timed region and are far larger than L2.
 The metric is layer-pass HBM GB/s: algorithmic bytes of the pass divided by its
 device time (CUDA events, max over ranks).  At one GPU the pass runs on two streams and the
 steps that carry no profiling hooks replay it from a CUDA graph (--eager, --no-overlap).  With N > 1 every rank calibrates
-its own token shard of the same layer (weak scaling, no data-path collective).
+its own token shard of the same layer (weak scaling); the one exchange of the method, the merge of the
+per-channel statistics over the ranks, is an all-reduce inside the timed step.
+
+After the headline region the default 1-GPU run also times, briefly, every other configuration (the same
+layer at 3 bits, the two OPT-125M cases, the LLaMA-13B layer, the OPT-66B FFN pair) and the forward check
+of two calibrated layers, and reports them under "workloads" / "forward_checks" of the same JSON line
+(--no-extras skips that).
 """
 from __future__ import annotations
 
@@ -98,13 +104,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def generate(wl: synth.Workload, device, rank: int):
-    X, W = {}, {}
-    for i, inp in enumerate(wl.inputs):
-        X[inp.name] = synth.make_activations(inp, wl.dtype, synth.tensor_seed(wl.seed, rank, i), device)
-    for i, lin in enumerate(wl.linears):
-        W[lin.name] = synth.make_weight(lin, wl.dtype, synth.tensor_seed(wl.seed, 0, 100 + i), device)
-    return X, W
+generate = synth.generate
 
 
 def oracle_pass(wl: synth.Workload, bits: int, Xb, Wb):
@@ -134,16 +134,30 @@ def cpu_sample(wl_full: synth.Workload, sample_tokens: int):
     return dataclasses.replace(wl_full, inputs=inputs)
 
 
+def workload_config(wl: synth.Workload, bits: int, world: int) -> dict:
+    """The ``config`` object of the JSON line: what is calibrated, the same for both arms."""
+    return {"workload": wl.name, "w_bits": bits, "w_gran": wl.w_gran, "group": wl.group,
+            "act_quant": wl.act_quant, "storage": wl.dtype, "tokens_per_gpu": wl.inputs[0].n_tokens,
+            "algorithmic_bytes_per_gpu": synth.algorithmic_bytes(wl, bits),
+            "cache": "inputs (GBs) far larger than the 126 MB L2",
+            "parallelism": "token shards, one per GPU" if world > 1 else "single GPU"}
+
+
+def sample_text(wl: synth.Workload, sample_tokens: int) -> str:
+    n = min(sample_tokens, wl.inputs[0].n_tokens)
+    return "first %d of %d tokens of every layer input, all weight matrices at full size" % (n, wl.inputs[0].n_tokens)
+
+
 def run_reference(args, wl, bits):
+    """The oracle arm: the CPU oracle alone (this process never loads the CUDA library)."""
     from oracle import aweq_oracle as orc
-    from paper_2311_01305_b200 import calibrate
     if int(os.environ.get("RANK", "0")) != 0:
         return
     swl = cpu_sample(wl, args.cpu_sample_tokens)
     X, W = generate(swl, "cpu", 0)
     Xb = {k: synth.raw_bits(v) for k, v in X.items()}
     Wb = {k: synth.raw_bits(v) for k, v in W.items()}
-    nbytes = calibrate_bytes(swl, bits)
+    nbytes = synth.algorithmic_bytes(swl, bits)
     for _ in range(args.warmup):
         oracle_pass(swl, bits, Xb, Wb)
     t0 = time.perf_counter()
@@ -151,12 +165,12 @@ def run_reference(args, wl, bits):
         oracle_pass(swl, bits, Xb, Wb)
     dt = (time.perf_counter() - t0) / args.steps
     gbs = nbytes / dt / 1e9
-    sample = "first %d tokens of every layer input, all weight matrices at full size" % args.cpu_sample_tokens
+    sample = sample_text(wl, args.cpu_sample_tokens)
     line = {
         "impl": "reference", "metric": "aweq_layer_pass_hbm_gbs", "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "w_bits": bits, "sample": sample},
+        "config": workload_config(wl, bits, max(1, args.gpus)),
         "tokens_per_s": swl.inputs[0].n_tokens / dt,
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": orc.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -165,44 +179,63 @@ def run_reference(args, wl, bits):
     print(json.dumps(line))
 
 
-def run_forward_check(args, wl, bits):
-    """Secondary benchmark: the forward check of every linear of a calibrated W8A8 layer.
-    A step is one check of the whole layer; the work is two dense contractions per linear
-    (unsigned 8-bit and 16-bit, 2 N C_in C_out flops each), so the bound is the tensor pipe.
-    The peak is the measured 16-bit GEMM rate scaled for the mix: the 8-bit half runs at
-    twice the 16-bit rate (nominal ratio), so 2F flops take at best 1.5 F / P16."""
+def gemm_peak():
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        try:
+            return float(json.load(open(pk))["bf16_tflops_sustained"]), "measured (sustained)"
+        except Exception:
+            pass
+    return FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def time_forward_check(wl, bits, X, W, steps, warmup):
+    """Forward check of every linear of the calibrated layer: (summary dict, last results, calibrator)."""
     from paper_2311_01305_b200 import aweq, calibrate
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
-    X, W = generate(wl, dev, 0)
     cal = calibrate.LayerCalibrator(wl, bits, X, W, None)
     cal.run()
-    for _ in range(max(1, args.warmup)):
+    res = None
+    for _ in range(max(1, warmup)):
         res = cal.forward_check(X, W)
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
     time.sleep(0.15)
     n0 = aweq.launch_count()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
-    for _ in range(args.steps):
+    for _ in range(steps):
         res = cal.forward_check(X, W)
     b.record()
     torch.cuda.synchronize()
     launches = aweq.launch_count() - n0
     clocks = sampler.stop()
-    ms = a.elapsed_time(b) / args.steps
+    ms = a.elapsed_time(b) / steps
     tokens = {i.name: i.n_tokens for i in wl.inputs}
     flops = sum(4.0 * tokens[l.input] * l.c_in * l.c_out for l in wl.linears)
-    p16 = FALLBACK_BF16_TFLOPS
-    kind = "fallback"
-    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(pk):
-        p16, kind = float(json.load(open(pk))["bf16_tflops_sustained"]), "measured (sustained)"
+    p16, kind = gemm_peak()
     w8a8 = wl.act_quant and bits == 8 and wl.w_gran == "row"
     peak = p16 * 2.0 / 1.5 if w8a8 else p16           # weight-only: both contractions are 16-bit
     tf = flops / ms / 1e9
+    out = {"ms_per_step": ms, "tflops": tf, "w8a8": w8a8, "launches": int(launches), "clocks": clocks,
+           "tokens": tokens, "steps": steps,
+           "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                        "peak_kind": ("16-bit GEMM rate of %s x 4/3 for the 8-bit / 16-bit mix" if w8a8
+                                      else "16-bit GEMM rate of %s") % kind, "traffic": None}}
+    return out, res, cal
+
+
+def run_forward_check(args, wl, bits):
+    """Secondary benchmark: the forward check of every linear of a calibrated layer.
+    A step is one check of the whole layer; the work is two dense contractions per linear
+    (2 N C_in C_out flops each), so the bound is the tensor pipe.  For W8A8 layers the peak is
+    the measured 16-bit GEMM rate scaled for the mix: the 8-bit half runs at twice the 16-bit
+    rate (nominal ratio), so 2F flops take at best 1.5 F / P16."""
+    from paper_2311_01305_b200 import aweq, calibrate
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    X, W = generate(wl, dev, 0)
+    fc, res, cal = time_forward_check(wl, bits, X, W, args.steps, args.warmup)
     worst = {n: float((me.abs().max() / (s4[1] / s4[3]).sqrt()).item()) for n, (me, s4) in res.items()}
     sqnr = {n: float(10.0 * torch.log10(s4[1] / s4[0]).item()) for n, (me, s4) in res.items()}
     # ablation (outside the timed region): equalisation and bias correction switched on and off
@@ -226,77 +259,33 @@ def run_forward_check(args, wl, bits):
                                                  for n, (me, s4) in r.items()}}
             del c, r
     print(json.dumps({
-        "metric": "aweq_forward_check_tflops", "value": tf, "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
-        "warmup": max(1, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": ("u8 x u8 -> s32 and %s -> f32" if w8a8 else "%s -> f32 (two contractions)") % wl.dtype,
+        "metric": "aweq_forward_check_tflops", "value": fc["tflops"], "unit": "TFLOP/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(1, args.warmup), "ms_per_step": fc["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": ("u8 x u8 -> s32 and %s -> f32" if fc["w8a8"] else "%s -> f32 (two contractions)") % wl.dtype,
         "data": "synthetic",
-        "config": {"workload": wl.name, "tokens": tokens, "linears": [l.name for l in wl.linears],
+        "config": {"workload": wl.name, "tokens": fc["tokens"], "linears": [l.name for l in wl.linears],
                    "cache": "operands (GBs) far larger than the 126 MB L2"},
-        "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
-                     "peak_kind": ("16-bit GEMM rate of %s x 4/3 for the 8-bit / 16-bit mix" if w8a8
-                                   else "16-bit GEMM rate of %s") % kind, "traffic": None},
-        "clocks": clocks, "gpu_launches": int(launches),
+        "roofline": fc["roofline"], "clocks": fc["clocks"], "gpu_launches": fc["launches"],
         "max_abs_mean_err_over_output_rms": worst, "output_sqnr_db": sqnr, "ablation": ablation}))
 
 
-def calibrate_bytes(wl, bits):
-    from paper_2311_01305_b200 import calibrate
-    return calibrate.algorithmic_bytes(wl, bits)
+# Measured share of the second read of W (step 4, after step 2 has streamed the same matrices) that
+# the L2 serves instead of HBM, per workload: ncu DRAM read bytes of the step-4 kernels of one pass
+# over their algorithmic read bytes, captured at 1/32 of the tokens (weights are full size at any
+# token count).  None = not captured for the kernels as they are now.
+W_SECOND_READ_FROM_L2 = {}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
-    ap.add_argument("--bits", type=int, default=0, help="weight bit-width (default: the workload's first)")
-    ap.add_argument("--tokens-scale", type=float, default=1.0, help="shrink the token count (profiling captures)")
-    ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
-    ap.add_argument("--no-overlap", action="store_true",
-                    help="issue every input's pass on one stream (default: two alternating streams)")
-    ap.add_argument("--eager", action="store_true",
-                    help="launch every timed step eagerly (default at 1 GPU: the steps that carry the event hooks "
-                         "are eager, the others replay the pass from a CUDA graph)")
-    ap.add_argument("--graph", action="store_true",
-                    help="replay the pass as one CUDA graph in the timed region (1 GPU; the dominant kernel is then "
-                         "timed in eager passes after it)")
-    ap.add_argument("--op", default="layer_pass", choices=["layer_pass", "forward_check"],
-                    help="forward_check: time the W8A8 forward check of the calibrated layer instead (1 GPU)")
-    args = ap.parse_args()
-
-    wl = synth.workloads(args.tokens_scale)[args.workload]
-    bits = args.bits or wl.w_bits[0]
-    if args.impl == "reference":
-        return run_reference(args, wl, bits)
-
-    from paper_2311_01305_b200 import build as _build
-    _build.build()                      # no-op when libaweq.so is up to date
+def time_layer_pass(wl, bits, X, W, steps, warmup, *, rank=0, world=1, local=0, dist=None,
+                    overlap=True, eager=False, graph_only=False):
+    """Times ``steps`` layer passes of one workload (CUDA events on the launching stream, max over
+    ranks) and, on every fourth of them, the dominant kernel through the library's event hooks.
+    Returns (calibrator, result dict)."""
     from paper_2311_01305_b200 import aweq, calibrate
-
-    if args.op == "forward_check":
-        return run_forward_check(args, wl, bits)
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the calibration pass has no CPU path")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-
-    X, W = generate(wl, dev, rank)
-    cal = (calibrate.ShardedLayerCalibrator(wl, bits, X, W, None) if world > 1
-           else calibrate.LayerCalibrator(wl, bits, X, W, None, overlap=not args.no_overlap))
-    nbytes = calibrate.algorithmic_bytes(wl, bits)
-    tokens = wl.inputs[0].n_tokens
+    dev = next(iter(X.values())).device
+    cal = (calibrate.ShardedLayerCalibrator(wl, bits, X, W, None, overlap=overlap) if world > 1
+           else calibrate.LayerCalibrator(wl, bits, X, W, None, overlap=overlap))
 
     def barrier():
         if dist is not None:
@@ -310,23 +299,23 @@ def main():
         return a, b
     # every fourth timed step carries the hooks (two event records per sweep cost 0.7 % of a pass, because
     # a record between two kernels undoes their programmatic overlap); the others run without them
-    hooked = [k for k in range(args.steps) if k % 4 == 0]
+    hooked = [k for k in range(steps) if k % 4 == 0]
     hooks = {k: [(ev_pair(), ev_pair() if wl.act_quant else None) for _ in cal.passes] for k in hooked}
     torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         cal.run()
     graph = None
-    if world == 1 and not args.eager:
+    if world == 1 and not eager:
         try:
             graph = cal.capture()           # without the event hooks: as graph nodes they cost 3 % of the pass
-            for _ in range(args.warmup):
+            for _ in range(warmup):
                 graph.replay()
         except Exception as exc:            # a capture that fails leaves the eager pass as it was
             sys.stderr.write("CUDA graph capture failed (%s); timing eager launches\n" % exc)
             graph = None
             torch.cuda.synchronize()
-    mixed = graph is not None and not args.graph
+    mixed = graph is not None and not graph_only
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
@@ -335,32 +324,28 @@ def main():
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     t_begin.record()
-    for k in range(args.steps):
-        if world > 1:
-            names = [i.name for i in wl.inputs if i.name in cal.out]
-            cal.events = {n: h for n, h in zip(names, hooks[k])} if k in hooks else None
-            cal.run()                       # statistics merged over the ranks inside the step
-        elif graph is not None and not (mixed and k in hooks):
+    for k in range(steps):
+        if graph is not None and not (mixed and k in hooks):
             graph.replay()
         else:
             for i, lp in enumerate(cal.passes):
                 es, ea = hooks[k][i] if k in hooks else (None, None)
                 lp.set_events(es, ea)
-            cal.run()
+            cal.run()                       # N > 1: the statistics are merged over the ranks inside the step
     t_end.record()
     barrier()
     launches = aweq.launch_count() - n0
     clocks = sampler.stop()
     if mixed:
         # replays go through no library call: a replay launches what an eager step launches
-        launches = launches // len(hooks) * args.steps
+        launches = launches // len(hooks) * steps
     elif graph is not None:
         # replays go through no library call: a replay launches what one eager pass launches.  The
         # dominant kernel is timed in eager passes after the timed region (hooks inside the graph
         # would be recorded by every replay, but as graph nodes of their own they slow it down).
         torch.cuda.synchronize()
         n1 = aweq.launch_count()
-        for k in range(args.steps):
+        for k in range(steps):
             for i, lp in enumerate(cal.passes):
                 es, ea = hooks[k][i] if k in hooks else (None, None)
                 lp.set_events(es, ea)
@@ -369,9 +354,7 @@ def main():
         launches = aweq.launch_count() - n1
     for lp in cal.passes:
         lp.set_events(None, None)
-    if world > 1:
-        cal.events = None
-    ms = t_begin.elapsed_time(t_end) / args.steps
+    ms = t_begin.elapsed_time(t_end) / steps
     if dist is not None:
         t = torch.tensor([ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -388,41 +371,151 @@ def main():
     if wl.act_quant:
         act_ms = [sum(ea[0].elapsed_time(ea[1]) for _, ea in hk) for hk in hooks.values()]
         act_bytes = sum(3 * i.n_tokens * i.c_in + 8 * i.n_tokens for i in wl.inputs)
-        dom = {"kernel": "rowquant_kernel / rowquant_wide_kernel (aweq_quant_act)", "bytes": act_bytes, "ms": statistics.mean(act_ms),
-               "launches_per_step": len(cal.passes), "stats_gbs": stats_bytes / statistics.mean(stats_ms) / 1e6}
+        dom = {"kernel": "rowquant_kernel / rowquant_wide_kernel (aweq_quant_act)", "bytes": act_bytes,
+               "ms": statistics.mean(act_ms), "launches_per_step": len(cal.passes),
+               "stats_gbs": stats_bytes / statistics.mean(stats_ms) / 1e6}
     peak, peak_kind = measured_peaks()
     achieved = dom["bytes"] / dom["ms"] / 1e6
-    # DRAM traffic per launch from the ncu counters summarised in
-    # profiles/stats_and_groupquant_llama7b_small.md (current kernel, 1/8 of the rows: reads are
-    # 1.0001 x the algorithmic bytes and scale with the rows; the per-split partials, at most
-    # 4.4 MB, do not).  Only the statistics kernel has counters that cover its whole output.
-    traffic = None
-    if not wl.act_quant:
-        traffic = (dom["bytes"] / dom["launches_per_step"]) * 1.0001 + 4.4e6
     roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
+                "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": None,
                 "launch_ms": dom["ms"] / dom["launches_per_step"], "timed_steps": sorted(hooks.keys()),
                 "bytes_per_launch": dom["bytes"] / dom["launches_per_step"]}
     if "stats_gbs" in dom:
         roofline["stats_gbs"] = dom["stats_gbs"]
-
+    nbytes = synth.algorithmic_bytes(wl, bits)
     gbs = world * nbytes / ms / 1e6
+    l2 = W_SECOND_READ_FROM_L2.get((wl.name, bits))
+    roofline["w_second_read_from_l2"] = l2
+    res = {"ms": ms, "gbs": gbs, "nbytes": nbytes, "launches": int(launches), "clocks": clocks, "status": status,
+           "roofline": roofline, "peak": peak,
+           "gbs_hbm_basis": None if l2 is None else world * (nbytes - l2 * synth.weight_bytes(wl)) / ms / 1e6,
+           "launch": ("CUDA graph replay; every fourth step eager, with the event hooks" if mixed
+                      else "one CUDA graph replay per step" if graph is not None else "eager"),
+           "schedule": ("two streams: column reductions and step 6 on one, factors and weight quantiser on the other"
+                        if getattr(cal, "overlap", False) else "one stream")}
+    return cal, res
+
+
+EXTRA_WORKLOADS = (("llama7b_layer_w4w3_g128", 3), ("opt125m_linear_w8a8", 8), ("opt125m_model_w8a8", 8),
+                   ("llama13b_layer_w8a8", 8), ("opt66b_ffn_w8a8", 8))
+EXTRA_FORWARD_CHECKS = (("llama7b_layer_w4w3_g128", 4), ("llama13b_layer_w8a8", 8))
+
+
+def run_extras(args, dev, skip):
+    """Every configuration other than the headline one, timed briefly on the same box with the same
+    code as the headline region (one GPU), and the forward check of two calibrated layers."""
+    table, checks = {}, {}
+    wls = synth.workloads(args.tokens_scale)
+    fc_of = dict(EXTRA_FORWARD_CHECKS)
+    for name, bits in EXTRA_WORKLOADS:
+        if (name, bits) == skip:
+            continue
+        wl = wls[name]
+        X, W = generate(wl, dev, 0)
+        cal, r = time_layer_pass(wl, bits, X, W, args.extra_steps, args.warmup, overlap=not args.no_overlap,
+                                 eager=args.eager, graph_only=args.graph)
+        rf = r["roofline"]
+        table["%s@w%d" % (name, bits)] = {
+            "bits": bits, "ms_per_step": r["ms"], "gbs": r["gbs"], "gbs_hbm_basis": r["gbs_hbm_basis"],
+            "pct_of_8000_gbs": 100.0 * r["gbs"] / NOMINAL_HBM_GBS,
+            "pct_of_measured_copy": 100.0 * r["gbs"] / r["peak"], "tokens_per_s": wl.inputs[0].n_tokens / (r["ms"] / 1e3),
+            "algorithmic_bytes": r["nbytes"], "steps": args.extra_steps, "gpu_launches": r["launches"],
+            "dominant_kernel": rf["kernel"], "frac": rf["frac"], "dominant_gbs": rf["achieved"],
+            "stats_gbs": rf.get("stats_gbs", rf["achieved"]), "launch": r["launch"],
+            "sm_mhz": r["clocks"].get("sm_mhz"), "reasons": r["clocks"].get("reasons")}
+        del cal
+        if fc_of.get(name) == bits and not args.no_forward_check:
+            fc, res, cal = time_forward_check(wl, bits, X, W, 2, 1)
+            checks["%s@w%d" % (name, bits)] = {
+                "ms_per_step": fc["ms_per_step"], "tflops": fc["tflops"], "frac": fc["roofline"]["frac"],
+                "peak": fc["roofline"]["peak"], "peak_kind": fc["roofline"]["peak_kind"], "steps": fc["steps"],
+                "gpu_launches": fc["launches"], "sm_mhz": fc["clocks"].get("sm_mhz"),
+                "reasons": fc["clocks"].get("reasons"),
+                "output_sqnr_db": {n: round(float(10.0 * torch.log10(s4[1] / s4[0]).item()), 3)
+                                   for n, (me, s4) in res.items()}}
+            del cal, res
+        del X, W
+        torch.cuda.empty_cache()
+    return table, checks
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--bits", type=int, default=0, help="weight bit-width (default: the workload's first)")
+    ap.add_argument("--tokens-scale", type=float, default=1.0, help="shrink the token count (profiling captures)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-tokens", type=int, default=262144)
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the short timed passes of the other configurations after the headline region")
+    ap.add_argument("--extra-steps", type=int, default=8, help="timed steps of each of those passes")
+    ap.add_argument("--no-forward-check", action="store_true", help="leave the forward checks out of the extras")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="issue every input's pass on one stream (default: two alternating streams)")
+    ap.add_argument("--eager", action="store_true",
+                    help="launch every timed step eagerly (default at 1 GPU: the steps that carry the event hooks "
+                         "are eager, the others replay the pass from a CUDA graph)")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the pass as one CUDA graph in the timed region (1 GPU; the dominant kernel is then "
+                         "timed in eager passes after it)")
+    ap.add_argument("--op", default="layer_pass", choices=["layer_pass", "forward_check"],
+                    help="forward_check: time the forward check of the calibrated layer instead (1 GPU)")
+    args = ap.parse_args()
+
+    wl = synth.workloads(args.tokens_scale)[args.workload]
+    bits = args.bits or wl.w_bits[0]
+    if args.impl == "reference":
+        return run_reference(args, wl, bits)
+
+    from paper_2311_01305_b200 import build as _build
+    _build.build()                      # no-op when libaweq.so is up to date
+    from paper_2311_01305_b200 import aweq  # noqa: F401  (fails loudly when the library is missing)
+
+    if args.op == "forward_check":
+        return run_forward_check(args, wl, bits)
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the calibration pass has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    X, W = generate(wl, dev, rank)
+    cal, r = time_layer_pass(wl, bits, X, W, args.steps, args.warmup, rank=rank, world=world, local=local, dist=dist,
+                             overlap=not args.no_overlap, eager=args.eager, graph_only=args.graph)
+    ms, gbs, nbytes, peak = r["ms"], r["gbs"], r["nbytes"], r["peak"]
+    tokens = wl.inputs[0].n_tokens
     line = {
         "metric": "aweq_layer_pass_hbm_gbs", "value": gbs, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "w_bits": bits, "w_gran": wl.w_gran, "group": wl.group,
-                   "act_quant": wl.act_quant, "storage": wl.dtype, "tokens_per_gpu": tokens,
-                   "algorithmic_bytes_per_gpu": nbytes, "cache": "inputs (GBs) far larger than the 126 MB L2",
-                   "parallelism": "token shards, one per GPU" if world > 1 else "single GPU",
-                   "launch": ("CUDA graph replay; every fourth step eager, with the event hooks" if mixed
-                              else "one CUDA graph replay per step" if graph is not None else "eager"),
-                   "schedule": ("two streams: column reductions and step 6 on one, factors and weight quantiser on the other"
-                                if getattr(cal, "overlap", False) else "one stream")},
+        "config": workload_config(wl, bits, world),
+        "launch_config": {"launch": r["launch"], "schedule": r["schedule"]},
         "tokens_per_s": world * tokens / (ms / 1e3),
         "pct_of_8000_gbs": 100.0 * gbs / world / NOMINAL_HBM_GBS,
         "pct_of_measured_copy": 100.0 * gbs / world / peak,
-        "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "device_status": status,
+        "value_hbm_basis": r["gbs_hbm_basis"],
+        "basis_note": ("value counts every algorithmic byte, including the second read of W, part of which the L2 "
+                       "serves (roofline.w_second_read_from_l2); value_hbm_basis leaves that part out. A percentage "
+                       "of the measured copy bandwidth above 100 is a read-mostly stream against a read+write copy, "
+                       "not more than the HBM can deliver"),
+        "roofline": r["roofline"], "clocks": r["clocks"], "gpu_launches": r["launches"], "device_status": r["status"],
     }
 
     # ---------------------------------------------------------------- end to end: host buffers in, results out
@@ -439,9 +532,9 @@ def main():
         def e2e_step():
             for k, v in hostW.items():
                 W[k].copy_(v, non_blocking=True)
-            for lp, inp in zip(cal.passes, [i for i in wl.inputs if i.name in cal.out]):
-                X[inp.name].copy_(hostX[inp.name], non_blocking=True)
-                lp(cal.ws, cal.status)
+            for k, v in hostX.items():
+                X[k].copy_(v, non_blocking=True)
+            cal.run()
             for n, d in host_out.items():
                 for k, t in d.items():
                     t.copy_(cal.out[n][k], non_blocking=True)
@@ -471,11 +564,17 @@ def main():
         t0 = time.perf_counter()
         oracle_pass(swl, bits, Xb, Wb)
         dt = time.perf_counter() - t0
-        sbytes = calibrate.algorithmic_bytes(swl, bits)
+        sbytes = synth.algorithmic_bytes(swl, bits)
         line["cpu_baseline"] = {"value": sbytes / dt / 1e9, "unit": "GB/s", "cores": orc.threads(), "kind": "oracle",
                                 "seconds": dt, "tokens_per_s": swl.inputs[0].n_tokens / dt,
-                                "sample": "first %d tokens of every layer input, all weight matrices at full size"
-                                          % args.cpu_sample_tokens}
+                                "sample": sample_text(wl, args.cpu_sample_tokens)}
+        del Xb, Wb
+
+    # ---------------------------------------------------------------- the other configurations, briefly
+    if world == 1 and not args.no_extras:
+        del cal, X, W
+        torch.cuda.empty_cache()
+        line["workloads"], line["forward_checks"] = run_extras(args, dev, (wl.name, bits))
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

@@ -280,6 +280,11 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
 #define AWEQ_FLAG_PHASE_QUANT 8
 #define AWEQ_FLAG_PHASE_ACT 16
 #define AWEQ_FLAG_ABSMAX_CRITERION 32   /* step 3 through aweq_factors_absmax (comparison criterion) */
+/* Token-sharded calibration (Section 3.3: the statistics are over all N inputs, wherever they
+ * are held): the QUANT part first re-forms xmin, xmax and xmean = sum / count from the exchange
+ * buffers stat_negmin_max / stat_sum_count of the argument block, which the caller has merged
+ * over the shards between the REDUCE and the QUANT part (one MAX and one SUM all-reduce). */
+#define AWEQ_FLAG_MERGED_STATS 64
 
 typedef struct {
     /* input */
@@ -300,6 +305,13 @@ typedef struct {
     /* optional profiling hooks: cudaEvent_t handles (or NULL) recorded on `stream`
      * immediately before and after step 1 and step 6 */
     void *ev_stats_begin, *ev_stats_end, *ev_act_begin, *ev_act_end;
+    /* optional exchange form of the step-1 statistics, both or neither; when given, the REDUCE
+     * part also writes
+     *   stat_negmin_max = float[2 C_in]   = { -xmin_j (j < C_in), xmax_j (j < C_in) }
+     *   stat_sum_count  = double[C_in + 1] = { sum_n X[n,j] (j < C_in), N }
+     * so that an element-wise MAX of the first and SUM of the second over several token shards
+     * are the statistics of their union (see AWEQ_FLAG_MERGED_STATS) */
+    float *stat_negmin_max; double *stat_sum_count;
 } aweq_layer_args;
 
 size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args);

@@ -31,6 +31,7 @@ OP_STATS, OP_WRANGE, OP_EQUALIZE_QUANTIZE, OP_BIAS_CORRECT, OP_QUANT_ACT = 1, 2,
 FLAG_NO_EQUALIZE, FLAG_NO_BIAS_CORRECT = 1, 2
 FLAG_PHASE_REDUCE, FLAG_PHASE_QUANT, FLAG_PHASE_ACT = 4, 8, 16
 FLAG_ABSMAX_CRITERION = 32
+FLAG_MERGED_STATS = 64
 
 _vp, _ll, _i, _sz = ctypes.c_void_p, ctypes.c_longlong, ctypes.c_int, ctypes.c_size_t
 
@@ -52,6 +53,7 @@ class LayerArgs(ctypes.Structure):
         ("mu_hat", _vp), ("pX", _vp), ("pW", _vp), ("scalars", _vp),
         ("Xq", _vp), ("act_step", _vp), ("act_zp", _vp), ("act_bits", _i), ("flags", _i),
         ("ev_stats_begin", _vp), ("ev_stats_end", _vp), ("ev_act_begin", _vp), ("ev_act_end", _vp),
+        ("stat_negmin_max", _vp), ("stat_sum_count", _vp),
     ]
 
 
@@ -302,10 +304,10 @@ class LayerPass:
 
     def __init__(self, X, Ws, bits, gran, group, codes, step, zp, epsmu, bias_in, bias_out, bias_out_f32,
                  xmin, xmax, xmean, wmin, wmax, s, rinv, mu_hat, pX=None, pW=None, scalars=None,
-                 Xq=None, act_step=None, act_zp=None, act_bits=8, flags=0):
+                 Xq=None, act_step=None, act_zp=None, act_bits=8, flags=0, stat_negmin_max=None, stat_sum_count=None):
         n = len(Ws)
         self._keep = (X, Ws, codes, step, zp, epsmu, bias_in, bias_out, bias_out_f32, xmin, xmax, xmean, wmin, wmax,
-                      s, rinv, mu_hat, pX, pW, scalars, Xq, act_step, act_zp)
+                      s, rinv, mu_hat, pX, pW, scalars, Xq, act_step, act_zp, stat_negmin_max, stat_sum_count)
         a = LayerArgs()
         a.X, a.dt, a.N, a.C_in, a.ldx = _ptr(X), dtype_tag(X), X.shape[0], X.shape[1], _ld(X)
         a.n_w = n
@@ -318,7 +320,8 @@ class LayerPass:
                 setattr(a, k, v)
         a.bits, a.gran, a.group = bits, gran, group
         for k, v in dict(xmin=xmin, xmax=xmax, xmean=xmean, wmin=wmin, wmax=wmax, s=s, rinv=rinv, mu_hat=mu_hat,
-                         pX=pX, pW=pW, scalars=scalars, Xq=Xq, act_step=act_step, act_zp=act_zp).items():
+                         pX=pX, pW=pW, scalars=scalars, Xq=Xq, act_step=act_step, act_zp=act_zp,
+                         stat_negmin_max=stat_negmin_max, stat_sum_count=stat_sum_count).items():
             setattr(a, k, _ptr(v))
         a.act_bits, a.flags = act_bits, flags
         self.args = a

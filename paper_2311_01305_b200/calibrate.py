@@ -18,33 +18,37 @@ import torch.distributed as dist
 from . import aweq, synth
 
 
-def algorithmic_bytes(wl: synth.Workload, bits: int) -> int:
-    """Bytes one layer pass must move: X once for the statistics; every W once
-    for its column ranges and once more, plus the packed codes and the
-    (Step, Z) pairs, for the fused rescale-quantise-pack; for W8A8 X a second
-    time plus one byte per element and a (Step, Z) pair per token."""
-    total = 0
+algorithmic_bytes = synth.algorithmic_bytes
+
+
+def exchange_layout(wl: synth.Workload):
+    """Where each fed input's statistics sit in the two flat exchange buffers of a token-sharded
+    pass: ({input name: (offset into the float32 buffer, offset into the float64 buffer)},
+    float32 elements, float64 elements).  An input with C_in channels takes 2 C_in floats
+    ({-xmin, xmax}) and C_in + 1 doubles ({column sums, token count}) plus one pad double, so
+    every slice starts on a 16-byte boundary.  Sizes only."""
+    off, mm, sc = {}, 0, 0
     for inp in wl.inputs:
-        total += 2 * inp.n_tokens * inp.c_in
-        if wl.act_quant:
-            total += 3 * inp.n_tokens * inp.c_in + 8 * inp.n_tokens
-    for lin in wl.linears:
-        n = lin.c_out * lin.c_in
-        pairs = lin.c_out if wl.w_gran == "row" else lin.c_out * (lin.c_in // wl.group)
-        total += 2 * n + 2 * n + n * bits // 8 + 8 * pairs
-    return total
+        if any(l.input == inp.name for l in wl.linears):
+            off[inp.name] = (mm, sc)
+            mm += 2 * inp.c_in
+            sc += inp.c_in + 2
+    return off, mm, sc
 
 
 class LayerCalibrator:
     def __init__(self, wl: synth.Workload, bits: int, X: Dict[str, torch.Tensor], W: Dict[str, torch.Tensor],
                  bias: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0, diagnostics: bool = True,
-                 overlap: bool = False):
+                 overlap: bool = False, exchange_buffers: bool = False):
         """``overlap``: split every pass into its parts (``FLAG_PHASE_*``) and issue the
         shared-memory-staged, HBM-bound kernels (the column reductions of steps 1-2 and step 6) on
         one CUDA stream and the short, issue-bound kernels that need no shared memory (factors,
         weight quantiser: steps 3-5) on another, each with its own scratch and ordered by events,
         so that the weight kernels of one input run beside the statistics sweep of the next;
-        ``run()`` forks from and joins back into the current stream."""
+        ``run()`` forks from and joins back into the current stream.
+        ``exchange_buffers``: give every pass the exchange form of its statistics (one flat
+        ``float32`` buffer {-xmin, xmax} and one flat ``float64`` buffer {sums, count} over all
+        inputs; see ``ShardedLayerCalibrator``)."""
         self.wl, self.bits = wl, bits
         dev = next(iter(X.values())).device
         td = synth.torch_dtype(wl.dtype)
@@ -53,10 +57,16 @@ class LayerCalibrator:
         self.out: Dict[str, Dict[str, torch.Tensor]] = {}
         self.passes: List[aweq.LayerPass] = []
         ws_bytes = 256
-        for inp in wl.inputs:
+        fed = [i for i in wl.inputs if any(l.input == i.name for l in wl.linears)]
+        self.stat_negmin_max = self.stat_sum_count = None
+        self._slices = []
+        if exchange_buffers:
+            layout, n_mm, n_sc = exchange_layout(wl)
+            self.stat_negmin_max = torch.empty(n_mm, **f32)
+            self.stat_sum_count = torch.zeros(n_sc, dtype=torch.float64, device=dev)
+            flags |= aweq.FLAG_MERGED_STATS
+        for inp in fed:
             lins = [l for l in wl.linears if l.input == inp.name]
-            if not lins:
-                continue
             x = X[inp.name]
             C = inp.c_in
             o = {k: torch.empty(C, **f32) for k in ("xmin", "xmax", "xmean", "wmin", "wmax", "s", "rinv", "mu_hat")}
@@ -68,6 +78,12 @@ class LayerCalibrator:
                 o["Xq"] = torch.empty((x.shape[0], C), dtype=torch.uint8, device=dev)
                 o["act_step"] = torch.empty(x.shape[0], **f32)
                 o["act_zp"] = torch.empty(x.shape[0], dtype=torch.int32, device=dev)
+            mm = sc = None
+            if exchange_buffers:
+                mm_off, sc_off = layout[inp.name]
+                mm = self.stat_negmin_max[mm_off:mm_off + 2 * C]
+                sc = self.stat_sum_count[sc_off:sc_off + C + 1]
+                self._slices.append((mm, sc))
             self.out[inp.name] = o
             codes, step, zp, epsmu, b_in, b_out, b_out32 = [], [], [], [], [], [], []
             for l in lins:
@@ -88,7 +104,7 @@ class LayerCalibrator:
                 x, [W[l.name] for l in lins], bits, gran, wl.group, codes, step, zp, epsmu, b_in, b_out, b_out32,
                 o["xmin"], o["xmax"], o["xmean"], o["wmin"], o["wmax"], o["s"], o["rinv"], o["mu_hat"],
                 o.get("pX"), o.get("pW"), o.get("scalars"), o.get("Xq"), o.get("act_step"), o.get("act_zp"), 8,
-                flags)
+                flags, mm, sc)
             ws_bytes = max(ws_bytes, lp.ws_bytes)
             self.passes.append(lp)
         self.ws = aweq.workspace(ws_bytes, dev)
@@ -103,11 +119,23 @@ class LayerCalibrator:
         self._fc_ws, self._fc_out = None, {}
         self.equalized = not (flags & aweq.FLAG_NO_EQUALIZE)
 
+    def _exchange(self, i: int) -> None:
+        """Between the REDUCE and the QUANT part of pass ``i``, on the stream that runs QUANT:
+        nothing for a single device (see ``ShardedLayerCalibrator``)."""
+
+    _split_parts = False            # a subclass with an exchange must run the parts separately
+
     def run(self) -> None:
-        """One calibration pass of the whole layer: one library call per input."""
+        """One calibration pass of the whole layer: one library call per input (or one per part
+        of every input, when the parts go to two streams)."""
         if not self.overlap:
-            for lp in self.passes:
-                lp(self.ws, self.status)
+            for i, lp in enumerate(self.passes):
+                if self._split_parts:
+                    lp(self.ws, self.status, aweq.FLAG_PHASE_REDUCE)
+                    self._exchange(i)
+                    lp(self.ws, self.status, aweq.FLAG_PHASE_QUANT | aweq.FLAG_PHASE_ACT)
+                else:
+                    lp(self.ws, self.status)
             return
         cur = torch.cuda.current_stream()
         big, small = self._streams
@@ -126,6 +154,7 @@ class LayerCalibrator:
         for i, lp in enumerate(self.passes):
             with torch.cuda.stream(small):
                 small.wait_event(self._ev_stats[i])
+                self._exchange(i)                  # sharded: beside the next input's sweep
                 lp(ws_small, self.status, aweq.FLAG_PHASE_QUANT)
                 self._ev_weights[i].record(small)
             if i + 1 < n:
@@ -247,75 +276,31 @@ class DecoderWalk:
                 "norms": self.norms, "folded": list(self.folded)}
 
 
-def allreduce_stats(xmin: torch.Tensor, xmax: torch.Tensor, xsum: torch.Tensor, count: torch.Tensor, group=None) -> None:
-    """The one exchange of a token-sharded calibration pass: per-channel minima, maxima,
-    binary64 sums and the token count of all ranks are merged in place (min / max / sum /
-    sum).  Works on any backend (NCCL on GPUs, gloo on CPU tensors)."""
-    dist.all_reduce(xmin, op=dist.ReduceOp.MIN, group=group)
-    dist.all_reduce(xmax, op=dist.ReduceOp.MAX, group=group)
-    dist.all_reduce(xsum, op=dist.ReduceOp.SUM, group=group)
-    dist.all_reduce(count, op=dist.ReduceOp.SUM, group=group)
+def exchange_stats(negmin_max: torch.Tensor, sum_count: torch.Tensor, group=None) -> None:
+    """The one exchange of a token-sharded calibration pass, in place, on any backend (NCCL on
+    GPUs, gloo on CPU tensors): ``negmin_max`` = {-xmin_j, xmax_j} merges with an element-wise
+    MAX, ``sum_count`` = {binary64 column sums, token count} with a SUM."""
+    dist.all_reduce(negmin_max, op=dist.ReduceOp.MAX, group=group)
+    dist.all_reduce(sum_count, op=dist.ReduceOp.SUM, group=group)
 
 
 class ShardedLayerCalibrator(LayerCalibrator):
-    """Token-sharded pass: every rank holds its own N tokens of each layer input and a
-    replica of the weights.  Step 1 runs on the local shard, the statistics are merged
-    with ``allreduce_stats`` (3 C_in values per channel plus one count), the mean is
-    re-formed from the merged sums by the library (an empty ``aweq_stats`` call in
-    accumulate mode), steps 2-5 run replicated and step 6 on the local shard."""
+    """Token-sharded pass: every rank holds its own N tokens of each layer input and a replica
+    of the weights.  It is the pass of ``LayerCalibrator`` -- same library calls, same two-stream
+    schedule -- with one exchange per input between its REDUCE and its QUANT part: the REDUCE
+    part leaves the shard's statistics in exchange form, ``exchange_stats`` merges them over the
+    ranks (two all-reduces of 2 C_in floats and C_in + 1 doubles), and the QUANT part re-forms
+    min / max / mean of the whole calibration set from the merged buffers
+    (``FLAG_MERGED_STATS``).  With two streams the exchange sits on the stream of the weight
+    kernels, so it runs beside the next input's sweep and only the last one is exposed.  Steps
+    2-5 are replicated (W is a few per cent of the bytes); step 6 works on the local shard."""
 
-    def __init__(self, wl, bits, X, W, bias=None, flags=0, group=None):
-        super().__init__(wl, bits, X, W, bias, flags, diagnostics=True)
+    _split_parts = True
+
+    def __init__(self, wl, bits, X, W, bias=None, flags=0, group=None, overlap=False):
+        super().__init__(wl, bits, X, W, bias, flags, diagnostics=True, overlap=overlap, exchange_buffers=True)
         self.group = group
-        self.events = None          # optional {input name: (stats pair, act pair)} of torch.cuda.Event to record
-        self._X, self._W, self._bias, self._flags = X, W, bias, flags
-        dev = self.ws.device
-        for inp in wl.inputs:
-            if inp.name in self.out:
-                o = self.out[inp.name]
-                o["xsum"] = torch.empty(inp.c_in, dtype=torch.float64, device=dev)
-                o["count"] = torch.zeros(1, dtype=torch.int64, device=dev)
 
-    def run(self) -> None:
-        wl, bits = self.wl, self.bits
-        gran = aweq.PER_ROW if wl.w_gran == "row" else aweq.PER_GROUP
-        dt = aweq.F16 if wl.dtype == "f16" else aweq.BF16
-        eq = not (self._flags & aweq.FLAG_NO_EQUALIZE)
-        bc = not (self._flags & aweq.FLAG_NO_BIAS_CORRECT)
-        for inp in wl.inputs:
-            lins = [l for l in wl.linears if l.input == inp.name]
-            if not lins:
-                continue
-            x, o = self._X[inp.name], self.out[inp.name]
-            ev = self.events.get(inp.name) if self.events else None
-            if ev:
-                ev[0][0].record()
-            aweq.aweq_stats(x, o["xmin"], o["xmax"], o["xmean"], xsum=o["xsum"], count=o["count"], ws=self.ws,
-                            st=self.status)
-            if ev:
-                ev[0][1].record()
-            allreduce_stats(o["xmin"], o["xmax"], o["xsum"], o["count"], self.group)
-            aweq.aweq_stats(x, o["xmin"], o["xmax"], o["xmean"], xsum=o["xsum"], count=o["count"], accumulate=True,
-                            ws=self.ws, st=self.status, N=0)
-            for i, l in enumerate(lins):
-                aweq.aweq_wrange(self._W[l.name], o["wmin"], o["wmax"], accumulate=i > 0, ws=self.ws, st=self.status)
-            aweq.aweq_factors(o["xmin"], o["xmax"], o["xmean"], o["wmin"], o["wmax"], o["s"], o["rinv"], o["mu_hat"],
-                              o.get("pX"), o.get("pW"), o.get("scalars"), st=self.status)
-            s = o["s"] if eq else None
-            mu = o["mu_hat"] if eq else o["xmean"]
-            for l in lins:
-                lo = self.out[l.name]
-                aweq.aweq_equalize_quantize(self._W[l.name], s, mu if bc else None, bits, gran, wl.group, lo["codes"],
-                                            lo["step"], lo["zp"], lo["epsmu"] if bc else None, ws=self.ws,
-                                            st=self.status)
-                if bc:
-                    b_in = None if self._bias is None else self._bias.get(l.name)
-                    aweq.aweq_bias_correct(lo["epsmu"], None, None, None, None, None, None, bits, gran, wl.group,
-                                           b_in, lo["bias"], lo["bias_f32"], dt)
-            if wl.act_quant:
-                if ev:
-                    ev[1][0].record()
-                aweq.aweq_quant_act(x, o["rinv"] if eq else None, 8, aweq.PER_ROW, None, o["Xq"], o["act_step"],
-                                    o["act_zp"], st=self.status)
-                if ev:
-                    ev[1][1].record()
+    def _exchange(self, i: int) -> None:
+        mm, sc = self._slices[i]
+        exchange_stats(mm, sc, self.group)

@@ -98,7 +98,7 @@ const char *aweq_strerror(aweq_status code)
 }
 
 const char *aweq_last_cuda_error(void) { return g_cuda_error; }
-int aweq_version(void) { return 100; }
+int aweq_version(void) { return 101; }
 unsigned long long aweq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 aweq_status aweq_plan_query(int op, long long rows, long long cols, long long plan[8])
@@ -325,6 +325,9 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
         if (!(a->bias_out && a->bias_out[i]) && !(a->bias_out_f32 && a->bias_out_f32[i])) return AWEQ_ERR_NULL;
     }
     if (a->Xq && (!a->act_step || !a->act_zp)) return AWEQ_ERR_NULL;
+    if ((a->stat_negmin_max == nullptr) != (a->stat_sum_count == nullptr)) return AWEQ_ERR_NULL;
+    if ((a->flags & AWEQ_FLAG_MERGED_STATS) && !a->stat_negmin_max) return AWEQ_ERR_NULL;
+    if (a->stat_negmin_max && (!aligned(a->stat_negmin_max, 4) || !aligned(a->stat_sum_count, 8))) return AWEQ_ERR_ALIGN;
     size_t col_part = 0;
     const size_t need = layer_ws_parts(a, &col_part);
     rc = check_ws(ws, ws_bytes, need);
@@ -340,8 +343,16 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     // steps 1-2
     if (phases & AWEQ_FLAG_PHASE_REDUCE) {
         if (a->ev_stats_begin) AWEQ_CUDA_OK(record_hook(a->ev_stats_begin, cs));
-        rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
-                        col_part, st, stream);
+        if (a->stat_negmin_max) {
+            // aweq_stats' checks, then the sweep that also leaves the exchange form of the statistics
+            if (!aligned(a->xmin, 16) || !aligned(a->xmax, 16) || !aligned(a->xmean, 4)) return AWEQ_ERR_ALIGN;
+            AWEQ_LOGF("aweq_stats N=%lld C_in=%lld (with exchange buffers) bytes=%lld\n", a->N, a->C_in, 2 * a->N * a->C_in);
+            rc = run_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col, st,
+                           cs, a->stat_negmin_max, a->stat_sum_count);
+        } else {
+            rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
+                            col_part, st, stream);
+        }
         if (rc != AWEQ_OK) return rc;
         if (a->ev_stats_end) AWEQ_CUDA_OK(record_hook(a->ev_stats_end, cs));
         // step 2: the matrices share the input, hence one range per input channel over all of them
@@ -355,6 +366,10 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     const float *rinv_used = eq ? a->rinv : nullptr;
     const float *mu_used = eq ? a->mu_hat : a->xmean;
     if (phases & AWEQ_FLAG_PHASE_QUANT) {
+    if (a->flags & AWEQ_FLAG_MERGED_STATS) {
+        rc = run_stats_from_exchange(a->stat_negmin_max, a->stat_sum_count, a->C_in, a->xmin, a->xmax, a->xmean, cs);
+        if (rc != AWEQ_OK) return rc;
+    }
     // step 3
     rc = ((a->flags & AWEQ_FLAG_ABSMAX_CRITERION) ? aweq_factors_absmax : aweq_factors)(
         a->xmin, a->xmax, a->xmean, a->wmin, a->wmax, a->C_in, a->s, a->rinv, a->mu_hat, a->pX, a->pW, a->scalars, st,

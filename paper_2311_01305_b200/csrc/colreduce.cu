@@ -365,11 +365,12 @@ __global__ void __launch_bounds__(kFinCols * kFinLanes)
 colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restrict__ pmax,
                           const double *__restrict__ psum, int nsplit, long long cols, long long nrows, float *omin,
                           float *omax, float *omean, double *osum, const long long *count, int accumulate,
-                          aweq_dev_status *st)
+                          aweq_dev_status *st, float *negmin_max, double *count_f64)
 {
     __shared__ float slo[kFinLanes][kFinCols], shi[kFinLanes][kFinCols];
     __shared__ double ssum[kFinLanes][kFinCols];
     pdl_begin();
+    if (count_f64 && blockIdx.x == 0 && threadIdx.x == 0) *count_f64 = (double)nrows;
     const int c = threadIdx.x % kFinCols, k0 = threadIdx.x / kFinCols;
     const long long j = (long long)blockIdx.x * kFinCols + c;
     float lo = INFINITY, hi = -INFINITY;
@@ -402,6 +403,10 @@ colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restric
     }
     omin[j] = lo;
     omax[j] = hi;
+    if (negmin_max) {                       // exchange form: one MAX all-reduce merges both extremes
+        negmin_max[j] = -lo;
+        negmin_max[cols + j] = hi;
+    }
     if (WITH_SUM) {
         if (osum) osum[j] = sum;
         omean[j] = total > 0 ? (float)(sum / (double)total) : 0.0f;
@@ -426,7 +431,8 @@ static size_t colreduce_smem_bytes(int slab_w, int stage_rows)
 template <class D, bool WITH_SUM>
 static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *omin,
                                     float *omax, float *omean, double *osum, long long *count, int accumulate,
-                                    void *ws, aweq_dev_status *st, cudaStream_t stream)
+                                    void *ws, aweq_dev_status *st, cudaStream_t stream, float *negmin_max = nullptr,
+                                    double *count_f64 = nullptr)
 {
     long long rows = 0;
     for (int k = 0; k < segs.n; ++k) rows += segs.rows[k];
@@ -449,7 +455,8 @@ static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *
     }
     AWEQ_LAUNCH(colreduce_finalize_kernel<WITH_SUM>, dim3((unsigned)((cols + kFinCols - 1) / kFinCols)),
                 dim3(kFinCols * kFinLanes), 0, stream, (const float *)pmin, (const float *)pmax, (const double *)psum,
-                nsplit_eff, cols, rows, omin, omax, omean, osum, (const long long *)count, accumulate, st);
+                nsplit_eff, cols, rows, omin, omax, omean, osum, (const long long *)count, accumulate, st, negmin_max,
+                count_f64);
     if (WITH_SUM && count) {
         AWEQ_LAUNCH(bump_count_kernel, dim3(1), dim3(1), 0, stream, count, rows, accumulate);
     }
@@ -469,18 +476,50 @@ void colreduce_describe(long long rows, long long cols, long long plan[8])
     plan[7] = p.stage_rows;
 }
 
+// Statistics of a token shard back from their exchange form (see run_stats): after the two
+// all-reduces the buffers hold the extremes, sums and token count of all shards.
+__global__ void stats_from_exchange_kernel(const float *__restrict__ negmin_max, const double *__restrict__ sum_count,
+                                           long long cols, float *xmin, float *xmax, float *xmean)
+{
+    pdl_begin();
+    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= cols) return;
+    const double total = sum_count[cols];
+    xmin[j] = -negmin_max[j];
+    xmax[j] = negmin_max[cols + j];
+    xmean[j] = total > 0.0 ? (float)(sum_count[j] / total) : 0.0f;
+}
+
+aweq_status run_stats_from_exchange(const float *negmin_max, const double *sum_count, long long C, float *xmin,
+                                    float *xmax, float *xmean, cudaStream_t stream)
+{
+    AWEQ_LAUNCH(stats_from_exchange_kernel, dim3((unsigned)((C + 255) / 256)), dim3(256), 0, stream, negmin_max,
+                sum_count, C, xmin, xmax, xmean);
+    return AWEQ_OK;
+}
+
+// negmin_max / sum_count (both or neither): also leave the statistics in exchange form,
+// negmin_max = float[2 C] = { -xmin, xmax }, sum_count = double[C + 1] = { column sums, N }.
 aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin, float *xmax,
                       float *xmean, double *xsum, long long *count, int accumulate, void *ws, aweq_dev_status *st,
-                      cudaStream_t stream)
+                      cudaStream_t stream, float *negmin_max, double *sum_count)
 {
+    if (negmin_max && sum_count) {
+        xsum = sum_count;
+        count = nullptr;
+        accumulate = 0;
+    }
+    double *count_f64 = (negmin_max && sum_count) ? sum_count + C : nullptr;
     ColSegs segs = {};
     segs.base[0] = reinterpret_cast<const uint16_t *>(X);
     segs.rows[0] = N;
     segs.ld[0] = ld;
     segs.n = 1;
     if (dt == AWEQ_F16)
-        return launch_colreduce<F16, true>(segs, C, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
-    return launch_colreduce<BF16, true>(segs, C, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream);
+        return launch_colreduce<F16, true>(segs, C, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream,
+                                           negmin_max, count_f64);
+    return launch_colreduce<BF16, true>(segs, C, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream, negmin_max,
+                                        count_f64);
 }
 
 aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld, float *wmin,
@@ -519,9 +558,11 @@ aweq_status run_wrange_multi(const void *const *W, const long long *C_out, const
 // ------------------------------------------------------------------ statistics without caller scratch
 // Scratch for aweq_stats_static: the per-split partials of one call.  It lives in
 // the library image, so every GPU that loads the library holds these bytes until
-// the process exits.  The partials need (row splits) x C_in x 16 bytes and the
-// number of row splits is at most 148 / ceil(C_in / 2048), so 148 x 2048 x 16
-// bytes cover every supported width.
+// the process exits.  The partials need (row splits) x (row phases) x C_in x 16
+// bytes; the number of row splits is at most 148 / ceil(C_in / 2048), and two row
+// phases are only used up to 768 columns (148 x 2 x 768 x 16 bytes), so
+// 148 x 2048 x 16 bytes cover every supported width.  The entry point compares the
+// planner's own figure with the array size as well.
 namespace aweq {
 constexpr size_t kStaticScratchBytes = (size_t)kColTargetCtas * kColThreads * 8 * 16 + 256;
 constexpr long long kStaticMaxCin = 16384;

@@ -182,7 +182,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
     }
 }
 // 1-D bulk copy global -> this CTA's shared memory, completion on an mbarrier.
-// Both addresses 16-byte aligned, bytes a multiple of 16.  No multicast.
+// Both addresses 16-byte aligned, bytes a multiple of 16.  The copy lands in this CTA only.
 __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

@@ -3,7 +3,7 @@
 // translation unit.  C[M x N] = A[M x K] B[N x K]^T, both operands K-contiguous.
 // The instantiations use 256 x 256 output tiles computed by CTA pairs (cta_group::2, cluster
 // 2 x 1): each CTA of a pair stages half of the A and half of the B tile, so no operand is
-// loaded twice and no multicast copy is involved.  Of the tile shapes tried on layer-sized
+// loaded twice and every TMA copy has a single destination CTA.  Of the tile shapes tried on layer-sized
 // problems this one was the fastest for both operand types.
 #pragma once
 #include "common.cuh"

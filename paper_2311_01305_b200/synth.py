@@ -123,6 +123,40 @@ def workloads(n_tokens_scale: float = 1.0) -> dict:
     return w
 
 
+def algorithmic_bytes(wl: Workload, bits: int) -> int:
+    """Bytes one layer pass must move: X once for the statistics; every W once
+    for its column ranges and once more, plus the packed codes and the
+    (Step, Z) pairs, for the fused rescale-quantise-pack; for W8A8 X a second
+    time plus one byte per element and a (Step, Z) pair per token.  Bookkeeping
+    for the benchmark: sizes only."""
+    total = 0
+    for inp in wl.inputs:
+        total += 2 * inp.n_tokens * inp.c_in
+        if wl.act_quant:
+            total += 3 * inp.n_tokens * inp.c_in + 8 * inp.n_tokens
+    for lin in wl.linears:
+        n = lin.c_out * lin.c_in
+        pairs = lin.c_out if wl.w_gran == "row" else lin.c_out * (lin.c_in // wl.group)
+        total += 2 * n + 2 * n + n * bits // 8 + 8 * pairs
+    return total
+
+
+def weight_bytes(wl: Workload) -> int:
+    """Bytes of all 16-bit weight matrices of the workload (one read of W)."""
+    return sum(2 * lin.c_out * lin.c_in for lin in wl.linears)
+
+
+def generate(wl: Workload, device, rank: int = 0):
+    """Every input and weight tensor of a workload: ({input name: X}, {linear name: W}).
+    ``rank`` selects the token shard (its own seed); the weights are the same on every rank."""
+    X, W = {}, {}
+    for i, inp in enumerate(wl.inputs):
+        X[inp.name] = make_activations(inp, wl.dtype, tensor_seed(wl.seed, rank, i), device)
+    for i, lin in enumerate(wl.linears):
+        W[lin.name] = make_weight(lin, wl.dtype, tensor_seed(wl.seed, 0, 100 + i), device)
+    return X, W
+
+
 def producers(wl: Workload) -> dict:
     """What produces each layer input of a decoder-shaped workload: {input name: (kind, name)}
     with kind "norm" (a normalisation layer's output: its gain and shift take 1/s) or

@@ -107,10 +107,11 @@ def test_ablation_switches():
         compare_layer(wl, 8, Xc, Wc, None, flags=flags)
 
 
-def test_sharded_path_with_one_rank_equals_fused_layer_pass():
-    """The token-sharded route (separate calls, statistics merged by an all-reduce and
-    re-formed by an empty accumulate call) on a one-rank NCCL group gives exactly what the
-    fused layer pass gives."""
+@pytest.mark.parametrize("overlap", [False, True])
+def test_sharded_path_with_one_rank_equals_fused_layer_pass(overlap):
+    """The token-sharded route (the same pass with the statistics leaving the REDUCE part in
+    exchange form, merged by two all-reduces and re-formed inside the QUANT part) on a one-rank
+    NCCL group gives exactly what the fused layer pass gives, on one stream and on two."""
     import socket
     import torch.distributed as dist
     from paper_2311_01305_b200 import calibrate
@@ -123,9 +124,14 @@ def test_sharded_path_with_one_rank_equals_fused_layer_pass():
                             device_id=torch.device("cuda", torch.cuda.current_device()))
     try:
         a = calibrate.LayerCalibrator(wl, 8, Xd, Wd, None)
-        b = calibrate.ShardedLayerCalibrator(wl, 8, Xd, Wd, None)
+        b = calibrate.ShardedLayerCalibrator(wl, 8, Xd, Wd, None, overlap=overlap)
         a.run(); b.run()
         torch.cuda.synchronize()
+        # the exchange buffers hold what the statistics say
+        C = wl.inputs[0].c_in
+        o = b.out[wl.inputs[0].name]
+        assert torch.equal(b.stat_negmin_max[:C], -o["xmin"]) and torch.equal(b.stat_negmin_max[C:2 * C], o["xmax"])
+        assert float(b.stat_sum_count[C]) == Xd[wl.inputs[0].name].shape[0]
     finally:
         dist.destroy_process_group()
     for name, outs in a.out.items():
