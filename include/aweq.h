@@ -216,6 +216,11 @@ aweq_status aweq_factors_absmax(const float *xmin, const float *xmax, const floa
  * step: float, zp: int, one per row ([C_out]), per group ([C_out x C_in/group])
  * or a single pair.  epsmu: float[C_out] or NULL.
  * ws: aweq_workspace_bytes(AWEQ_OP_EQUALIZE_QUANTIZE, C_out, C_in, bits, gran, group).
+ * Non-finite elements never fault.  An infinite element makes Step infinite and every code of
+ * its row / group equal to the zero-point's clamp, as Eq. 1 evaluated literally gives.  A NaN
+ * element is ignored by the extremes (Step, Z and every other code are as if it were absent);
+ * the codes of the eight consecutive columns that share its 16-byte input vector are unspecified.
+ * The same holds for step 6.
  */
 aweq_status aweq_equalize_quantize(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ldw,
                                    const float *s, const float *mu_hat,

@@ -32,7 +32,8 @@
  * follow the same rule):
  *   - dead channels (a zero or non-finite range): s = 1;
  *   - a constant vector (Step would be 0): Step = |lo|, or 1 when lo == 0;
- *   - zero-point and rounded values saturate to the int32 range;
+ *   - zero-point and rounded values saturate to the int32 range (the rule is
+ *     this build's; what it gives is pinned by hand-worked vectors);
  *   - sub-byte code packing: 4-bit two per byte, low nibble first; 3-bit as a
  *     dense little-endian bit stream, eight codes per three bytes.
  */
@@ -675,4 +676,23 @@ void oracle_forward_check_weights(const uint8_t *codes, const float *step, const
     }
     sums[3] = (double)N * (double)C_out;
     free(sq);
+}
+
+/* ------------------------------------------------------------------ */
+/* Signed relabelling of 8-bit codes (Eq. 1 with the code range moved   */
+/* from [0, 255] to [-128, 127]): q' = q - 128, Z' = Z - 128, so that   */
+/* Step (q' - Z') = Step (q - Z).  Z' saturates to the int32 range like */
+/* every zero-point here.  codes: n bytes; zp / zp_out: nz values or    */
+/* NULL.                                                               */
+/* ------------------------------------------------------------------ */
+void oracle_relabel_signed(const uint8_t *codes, int64_t n, int8_t *out, const int32_t *zp, int64_t nz,
+                           int32_t *zp_out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = (int8_t)((int)codes[i] - 128);
+    if (zp && zp_out)
+        for (int64_t k = 0; k < nz; ++k) {
+            int64_t z = (int64_t)zp[k] - 128;
+            if (z < (int64_t)INT32_MIN) z = (int64_t)INT32_MIN;
+            zp_out[k] = (int32_t)z;
+        }
 }

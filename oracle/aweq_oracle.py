@@ -256,6 +256,17 @@ def fold_scale(P, dtype, rinv):
     return out
 
 
+def relabel_signed(codes, zp=None):
+    """8-bit codes q -> q - 128 (int8), zero-points Z -> Z - 128 (saturating) -> (codes_signed, zp_signed or None)."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(codes.shape, np.int8)
+    zp_in = None if zp is None else np.ascontiguousarray(zp, dtype=np.int32)
+    zp_out = None if zp is None else np.empty(zp_in.shape, np.int32)
+    _load().oracle_relabel_signed(_p(codes), i64(codes.size), _p(out), _p(zp_in), i64(0 if zp is None else zp_in.size),
+                                  _p(zp_out))
+    return out, zp_out
+
+
 def forward_check_weights(codes, step, zp, bits, gran, group, rinv, bias_q, X, W, dtype, bias=None):
     """Eq. 11 on data for a weight-only layer -> (mean_err[C_out] f64, sums[4] f64); packed codes as
     ``equalize_quantize`` returns them, ``rinv`` binary32 or None."""

@@ -278,8 +278,10 @@ __device__ __forceinline__ QParams make_qparams(float lo, float hi, int qmax)
     asm("cvt.rni.sat.s32.f32 %0, %1;" : "=r"(zi) : "f"(-z));    // saturating; NaN -> 0
     p.zp = zi;
     // |lo / Step| < 4e6 keeps every clamped value below 2^22, where adding 1.5 * 2^23 rounds
-    // exactly like rint; an infinite 1 / Step makes z infinite or NaN and fails the test
-    p.fast = fabsf(z) < 4.0e6f;
+    // exactly like rint; an infinite 1 / Step makes z infinite or NaN and fails the test.  An
+    // infinite Step (an infinite element in the vector) has 1 / Step = 0 and z = 0: it must
+    // take the literal path too, where Inf * 0 = NaN becomes code Z as the definition says
+    p.fast = fabsf(z) < 4.0e6f && st <= 3.0e38f;
     return p;
 }
 // exact reference form of one code: clamp(rint(fl(v*inv)) + Z, 0, qmax) with saturating int32

@@ -140,13 +140,17 @@ def test_decoder_walk_matches_oracle_in_the_same_order(kind, dtype, act_quant, b
 
 
 @pytest.mark.parametrize("shape", [(300, 768), (7, 13), (1, 1)])
-def test_relabel_signed_keeps_the_dequantised_values(shape):
-    """q' = q - 128, Z' = Z - 128 (checked against NumPy integer arithmetic, the definition); the
-    de-quantised values Step (q' - Z') are those of the unsigned codes."""
+def test_relabel_signed_matches_the_oracle(shape):
+    """q' = q - 128, Z' = Z - 128 against the oracle's routine, zero-points at the int32 edge
+    included (Z' saturates); the de-quantised values Step (q' - Z') are those of the unsigned codes."""
     from paper_2311_01305_b200 import aweq
     rng = np.random.default_rng(shape[0])
     q = rng.integers(0, 256, shape).astype(np.uint8)
     zp = rng.integers(-300, 600, shape[0]).astype(np.int32)
+    zp[0] = -2147483648 + 5                      # saturates
+    if shape[0] > 2:
+        zp[1], zp[2] = -2147483648 + 128, 2147483647
+    o_q, o_z = orc.relabel_signed(q, zp)
     out, check = util.guarded(shape, torch.uint8)
     zp_out, check_z = util.guarded((shape[0],), torch.int32)
     aweq.aweq_relabel_signed(torch.from_numpy(q).to(DEV), out, torch.from_numpy(zp).to(DEV), zp_out)
@@ -154,11 +158,14 @@ def test_relabel_signed_keeps_the_dequantised_values(shape):
     check()
     check_z()
     qs = out.cpu().numpy().view(np.int8)
-    assert np.array_equal(qs.astype(np.int32), q.astype(np.int32) - 128)
-    assert np.array_equal(zp_out.cpu().numpy(), zp - 128)
-    assert np.array_equal(qs.astype(np.int64) - zp_out.cpu().numpy()[:, None], q.astype(np.int64) - zp[:, None])
+    assert np.array_equal(qs, o_q)
+    assert np.array_equal(zp_out.cpu().numpy(), o_z)
+    assert zp_out.cpu().numpy()[0] == -2147483648
+    keep = zp.astype(np.int64) - 128 >= -2147483648
+    assert np.array_equal((qs.astype(np.int64) - zp_out.cpu().numpy().astype(np.int64)[:, None])[keep],
+                          (q.astype(np.int64) - zp.astype(np.int64)[:, None])[keep])
     # in place, codes only
     t = torch.from_numpy(q).to(DEV)
     aweq.aweq_relabel_signed(t)
     torch.cuda.synchronize()
-    assert np.array_equal(t.cpu().numpy().view(np.int8).astype(np.int32), q.astype(np.int32) - 128)
+    assert np.array_equal(t.cpu().numpy().view(np.int8), orc.relabel_signed(q)[0])

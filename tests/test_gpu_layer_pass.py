@@ -66,9 +66,7 @@ def compare_layer(wl, bits, Xc, Wc, bias_c=None, flags=0):
             util.assert_same_values(lo["codes"].numpy(), r["codes"], l.name + " codes")
             if bc:
                 assert np.allclose(lo["bias_f32"].numpy(), r["bias_f32"], rtol=0, atol=1e-5)
-                got = orc.decode16(util.bits(lo["bias"]), util.odt(lo["bias"]))
-                want = orc.decode16(r["bias_16"], util.odt(lo["bias"]))
-                assert np.all(np.abs(got - want) <= util.bias16_tolerance(want, util.odt(lo["bias"])))
+                util.check_bias16(lo["bias"], lo["bias_f32"], r["bias_16"])
         if wl.act_quant:
             util.assert_same_values(o["act_zp"], ref["act"][2], "act zp")
             util.assert_same_values(o["act_step"], ref["act"][1], "act step")

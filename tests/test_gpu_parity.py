@@ -176,7 +176,10 @@ def test_factors_match_oracle(C_in):
     Wc = util.rand16((64, C_in), torch.float16, seed=C_in + 1, scale=0.02)
     xs, wr, f = _oracle_front(Xc, [Wc])
     d = dev_factors(xs[0], xs[1], xs[2], wr[0], wr[1])
-    for k in ("s", "rinv", "pX", "pW"):
+    # Eq. 10 is evaluated in binary64 and rounded once on both sides: identical factors
+    util.assert_same_values(d["s"], f["s"], "s")
+    util.assert_same_values(d["rinv"], f["rinv"], "rinv")
+    for k in ("pX", "pW"):
         assert np.allclose(d[k], f[k], rtol=1e-6, atol=0), k
     assert np.allclose(d["mu_hat"], f["mu_hat"], rtol=1e-6, atol=1e-12)
     assert np.allclose(d["scalars"], f["scalars"], rtol=1e-6, atol=0)
@@ -283,6 +286,63 @@ def test_equalize_quantize_degenerate_rows():
         check_weights(Xc, Wc, bits, gran, group, equalize=True)
 
 
+def test_equalize_quantize_int32_saturation():
+    """The hand-worked saturation cases of the quantiser (a tiny spread on a huge offset; the
+    zero-point or the rounded values leave the int32 range) through step 4: 16-bit ones times
+    factors that carry the values, so that W^ = s exactly."""
+    cases = [([8421504.0, 8421505.0], -2147483392, [0, 255]), ([8421505.0, 8421506.0], -2147483648, [0, 0]),
+             ([2.0 ** 41 - 2.0 ** 17, 2.0 ** 41], -2147483648, [0, 0])]
+    for dtype in (torch.float16, torch.bfloat16):
+        for C_in in (8, 264):
+            Wc = torch.ones((2, C_in), dtype=dtype)
+            Wc[1] = -1.0                                       # the mirrored row: Z above the range
+            for vals, zp_want, codes_want in cases:
+                s = np.array([vals[j % 2] for j in range(C_in)], np.float32)
+                mu = np.zeros(C_in, np.float32)
+                o = orc.equalize_quantize(util.bits(Wc), util.odt(Wc), s, mu, 8, orc.PER_ROW)
+                d = dev_equalize_quantize(Wc.to(DEV), s, mu, 8, aweq.PER_ROW, 0)
+                util.assert_same_values(d[2], o[2], "zero-points")
+                util.assert_same_values(d[1], o[1], "Step")
+                util.assert_same_values(d[0], o[0], "codes")
+                assert d[2][0] == zp_want and d[0][0, :2].tolist() == codes_want
+                if vals[0] == 8421505.0:
+                    assert d[2][1] == 2147483647 and not d[0][1].any()
+
+
+def _nan_vector_mask(t16: torch.Tensor, bits: int) -> np.ndarray:
+    """True for the packed bytes that hold codes of a 16-byte input vector containing a NaN
+    (eight columns = `bits` bytes); rows must be whole vectors."""
+    nan = torch.isnan(t16.float()).numpy()
+    vec = nan.reshape(nan.shape[0], -1, 8).any(axis=2)
+    return np.repeat(vec, bits, axis=1)
+
+
+@pytest.mark.parametrize("gran,group,bits", [(1, 0, 8), (2, 128, 4), (2, 128, 3), (2, 32, 4)])
+def test_equalize_quantize_nonfinite_inputs(gran, group, bits):
+    """Inf / NaN elements injected on the host.  Infinite elements: every code, Step and
+    zero-point equals the oracle's.  NaN elements: the extremes ignore them on both sides, so
+    Step, Z and all codes outside the NaN's own 16-byte vector equal the oracle's."""
+    C_out, C_in = 24, 512
+    W = torch.randn((C_out, C_in), generator=torch.Generator().manual_seed(77)) * 0.02
+    W[1, 5] = float("inf")
+    W[2, 130] = float("-inf")
+    W[4, 0] = float("inf"); W[4, 300] = float("-inf")
+    W[6, 128:256] = float("inf")
+    s = (torch.rand(C_in, generator=torch.Generator().manual_seed(78)) + 0.5).numpy()
+    for with_nan in (False, True):
+        if with_nan:
+            W[3, 7] = float("nan")
+            W[5, 511] = float("nan"); W[5, 256] = float("inf")
+        Wc = W.to(torch.float16)
+        o = orc.equalize_quantize(util.bits(Wc), orc.F16, s, None, bits, gran, group)
+        d = dev_equalize_quantize(Wc.to(DEV), s, None, bits, gran, group)
+        util.assert_same_values(d[2], o[2], "zero-points")
+        util.assert_same_values(d[1], o[1], "Step")
+        keep = ~_nan_vector_mask(Wc, bits)
+        assert keep.all() != with_nan
+        util.assert_same_values(d[0][keep], o[0][keep], "codes")
+
+
 # ------------------------------------------------------------------ step 5
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
 @pytest.mark.parametrize("bits,gran,group", [(8, 1, 0), (4, 2, 128), (3, 2, 128), (4, 0, 0)])
@@ -311,9 +371,7 @@ def test_bias_correct_both_routes(bits, gran, group, dtype):
             ref32 = o_f32 if with_bias else orc.bias_correct(o_delta, None, util.odt(bias_c))[0]
             ref16 = o_16 if with_bias else orc.bias_correct(o_delta, None, util.odt(bias_c))[1]
             assert np.allclose(b32.cpu().numpy(), ref32, rtol=0, atol=1e-5)
-            got16 = orc.decode16(util.bits(b16), util.odt(bias_c))
-            want16 = orc.decode16(ref16, util.odt(bias_c))
-            assert np.all(np.abs(got16 - want16) <= util.bias16_tolerance(want16, util.odt(bias_c)))
+            util.check_bias16(b16, b32, ref16)
 
 
 # ------------------------------------------------------------------ step 6
@@ -393,6 +451,38 @@ def test_quant_act_degenerate_rows():
     d = dev_quant_act(Xc.to(DEV), None, 8, aweq.PER_ROW)
     for a, b in zip(d, o):
         util.assert_same_values(a, b)
+
+
+def test_quant_act_int32_saturation_and_nonfinite():
+    """Step 6 on the hand-worked saturation cases (ones times 1/s values that carry the data)
+    and on rows with Inf / NaN elements: the oracle's numbers, element by element."""
+    C = 520
+    Xc = torch.ones((4, C), dtype=torch.float16)
+    Xc[3] = -1.0
+    for vals, zp_want, codes_want in [([8421504.0, 8421505.0], -2147483392, [0, 255]),
+                                      ([8421505.0, 8421506.0], -2147483648, [0, 0])]:
+        rinv = np.array([vals[j % 2] for j in range(C)], np.float32)
+        o = orc.quant_act(util.bits(Xc), orc.F16, rinv, orc.PER_ROW)
+        d = dev_quant_act(Xc.to(DEV), rinv, 8, aweq.PER_ROW)
+        for a, b in zip(d, o):
+            util.assert_same_values(a, b)
+        assert d[2][0] == zp_want and d[0][0, :2].tolist() == codes_want
+    assert d[2][3] == 2147483647 and not d[0][3].any()
+    X = torch.randn((6, C), generator=torch.Generator().manual_seed(5))
+    X[1, 9] = float("inf")
+    X[2, 100] = float("-inf")
+    X[5, 0] = float("inf"); X[5, 519] = float("-inf")
+    for with_nan in (False, True):
+        if with_nan:
+            X[3, 3] = float("nan")
+            X[4, 0] = float("inf"); X[4, 519] = float("nan")
+        Xc = X.to(torch.float16)
+        o = orc.quant_act(util.bits(Xc), orc.F16, None, orc.PER_ROW)
+        d = dev_quant_act(Xc.to(DEV), None, 8, aweq.PER_ROW)
+        util.assert_same_values(d[2], o[2], "zero-points")
+        util.assert_same_values(d[1], o[1], "Step")
+        keep = ~_nan_vector_mask(Xc, 8)
+        util.assert_same_values(d[0][keep], o[0][keep], "codes")
 
 
 # ------------------------------------------------------------------ host-side validation (no fault, an error code)

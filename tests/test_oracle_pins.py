@@ -701,3 +701,24 @@ def test_absmax_criterion_closed_form_and_what_it_balances():
     assert np.array_equal(g["s"], orc.factors(xmin, xmax, xmean, wmin, wmax)["s"])   # the default is the paper's
     # the diagnostics stay range-based under either criterion
     assert np.array_equal(f["pX"], g["pX"]) and np.array_equal(f["pW"], g["pW"])
+
+
+# ---------------------------------------------------------------- signed relabelling of 8-bit codes
+def test_relabel_signed_keeps_dequantised_values_and_saturates():
+    """q' = q - 128 and Z' = Z - 128 leave Step (q - Z) unchanged (Eq. 1 de-quantised, with the
+    code range moved); checked on all 256 codes with integers typed here, by the two's-complement
+    identity (subtracting 128 modulo 256 flips the top bit), and at the int32 edge, where Z'
+    saturates instead of wrapping."""
+    q = np.arange(256, dtype=np.uint8)
+    zp = np.array([0, 128, -7, 300, 2147483647, -2147483648 + 128, -2147483648 + 127, -2147483648], np.int32)
+    qs, zs = orc.relabel_signed(q, zp)
+    assert qs.dtype == np.int8 and qs[0] == -128 and qs[128] == 0 and qs[255] == 127
+    assert np.array_equal(qs.astype(np.int64), np.arange(256) - 128)
+    assert np.array_equal(qs.view(np.uint8), q ^ 0x80)
+    assert zs.tolist() == [-128, 0, -135, 172, 2147483519, -2147483648, -2147483648, -2147483648]
+    ok = zp.astype(np.int64) - 128 >= -2147483648           # where nothing saturates the values are kept
+    step = 0.37
+    for k in np.flatnonzero(ok):
+        assert np.array_equal(step * (qs.astype(np.int64) - int(zs[k])), step * (q.astype(np.int64) - int(zp[k])))
+    only_codes, none = orc.relabel_signed(q.reshape(16, 16))
+    assert none is None and only_codes.shape == (16, 16)

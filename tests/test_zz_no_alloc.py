@@ -5,12 +5,16 @@ where cudaMalloc's device-wide synchronisation is not acceptable).  The scratch
 is an array built into the library.  The test drives the entry point through
 the C ABI twice in a row, on different shapes so that the second call runs over
 what the first one left in the shared array, and compares each result with the
-ordinary aweq_stats entry point, which takes caller scratch.  This file is
-collected last on purpose."""
+ordinary aweq_stats entry point, which takes caller scratch, and with the CPU
+oracle.  The shapes include the widths at which the built-in array is exactly
+full (2048 columns), the widest accepted row (16384) and the narrow layout that
+keeps two sets of partials per row split (768).  This file is collected last on
+purpose."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import aweq_oracle as orc
 from tests import util
 
 pytestmark = pytest.mark.gpu
@@ -33,7 +37,8 @@ def _both(aweq, X):
 
 def test_static_scratch_entry_matches_stats_twice_in_a_row():
     from paper_2311_01305_b200 import aweq
-    shapes = [((6000, 4096), torch.bfloat16), ((777, 1032), torch.float16)]
+    shapes = [((6000, 4096), torch.bfloat16), ((777, 1032), torch.float16), ((1500, 2048), torch.float16),
+              ((24, 16384), torch.bfloat16), ((5000, 768), torch.float16)]
     for shape, dtype in shapes:
         Xc = util.rand16(shape, dtype, seed=shape[0], offset=2.0, outlier_cols=6)
         ref, got = _both(aweq, Xc.cuda())
@@ -41,6 +46,10 @@ def test_static_scratch_entry_matches_stats_twice_in_a_row():
         util.assert_same_values(got[1], ref[1], "xmax")
         mean_abs = np.abs(Xc.double().numpy()).mean(axis=0)
         assert np.all(np.abs(got[2].astype(np.float64) - ref[2]) <= util.mean_tolerance(ref[2], mean_abs))
+        o = orc.stats(util.bits(Xc), util.odt(Xc))
+        util.assert_same_values(got[0], o[0], "xmin against the oracle")
+        util.assert_same_values(got[1], o[1], "xmax against the oracle")
+        assert np.all(np.abs(got[2].astype(np.float64) - o[2]) <= util.mean_tolerance(o[2], mean_abs))
 
 
 def test_static_scratch_entry_rejects_sizes_beyond_its_limit():

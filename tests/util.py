@@ -92,12 +92,18 @@ def bits_of(t):
     return bits(t)
 
 
-def bias16_tolerance(ref, dtype_tag):
-    """1e-3 absolute (the stated bound for fp16 biases), but never tighter than one
-    unit in the last place of the 16-bit format at that magnitude: a binary32 value
-    that sits next to a rounding tie may legitimately round to the neighbouring
-    16-bit value (bf16 has 8 significant bits: one ulp is 2e-3 already at 0.25)."""
-    mant = 10 if dtype_tag == orc.F16 else 7
-    a = np.maximum(np.abs(np.asarray(ref, dtype=np.float64)), 2.0 ** -14)
-    ulp = 2.0 ** (np.floor(np.log2(a)) - mant)
-    return np.maximum(1e-3, ulp)
+def check_bias16(bias16: torch.Tensor, bias32: torch.Tensor, ref16_bits) -> None:
+    """The 16-bit corrected bias is the library's own binary32 bias rounded once to the 16-bit
+    type (exactly), and agrees with the oracle's 16-bit bias to 1e-3 absolute for fp16; a bf16
+    value (8 significant bits: one ulp is 2e-3 already at 0.25) may sit one ulp from the
+    oracle's when the two binary32 values straddle a rounding boundary."""
+    tag = odt(bias16)
+    b32 = bias32.detach().cpu().numpy()
+    assert_same_values(bits(bias16), orc.encode16(b32, tag), "16-bit bias = round16(binary32 bias)")
+    got = orc.decode16(bits(bias16), tag).astype(np.float64)
+    want = orc.decode16(np.asarray(ref16_bits), tag).astype(np.float64)
+    tol = np.full(want.shape, 1e-3)
+    if tag == orc.BF16:
+        a = np.maximum(np.abs(want), 2.0 ** -126)
+        tol = np.maximum(tol, 2.0 ** (np.floor(np.log2(a)) - 7))
+    assert np.all(np.abs(got - want) <= tol)
