@@ -464,6 +464,9 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="replay the pass as one CUDA graph in the timed region (1 GPU; the dominant kernel is then "
                          "timed in eager passes after it)")
+    ap.add_argument("--profile-pass", action="store_true",
+                    help="after the timed region, issue one more eager pass between cudaProfilerStart and "
+                         "cudaProfilerStop (a range for a profiler started with profiling off; not timed)")
     ap.add_argument("--op", default="layer_pass", choices=["layer_pass", "forward_check"],
                     help="forward_check: time the forward check of the calibrated layer instead (1 GPU)")
     args = ap.parse_args()
@@ -517,6 +520,13 @@ def main():
                        "not more than the HBM can deliver"),
         "roofline": r["roofline"], "clocks": r["clocks"], "gpu_launches": r["launches"], "device_status": r["status"],
     }
+
+    if args.profile_pass and world == 1:
+        torch.cuda.synchronize()
+        torch.cuda.profiler.start()
+        cal.run()
+        torch.cuda.synchronize()
+        torch.cuda.profiler.stop()
 
     # ---------------------------------------------------------------- end to end: host buffers in, results out
     if not args.no_e2e:

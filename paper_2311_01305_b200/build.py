@@ -77,14 +77,27 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 def _build_locked(force: bool, verbose: bool) -> str:
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
-    deps = srcs + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) + [
+    headers = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) + [
         os.path.join(os.path.dirname(HERE), "include", "aweq.h"), os.path.abspath(__file__)]
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest(deps):
-        return LIB
     os.makedirs(OBJ, exist_ok=True)
     objs = [os.path.join(OBJ, os.path.basename(s)[:-3] + ".o") for s in srcs]
-    with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, len(srcs))) as ex:
-        logs = list(ex.map(lambda so: _compile(so[0], so[1], verbose), zip(srcs, objs)))
+    # an object is stale when its source, a header it includes (directly: the headers here do not
+    # include one another beyond common.cuh / kernels.h / aweq.h) or this script is newer
+    def stale(src, obj):
+        if force or not os.path.exists(obj):
+            return True
+        text = open(src).read()
+        deps = [src, os.path.abspath(__file__)]
+        for h in headers:
+            name = os.path.basename(h)
+            if name in ("common.cuh", "kernels.h", "aweq.h") or ('"%s"' % name) in text:
+                deps.append(h)
+        return os.path.getmtime(obj) < _newest(deps)
+    todo = [(s, o) for s, o in zip(srcs, objs) if stale(s, o)]
+    if not todo and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest(objs):
+        return LIB
+    with concurrent.futures.ThreadPoolExecutor(max_workers=8) as ex:
+        logs = list(ex.map(lambda so: _compile(so[0], so[1], verbose), todo))
     if verbose:
         sys.stderr.write("\n".join(logs))
     cmd = [_nvcc(), "-shared", "-o", LIB, *objs, "-Xcompiler", "-fPIC"]

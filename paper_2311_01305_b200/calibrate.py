@@ -36,10 +36,31 @@ def exchange_layout(wl: synth.Workload):
     return off, mm, sc
 
 
+def schedule_order(wl: synth.Workload) -> List[str]:
+    """Order in which the two-stream schedule takes the layer inputs (names).  The weight kernels
+    of an input run beside the next input's statistics sweep and those of the last input have
+    nothing to hide under, so the input that feeds the fewest weight bytes goes last and the
+    one that feeds the most is followed by the longest sweep.  Sizes only; every output is the
+    same in any order."""
+    fed = [i for i in wl.inputs if any(l.input == i.name for l in wl.linears)]
+    if len(fed) < 3:
+        return [i.name for i in fed]
+    wbytes = {i.name: sum(2 * l.c_out * l.c_in for l in wl.linears if l.input == i.name) for i in fed}
+    xbytes = {i.name: 2 * i.n_tokens * i.c_in for i in fed}
+    last = min(reversed(fed), key=lambda i: wbytes[i.name])
+    rest = [i for i in fed if i is not last]
+    heavy = max(rest, key=lambda i: wbytes[i.name])
+    long_sweep = max(rest, key=lambda i: xbytes[i.name])
+    if long_sweep is not heavy:
+        rest.remove(long_sweep)
+        rest.insert(rest.index(heavy) + 1, long_sweep)
+    return [i.name for i in rest] + [last.name]
+
+
 class LayerCalibrator:
     def __init__(self, wl: synth.Workload, bits: int, X: Dict[str, torch.Tensor], W: Dict[str, torch.Tensor],
                  bias: Optional[Dict[str, torch.Tensor]] = None, flags: int = 0, diagnostics: bool = True,
-                 overlap: bool = False, exchange_buffers: bool = False):
+                 overlap: bool = False, exchange_buffers: bool = False, order: Optional[List[str]] = None):
         """``overlap``: split every pass into its parts (``FLAG_PHASE_*``) and issue the
         shared-memory-staged, HBM-bound kernels (the column reductions of steps 1-2 and step 6) on
         one CUDA stream and the short, issue-bound kernels that need no shared memory (factors,
@@ -48,7 +69,9 @@ class LayerCalibrator:
         ``run()`` forks from and joins back into the current stream.
         ``exchange_buffers``: give every pass the exchange form of its statistics (one flat
         ``float32`` buffer {-xmin, xmax} and one flat ``float64`` buffer {sums, count} over all
-        inputs; see ``ShardedLayerCalibrator``)."""
+        inputs; see ``ShardedLayerCalibrator``).
+        ``order``: names of the fed inputs in the order ``run()`` takes them (default: as the
+        workload lists them, or ``schedule_order`` with two streams)."""
         self.wl, self.bits = wl, bits
         dev = next(iter(X.values())).device
         td = synth.torch_dtype(wl.dtype)
@@ -58,6 +81,12 @@ class LayerCalibrator:
         self.passes: List[aweq.LayerPass] = []
         ws_bytes = 256
         fed = [i for i in wl.inputs if any(l.input == i.name for l in wl.linears)]
+        if order is None and overlap:
+            order = schedule_order(wl)
+        if order is not None:
+            by_name = {i.name: i for i in fed}
+            assert sorted(order) == sorted(by_name), "order must name every fed input once"
+            fed = [by_name[n] for n in order]
         self.stat_negmin_max = self.stat_sum_count = None
         self._slices = []
         if exchange_buffers:

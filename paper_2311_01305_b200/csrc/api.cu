@@ -66,8 +66,10 @@ static aweq_status check_ws(void *ws, size_t ws_bytes, size_t need)
     return AWEQ_OK;
 }
 
-static size_t eq_ws_bytes(long long rows, long long cols, int gran)
+static size_t eq_ws_bytes(long long rows, long long cols, int bits, int gran, int group)
 {
+    // per group of 128: the (window, row) partial sums of eps . E[x^]
+    if (gran == AWEQ_PER_GROUP) return groupquant_supported(bits, group) ? round256(groupquant_ws_bytes(rows, cols)) : 0;
     if (gran != AWEQ_PER_TENSOR) return 0;
     // per-tensor: column extremes of W (2 x float[cols]) + lo/hi + the column-reduction scratch
     return round256((size_t)cols * 8) + 256 + colreduce_ws_bytes(rows, cols);
@@ -116,12 +118,11 @@ aweq_status aweq_plan_query(int op, long long rows, long long cols, long long pl
 
 size_t aweq_workspace_bytes(int op, long long rows, long long cols, int bits, int gran, int group)
 {
-    (void)bits; (void)group;
     if (cols <= 0 || rows < 0) return 0;
     switch (op) {
     case AWEQ_OP_STATS:
     case AWEQ_OP_WRANGE: return colreduce_ws_bytes(rows, cols);
-    case AWEQ_OP_EQUALIZE_QUANTIZE: return eq_ws_bytes(rows, cols, gran);
+    case AWEQ_OP_EQUALIZE_QUANTIZE: return eq_ws_bytes(rows, cols, bits, gran, group);
     default: return 0;
     }
 }
@@ -187,7 +188,7 @@ static aweq_status equalize_quantize_impl(const void *W, aweq_dtype dt, long lon
     if (rc != AWEQ_OK) return rc;
     if (!codes || !step || !zp) return AWEQ_ERR_NULL;
     if (!aligned(codes, 16) || (s && !aligned(s, 16)) || (mu_hat && !aligned(mu_hat, 16))) return AWEQ_ERR_ALIGN;
-    rc = check_ws(ws, ws_bytes, eq_ws_bytes(C_out, C_in, gran));
+    rc = check_ws(ws, ws_bytes, eq_ws_bytes(C_out, C_in, bits, gran, group));
     if (rc != AWEQ_OK) return rc;
     AWEQ_LOGF("aweq_equalize_quantize C_out=%lld C_in=%lld bits=%d gran=%d group=%d bytes=%lld\n", C_out, C_in, bits,
               (int)gran, group, 2 * C_out * C_in + C_out * C_in * bits / 8);
@@ -196,6 +197,8 @@ static aweq_status equalize_quantize_impl(const void *W, aweq_dtype dt, long lon
         if (!rowquant_supported(C_out, C_in)) return AWEQ_ERR_SHAPE;
         return run_rowquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, codes, step, zp, epsmu, bias, st, cs);
     }
+    if (gran == AWEQ_PER_GROUP && groupquant_supported(bits, group))
+        return run_groupquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, codes, step, zp, epsmu, bias, ws, cs);
     if (gran == AWEQ_PER_GROUP)
         return run_warpquant(W, dt, C_out, C_in, ldw, s, mu_hat, bits, true, group, nullptr, codes, step, zp, epsmu,
                              bias, st, cs);
@@ -277,7 +280,7 @@ static size_t layer_ws_parts(const aweq_layer_args *a, size_t *col_part)
     for (int i = 0; i < a->n_w; ++i) {
         size_t c = colreduce_ws_bytes(a->C_out[i], a->C_in);
         if (c > col) col = c;
-        size_t e = eq_ws_bytes(a->C_out[i], a->C_in, a->gran);
+        size_t e = eq_ws_bytes(a->C_out[i], a->C_in, a->bits, a->gran, a->group);
         if (e > eq) eq = e;
     }
     col = round256(col);

@@ -34,6 +34,12 @@ aweq_status run_warpquant(const void *X, aweq_dtype dt, long long nrows, long lo
                           const float *scale, const float *mu, int bits, bool weights, int group,
                           const float *lo_hi, unsigned char *out, float *step, int *zp, float *epsmu,
                           const BiasIO &bias, aweq_dev_status *st, cudaStream_t stream);
+// group-128 quantiser with column windows (3, 4 or 8 bits); ws: groupquant_ws_bytes
+bool groupquant_supported(int bits, int group);
+size_t groupquant_ws_bytes(long long rows, long long cols);
+aweq_status run_groupquant(const void *W, aweq_dtype dt, long long nrows, long long cols, long long ld,
+                           const float *scale, const float *mu, int bits, unsigned char *out, float *step, int *zp,
+                           float *epsmu, const BiasIO &bias, void *ws, cudaStream_t stream);
 aweq_status run_scaled_tensor_range(const float *cmin, const float *cmax, const float *scale, long long C,
                                     float *lo_hi, cudaStream_t stream);
 aweq_status run_bias_apply(const float *epsmu, const void *bias_in, void *bias_out, float *bias_out_f32,

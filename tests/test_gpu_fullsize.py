@@ -92,7 +92,8 @@ def check_weight_rows(wl, W, bits, gran, group, seed, nrows=24):
     zp = torch.empty(pairs, dtype=torch.int32, device=DEV)
     epsmu = torch.empty(C_out, device=DEV)
     st = aweq.new_status()
-    aweq.aweq_equalize_quantize(W, s.to(DEV), mu.to(DEV), bits, gran, group, codes, step, zp, epsmu, st=st)
+    ws = aweq.workspace(aweq.workspace_bytes(aweq.OP_EQUALIZE_QUANTIZE, C_out, C_in, bits, gran, group))
+    aweq.aweq_equalize_quantize(W, s.to(DEV), mu.to(DEV), bits, gran, group, codes, step, zp, epsmu, ws=ws, st=st)
     torch.cuda.synchronize()
     assert aweq.read_status(st)["wait_timeout"] == 0
     rows = torch.randperm(C_out, generator=torch.Generator().manual_seed(seed))[:nrows].sort().values

@@ -250,7 +250,9 @@ def test_equalize_quantize_per_row(C_out, C_in, bits, dtype):
 @pytest.mark.parametrize("C_out,C_in,bits,group", [(300, 4096, 4, 128), (300, 4096, 3, 128), (64, 11008, 4, 128),
                                                    (64, 11008, 3, 128), (37, 768, 4, 8), (37, 776, 3, 8),
                                                    (37, 784, 3, 16), (19, 1056, 4, 32), (19, 1088, 8, 64),
-                                                   (19, 2304, 2, 256), (21, 640, 5, 128), (21, 1024, 3, 256)])
+                                                   (19, 2304, 2, 256), (21, 640, 5, 128), (21, 1024, 3, 256),
+                                                   (1, 128, 4, 128), (7, 384, 3, 128), (9, 640, 8, 128),
+                                                   (301, 4224, 4, 128), (8, 256, 3, 128), (40, 1152, 8, 128)])
 def test_equalize_quantize_per_group(C_out, C_in, bits, group, dtype):
     Xc = util.rand16((128, C_in), dtype, seed=C_in + bits, offset=2.0, outlier_cols=6)
     Wc = util.rand16((C_out, C_in), dtype, seed=C_out * 3 + C_in, scale=0.02)
@@ -264,6 +266,23 @@ def test_equalize_quantize_per_tensor_and_rtn(bits):
     check_weights(Xc, Wc, bits, aweq.PER_TENSOR, 0)
     check_weights(Xc, Wc, bits, aweq.PER_ROW, 0, equalize=False)
     check_weights(Xc, Wc, bits, aweq.PER_GROUP, 8, equalize=False)
+    W2 = util.rand16((45, 1408), torch.bfloat16, seed=3, scale=0.02)
+    X2 = util.rand16((64, 1408), torch.bfloat16, seed=4, offset=2.0, outlier_cols=6)
+    check_weights(X2, W2, bits, aweq.PER_GROUP, 128, equalize=False)
+
+
+@pytest.mark.parametrize("bits,gran,group", [(4, 2, 128), (3, 2, 128), (8, 1, 0), (4, 2, 32)])
+def test_equalize_quantize_row_pitch(bits, gran, group):
+    """W as a column slice of a wider matrix (row pitch larger than C_in)."""
+    big = util.rand16((70, 1160), torch.bfloat16, seed=31, scale=0.02).to(DEV)
+    W = big[:, 8:8 + 1024]
+    s = (torch.rand(1024, generator=torch.Generator().manual_seed(2)) + 0.5).numpy()
+    mu = (torch.randn(1024, generator=torch.Generator().manual_seed(3)) * 0.2).numpy()
+    o = orc.equalize_quantize(util.bits(W), orc.BF16, s, mu, bits, gran, group)
+    d = dev_equalize_quantize(W, s, mu, bits, gran, group)
+    util.assert_same_values(d[2], o[2], "zero-points")
+    util.assert_same_values(d[1], o[1], "Step")
+    util.assert_same_values(d[0], o[0], "codes")
 
 
 def test_equalize_quantize_degenerate_rows():
@@ -293,7 +312,7 @@ def test_equalize_quantize_int32_saturation():
     cases = [([8421504.0, 8421505.0], -2147483392, [0, 255]), ([8421505.0, 8421506.0], -2147483648, [0, 0]),
              ([2.0 ** 41 - 2.0 ** 17, 2.0 ** 41], -2147483648, [0, 0])]
     for dtype in (torch.float16, torch.bfloat16):
-        for C_in in (8, 264):
+        for C_in in (8, 264, 384):
             Wc = torch.ones((2, C_in), dtype=dtype)
             Wc[1] = -1.0                                       # the mirrored row: Z above the range
             for vals, zp_want, codes_want in cases:
@@ -307,6 +326,13 @@ def test_equalize_quantize_int32_saturation():
                 assert d[2][0] == zp_want and d[0][0, :2].tolist() == codes_want
                 if vals[0] == 8421505.0:
                     assert d[2][1] == 2147483647 and not d[0][1].any()
+                if C_in % 128 == 0:                            # the same through the group quantiser
+                    o = orc.equalize_quantize(util.bits(Wc), util.odt(Wc), s, mu, 8, orc.PER_GROUP, 128)
+                    d = dev_equalize_quantize(Wc.to(DEV), s, mu, 8, aweq.PER_GROUP, 128)
+                    util.assert_same_values(d[2], o[2], "zero-points")
+                    util.assert_same_values(d[1], o[1], "Step")
+                    util.assert_same_values(d[0], o[0], "codes")
+                    assert d[2][0] == zp_want and d[0][0, :2].tolist() == codes_want
 
 
 def _nan_vector_mask(t16: torch.Tensor, bits: int) -> np.ndarray:

@@ -47,7 +47,10 @@ def test_host_helpers(lib):
     big = lib.aweq_workspace_bytes(1, 262144, 11008, 0, 0, 0)
     assert 0 < small < big < 64 << 20
     assert lib.aweq_workspace_bytes(6, 262144, 4096, 8, 1, 0) == 0
-    assert lib.aweq_workspace_bytes(4, 4096, 4096, 4, 2, 128) == 0
+    # groups of 128 at 3 / 4 / 8 bits: one float per (256-column window, row) for the eps . E[x^] partials
+    assert lib.aweq_workspace_bytes(4, 4096, 4096, 4, 2, 128) == 16 * 4096 * 4
+    assert lib.aweq_workspace_bytes(4, 4101, 11008, 3, 2, 128) == (43 * 4104 * 4 + 255) // 256 * 256
+    assert lib.aweq_workspace_bytes(4, 4096, 4096, 4, 2, 64) == 0
     assert lib.aweq_workspace_bytes(4, 4096, 4096, 4, 0, 0) > 0
 
 
