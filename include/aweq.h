@@ -103,7 +103,8 @@ unsigned long long aweq_launch_count(void);
  *   column reduction: {CTAs, threads, shared bytes, column slabs, slab width in 16-byte vectors,
  *                      row splits, row phases, rows per stage}
  *   row quantisers:   {CTAs, threads, shared bytes, threads per row, vectors per thread,
- *                      rows per stage, stages, 1 if the wide-row kernel is used}
+ *                      rows per stage, stages, kernel: 0 staged, 1 staged for wide rows, 2 plain
+ *                      loads without stages (rows per stage and stages are 0 then)}
  * Returns AWEQ_ERR_SHAPE when the shape is not supported, AWEQ_ERR_UNSUPPORTED for other ops. */
 aweq_status aweq_plan_query(int op, long long rows, long long cols, long long plan[8]);
 

@@ -1,0 +1,33 @@
+// Host side of the direct (plain-load) row quantiser: which rows it takes and the dispatch
+// to its instantiations.
+#include "rowdirect_impl.cuh"
+#include "kernels.h"
+
+namespace aweq {
+
+// The smallest team (1, 2, 4 or 8 warps) whose threads hold the row in at most ten vectors each.
+// Weight matrices take this kernel whenever such a team exists (rows of up to 20480 columns);
+// the per-token quantiser of step 6 only for rows of up to 5120 columns, where it measured
+// faster than the staged kernel (a long run over hundreds of thousands of rows keeps the
+// staged ring full, a matrix of a few thousand rows does not).
+bool plan_rowdirect(long long cols, bool weights, int *team_warps, int *V)
+{
+    const int nvec = (int)(cols / 8);
+    if (!weights && nvec > 384) return false;
+    for (int tw = 1; tw <= 8; tw *= 2) {
+        const int v = (nvec + tw * 32 - 1) / (tw * 32);
+        if (v <= kRqMaxV) {
+            *team_warps = tw;
+            *V = v;
+            return true;
+        }
+    }
+    return false;
+}
+
+aweq_status run_rowdirect(const RowQuantParams &p, int team_warps, int V, int mode, aweq_dtype dt, cudaStream_t stream)
+{
+    return dt == AWEQ_F16 ? rd_launch_f16(p, team_warps, V, mode, stream) : rd_launch_bf16(p, team_warps, V, mode, stream);
+}
+
+}  // namespace aweq

@@ -1,6 +1,6 @@
 // Host side of the row quantiser: how a row is split over threads, how many rows
 // form a stage, and the dispatch to the fp16 / bf16 instantiations.
-#include "rowquant_impl.cuh"
+#include "rowdirect_impl.cuh"
 
 namespace aweq {
 
@@ -71,6 +71,16 @@ bool rowquant_supported(long long nrows, long long cols)
 bool rowquant_describe(long long rows, long long cols, bool weights, long long plan[8])
 {
     RowQuantPlan pl;
+    int tw = 0, dv = 0;
+    if (plan_rowdirect(cols, weights, &tw, &dv)) {
+        // the plain-load kernel: no stages; teams take rows one by one
+        const int teams = kRdThreads / (tw * 32), per_sm = dv <= 4 ? 3 : 2;
+        long long grid = (rows + teams - 1) / teams;
+        if (grid > (long long)kSmCount * per_sm) grid = (long long)kSmCount * per_sm;
+        plan[0] = grid < 1 ? 1 : grid; plan[1] = kRdThreads; plan[2] = (long long)sizeof(RdSmem); plan[3] = tw * 32;
+        plan[4] = dv; plan[5] = 0; plan[6] = 0; plan[7] = 2;
+        return true;
+    }
     const bool wide = !weights && plan_rowquant_wide(rows, cols, &pl);
     if (!wide && !plan_rowquant(rows, cols, &pl)) return false;
     plan[0] = pl.grid; plan[1] = pl.NT; plan[2] = (long long)pl.smem; plan[3] = pl.team; plan[4] = pl.V;
@@ -84,9 +94,11 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
                          float *step, int *zp, float *epsmu, const BiasIO &bias, aweq_dev_status *st,
                          cudaStream_t stream)
 {
-    RowQuantPlan pl;
-    const bool wide = !weights && plan_rowquant_wide(nrows, cols, &pl);
-    if (!wide && !plan_rowquant(nrows, cols, &pl)) return AWEQ_ERR_SHAPE;
+    RowQuantPlan pl = {};
+    int tw = 0, dv = 0;
+    const bool direct = plan_rowdirect(cols, weights, &tw, &dv);
+    const bool wide = !direct && !weights && plan_rowquant_wide(nrows, cols, &pl);
+    if (!direct && !wide && !plan_rowquant(nrows, cols, &pl)) return AWEQ_ERR_SHAPE;
     RowQuantParams p;
     p.X = reinterpret_cast<const uint16_t *>(X);
     p.nrows = nrows; p.ld = ld; p.nvec = (int)(cols / 8);
@@ -95,8 +107,9 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     p.step = step; p.zp = zp; p.epsmu = epsmu; p.bits = bits; p.bias = bias;
     p.team = pl.team; p.rows_per_stage = pl.rows_per_stage; p.stages = pl.stages; p.ntiles = pl.ntiles;
     p.st = st;
-    if (wide) return run_rowquant_wide(p, pl, dt, stream);
     const int mode = !weights ? 0 : ((mu && epsmu) ? 1 : 2);
+    if (direct) return run_rowdirect(p, tw, dv, mode, dt, stream);
+    if (wide) return run_rowquant_wide(p, pl, dt, stream);
     return dt == AWEQ_F16 ? rq_launch_f16(p, pl, mode, stream) : rq_launch_bf16(p, pl, mode, stream);
 }
 
