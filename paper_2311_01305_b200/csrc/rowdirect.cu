@@ -5,11 +5,11 @@
 
 namespace aweq {
 
-// The smallest team (1, 2, 4 or 8 warps) whose threads hold the row in at most ten vectors each.
-// Weight matrices take this kernel whenever such a team exists (rows of up to 20480 columns);
-// the per-token quantiser of step 6 only for rows of up to 5120 columns, where it measured
-// faster than the staged kernel (a long run over hundreds of thousands of rows keeps the
-// staged ring full, a matrix of a few thousand rows does not).
+// The smallest team (1, 2, 4 or 8 warps) whose threads hold the row in at most ten vectors each;
+// beyond 20480 columns a whole CTA of 32 warps with at most five vectors per thread.  Weight
+// matrices always take this kernel; the per-token quantiser of step 6 only for rows of up to
+// 3072 columns, where it measured faster than the staged kernel (a long run over hundreds of
+// thousands of rows keeps the staged ring full, a matrix of a few thousand rows does not).
 bool plan_rowdirect(long long cols, bool weights, int *team_warps, int *V)
 {
     const int nvec = (int)(cols / 8);
@@ -21,6 +21,12 @@ bool plan_rowdirect(long long cols, bool weights, int *team_warps, int *V)
             *V = v;
             return true;
         }
+    }
+    const int v = (nvec + 1023) / 1024;
+    if (v <= 5) {
+        *team_warps = 32;
+        *V = v;
+        return true;
     }
     return false;
 }

@@ -20,10 +20,12 @@
 namespace aweq {
 
 constexpr int kRdThreads = 256;
+// threads of a CTA: 256 (several teams), or the team itself when it has more than 8 warps
+__host__ __device__ constexpr int rd_threads(int TW) { return TW > 8 ? TW * 32 : kRdThreads; }
 
 struct RdSmem {
-    float2 red[2][kRdThreads / 32];
-    float rsum[2][kRdThreads / 32];
+    float2 red[2][32];
+    float rsum[2][32];
 };
 
 template <class D, bool SC_REGS>
@@ -92,13 +94,13 @@ __device__ __forceinline__ void rd_codes(const float2 (&x)[4], const QParams &q,
 
 // V: vectors per thread; TW: warps per team
 template <class D, int V, int TW, bool MU, bool BYTES_OUT>
-__global__ void __launch_bounds__(kRdThreads, V <= 4 ? 3 : 2)
+__global__ void __launch_bounds__(rd_threads(TW), TW > 8 ? 1 : V <= 4 ? 3 : 2)
 rowdirect_kernel(const RowQuantParams p)
 {
     __shared__ RdSmem sm;
     pdl_begin();
     constexpr int T = TW * 32;
-    constexpr int teams = kRdThreads / T;
+    constexpr int teams = rd_threads(TW) / T;
     constexpr bool SC_REGS = V <= 4;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tm = threadIdx.x / T, tt = threadIdx.x % T;
@@ -194,12 +196,12 @@ rowdirect_kernel(const RowQuantParams p)
 template <class D, int V, int TW, bool MU, bool BYTES_OUT>
 static aweq_status rd_launch_one(const RowQuantParams &p, cudaStream_t stream)
 {
-    constexpr int teams = kRdThreads / (TW * 32);
-    constexpr int per_sm = V <= 4 ? 3 : 2;
+    constexpr int teams = rd_threads(TW) / (TW * 32);
+    constexpr int per_sm = TW > 8 ? 1 : V <= 4 ? 3 : 2;
     long long grid = (p.nrows + teams - 1) / teams;
     if (grid > (long long)kSmCount * per_sm) grid = (long long)kSmCount * per_sm;
     if (grid < 1) grid = 1;
-    AWEQ_LAUNCH((rowdirect_kernel<D, V, TW, MU, BYTES_OUT>), dim3((unsigned)grid), dim3(kRdThreads), 0, stream, p);
+    AWEQ_LAUNCH((rowdirect_kernel<D, V, TW, MU, BYTES_OUT>), dim3((unsigned)grid), dim3(rd_threads(TW)), 0, stream, p);
     return AWEQ_OK;
 }
 
@@ -222,6 +224,7 @@ static aweq_status rd_launch(const RowQuantParams &p, int team_warps, int V, int
     AWEQ_RD_CASE(2, 6) AWEQ_RD_CASE(2, 7) AWEQ_RD_CASE(2, 8) AWEQ_RD_CASE(2, 9) AWEQ_RD_CASE(2, 10)
     AWEQ_RD_CASE(4, 6) AWEQ_RD_CASE(4, 7) AWEQ_RD_CASE(4, 8) AWEQ_RD_CASE(4, 9) AWEQ_RD_CASE(4, 10)
     AWEQ_RD_CASE(8, 6) AWEQ_RD_CASE(8, 7) AWEQ_RD_CASE(8, 8) AWEQ_RD_CASE(8, 9) AWEQ_RD_CASE(8, 10)
+    AWEQ_RD_CASE(32, 3) AWEQ_RD_CASE(32, 4) AWEQ_RD_CASE(32, 5)
 #undef AWEQ_RD_CASE
     return AWEQ_ERR_UNSUPPORTED;
 }
