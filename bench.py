@@ -406,7 +406,6 @@ def run_extras(args, dev, skip):
     code as the headline region (one GPU), and the forward check of two calibrated layers."""
     table, checks = {}, {}
     wls = synth.workloads(args.tokens_scale)
-    fc_of = dict(EXTRA_FORWARD_CHECKS)
     for name, bits in EXTRA_WORKLOADS:
         if (name, bits) == skip:
             continue
@@ -423,8 +422,12 @@ def run_extras(args, dev, skip):
             "dominant_kernel": rf["kernel"], "frac": rf["frac"], "dominant_gbs": rf["achieved"],
             "stats_gbs": rf.get("stats_gbs", rf["achieved"]), "launch": r["launch"],
             "sm_mhz": r["clocks"].get("sm_mhz"), "reasons": r["clocks"].get("reasons")}
-        del cal
-        if fc_of.get(name) == bits and not args.no_forward_check:
+        del cal, X, W
+        torch.cuda.empty_cache()
+    if not args.no_forward_check:
+        for name, bits in EXTRA_FORWARD_CHECKS:
+            wl = wls[name]
+            X, W = generate(wl, dev, 0)
             fc, res, cal = time_forward_check(wl, bits, X, W, 2, 1)
             checks["%s@w%d" % (name, bits)] = {
                 "ms_per_step": fc["ms_per_step"], "tflops": fc["tflops"], "frac": fc["roofline"]["frac"],
@@ -433,9 +436,8 @@ def run_extras(args, dev, skip):
                 "reasons": fc["clocks"].get("reasons"),
                 "output_sqnr_db": {n: round(float(10.0 * torch.log10(s4[1] / s4[0]).item()), 3)
                                    for n, (me, s4) in res.items()}}
-            del cal, res
-        del X, W
-        torch.cuda.empty_cache()
+            del cal, res, X, W
+            torch.cuda.empty_cache()
     return table, checks
 
 

@@ -237,7 +237,7 @@ def check_weights(Xc, Wc, bits, gran, group, equalize=True):
 
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
 @pytest.mark.parametrize("C_out,C_in,bits", [(4, 8, 8), (33, 24, 8), (768, 768, 8), (100, 3072, 8), (300, 4096, 8),
-                                             (40, 5120, 8), (20, 9216, 8), (12, 13824, 8), (9, 36864, 8),
+                                             (40, 5120, 8), (20, 9216, 8), (12, 13824, 8), (9, 36864, 8), (6, 24576, 8), (5, 30720, 8), (3, 40960, 8),
                                              (64, 1032, 4), (64, 776, 3), (50, 512, 2), (31, 264, 5), (17, 520, 6),
                                              (23, 2056, 7)])
 def test_equalize_quantize_per_row(C_out, C_in, bits, dtype):
@@ -419,7 +419,7 @@ def dev_quant_act(X, rinv, bits, gran, lo_hi=None):
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
 @pytest.mark.parametrize("N,C_in", [(1, 8), (5, 24), (2048, 768), (1000, 3072), (777, 4096), (300, 5120),
                                     (130, 9216), (129, 11008), (65, 13824), (33, 36864), (20, 40960),
-                                    (70, 10248), (41, 20488), (1, 13824)])
+                                    (70, 10248), (41, 20488), (1, 13824), (23, 24576), (9, 24568)])
 def test_quant_act_per_token(N, C_in, dtype):
     Xc = util.rand16((N, C_in), dtype, seed=N + C_in, offset=1.0, outlier_cols=min(6, C_in // 4))
     Wc = util.rand16((16, C_in), dtype, seed=5, scale=0.02)
