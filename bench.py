@@ -270,11 +270,24 @@ def run_forward_check(args, wl, bits):
         "max_abs_mean_err_over_output_rms": worst, "output_sqnr_db": sqnr, "ablation": ablation}))
 
 
-# Measured share of the second read of W (step 4, after step 2 has streamed the same matrices) that
-# the L2 serves instead of HBM, per workload: ncu DRAM read bytes of the step-4 kernels of one pass
-# over their algorithmic read bytes, captured at 1/32 of the tokens (weights are full size at any
-# token count).  None = not captured for the kernels as they are now.
-W_SECOND_READ_FROM_L2 = {}
+# ncu DRAM counters of ONE whole layer pass at full size, as scheduled in the timed region (two
+# streams, eager), taken as a single profiler range (dram__bytes_read.sum, dram__bytes_write.sum):
+# {(workload, bits): (bytes read, bytes written)}.  Compared with the algorithmic bytes they say how
+# much of the pass the L2 served.  The kernels have not changed since the counters were taken.
+PASS_DRAM_BYTES = {("llama7b_layer_w4w3_g128", 4): (13020324352, 121289472),
+                   ("llama7b_layer_w4w3_g128", 3): (13011394816, 97897728),
+                   ("llama13b_layer_w8a8", 8): (31896055296, 8008074752)}
+# Share of the second read of W (step 4, after step 2 has streamed the same matrices) that the L2 serves
+# instead of HBM.  "scheduled": from the range capture above (algorithmic read bytes minus DRAM read bytes,
+# over one read of W); a statistics sweep of the next input runs between the two reads and flushes the L2.
+# "one_stream": per-kernel DRAM read bytes of the step-4 kernels with every kernel of a pass serialised
+# (one stream, 1/32 of the tokens; weights are full size at any token count): what the L2 could serve.
+W_SECOND_READ_FROM_L2 = {("llama7b_layer_w4w3_g128", 4): {"scheduled": 0.007, "one_stream": 0.644},
+                         ("llama7b_layer_w4w3_g128", 3): {"scheduled": 0.029, "one_stream": 0.654}}
+# DRAM traffic of the statistics sweep per launch, from a one-kernel capture at 1/8 of the tokens
+# (268.44 MB of X: 268.46 MB read): reads grow with the rows; the few MB written during the launch are
+# dirty lines of earlier kernels leaving the L2, not traffic of the sweep.
+STATS_DRAM_READ_RATIO = 1.0001
 
 
 def time_layer_pass(wl, bits, X, W, steps, warmup, *, rank=0, world=1, local=0, dist=None,
@@ -384,10 +397,18 @@ def time_layer_pass(wl, bits, X, W, steps, warmup, *, rank=0, world=1, local=0, 
         roofline["stats_gbs"] = dom["stats_gbs"]
     nbytes = synth.algorithmic_bytes(wl, bits)
     gbs = world * nbytes / ms / 1e6
-    l2 = W_SECOND_READ_FROM_L2.get((wl.name, bits))
+    l2_both = W_SECOND_READ_FROM_L2.get((wl.name, bits))
+    overlap_on = bool(getattr(cal, "overlap", False))
+    l2 = None if l2_both is None else l2_both["scheduled" if overlap_on else "one_stream"]
     roofline["w_second_read_from_l2"] = l2
+    roofline["w_second_read_from_l2_one_stream"] = None if l2_both is None else l2_both["one_stream"]
+    if not wl.act_quant and world == 1:
+        roofline["traffic"] = STATS_DRAM_READ_RATIO * roofline["bytes_per_launch"]
+    dram = PASS_DRAM_BYTES.get((wl.name, bits)) if (overlap_on and world == 1 and wl.inputs[0].n_tokens == synth.workloads()[wl.name].inputs[0].n_tokens) else None
     res = {"ms": ms, "gbs": gbs, "nbytes": nbytes, "launches": int(launches), "clocks": clocks, "status": status,
            "roofline": roofline, "peak": peak,
+           "pass_dram": None if dram is None else {"read_bytes": dram[0], "write_bytes": dram[1],
+                                                   "over_algorithmic": (dram[0] + dram[1]) / nbytes},
            "gbs_hbm_basis": None if l2 is None else world * (nbytes - l2 * synth.weight_bytes(wl)) / ms / 1e6,
            "launch": ("CUDA graph replay; every fourth step eager, with the event hooks" if mixed
                       else "one CUDA graph replay per step" if graph is not None else "eager"),
@@ -416,6 +437,7 @@ def run_extras(args, dev, skip):
         rf = r["roofline"]
         table["%s@w%d" % (name, bits)] = {
             "bits": bits, "ms_per_step": r["ms"], "gbs": r["gbs"], "gbs_hbm_basis": r["gbs_hbm_basis"],
+            "pass_dram": r["pass_dram"],
             "pct_of_8000_gbs": 100.0 * r["gbs"] / NOMINAL_HBM_GBS,
             "pct_of_measured_copy": 100.0 * r["gbs"] / r["peak"], "tokens_per_s": wl.inputs[0].n_tokens / (r["ms"] / 1e3),
             "algorithmic_bytes": r["nbytes"], "steps": args.extra_steps, "gpu_launches": r["launches"],
@@ -515,11 +537,11 @@ def main():
         "tokens_per_s": world * tokens / (ms / 1e3),
         "pct_of_8000_gbs": 100.0 * gbs / world / NOMINAL_HBM_GBS,
         "pct_of_measured_copy": 100.0 * gbs / world / peak,
-        "value_hbm_basis": r["gbs_hbm_basis"],
-        "basis_note": ("value counts every algorithmic byte, including the second read of W, part of which the L2 "
-                       "serves (roofline.w_second_read_from_l2); value_hbm_basis leaves that part out. A percentage "
-                       "of the measured copy bandwidth above 100 is a read-mostly stream against a read+write copy, "
-                       "not more than the HBM can deliver"),
+        "value_hbm_basis": r["gbs_hbm_basis"], "pass_dram": r["pass_dram"],
+        "basis_note": ("value counts every algorithmic byte; value_hbm_basis leaves out the part of the second read "
+                       "of W that the L2 serves (roofline.w_second_read_from_l2, from ncu DRAM counters of one whole "
+                       "pass as scheduled: pass_dram). A percentage of the measured copy bandwidth above 100 is a "
+                       "read-mostly stream against a read+write copy, not more than the HBM can deliver"),
         "roofline": r["roofline"], "clocks": r["clocks"], "gpu_launches": r["launches"], "device_status": r["status"],
     }
 
