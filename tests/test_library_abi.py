@@ -146,3 +146,26 @@ def test_row_quantiser_plans_fit_the_hardware(lib):
     # beyond the supported width the query says so instead of planning something that cannot launch
     assert _plan(lib, 6, 100, 40968)[0] == 2 and _plan(lib, 4, 100, 81920)[0] == 2
     assert _plan(lib, 6, 100, 36)[0] == 2 and _plan(lib, 5, 100, 64)[0] == 9
+
+
+def test_reference_arm_of_the_bench_loads_only_the_oracle():
+    """`bench.py --impl reference` times the oracle alone: the process must map the oracle's shared
+    object and never the CUDA library (checked from /proc/<pid>/maps at exit of a tiny run)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import sys, runpy, atexit\n"
+            "def report():\n"
+            "    maps = open('/proc/self/maps').read()\n"
+            "    sys.stderr.write('MAPS libaweq.so=%d libaweq_oracle.so=%d\\n' % ('libaweq.so' in maps, 'libaweq_oracle.so' in maps))\n"
+            "atexit.register(report)\n"
+            "sys.argv = ['bench.py', '--impl', 'reference', '--steps', '1', '--warmup', '0', '--cpu-sample-tokens', '64',\n"
+            "            '--workload', 'opt125m_linear_w8a8']\n"
+            "runpy.run_path('bench.py', run_name='__main__')\n")
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    assert "MAPS libaweq.so=0 libaweq_oracle.so=1" in r.stderr, r.stderr[-500:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["gpu_launches"] == 0
+    assert set(line["config"]) >= {"workload", "w_bits", "w_gran", "group", "act_quant", "storage"}
