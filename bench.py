@@ -378,8 +378,10 @@ def time_layer_pass(wl, bits, X, W, steps, warmup, *, rank=0, world=1, local=0, 
 
     # dominant kernel: the statistics sweep (W8A8 workloads: the activation quantiser moves more bytes)
     stats_ms = [sum(es[0].elapsed_time(es[1]) for es, _ in hk) for hk in hooks.values()]
-    stats_bytes = sum(2 * i.n_tokens * i.c_in for i in wl.inputs)
-    dom = {"kernel": "colreduce_kernel (aweq_stats)", "bytes": stats_bytes, "ms": statistics.mean(stats_ms),
+    # where steps 1 and 2 of an input share one launch, the hooks around step 1 time both: count the weights too
+    fused_w = sum(lp.weight_bytes for lp in cal.passes if lp.fused_ranges)
+    stats_bytes = sum(2 * i.n_tokens * i.c_in for i in wl.inputs) + fused_w
+    dom = {"kernel": "colreduce_kernel (aweq_stats" + (" + aweq_wrange, one launch" if fused_w else "") + ")", "bytes": stats_bytes, "ms": statistics.mean(stats_ms),
            "launches_per_step": len(cal.passes)}
     if wl.act_quant:
         act_ms = [sum(ea[0].elapsed_time(ea[1]) for _, ea in hk) for hk in hooks.values()]

@@ -321,6 +321,11 @@ typedef struct {
 } aweq_layer_args;
 
 size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args);
+/* 1 when the pass takes steps 1 and 2 of this input in ONE launch (at most three matrices of at most
+ * 400 MB together share the input: every CTA of the statistics sweep then also reduces its share of
+ * their rows), else 0.
+ * The profiling hooks around step 1 then bracket both steps.  Host logic only. */
+int aweq_layer_pass_fuses_ranges(const aweq_layer_args *args);
 aweq_status aweq_layer_pass(const aweq_layer_args *args, void *ws, size_t ws_bytes,
                             aweq_dev_status *st, void *stream);
 

@@ -78,6 +78,8 @@ _lib.aweq_bias_correct.argtypes = [_vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _ll, _
 _lib.aweq_quant_act.argtypes = [_vp, _i, _ll, _ll, _ll, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.aweq_layer_pass_workspace_bytes.restype = _sz
 _lib.aweq_layer_pass_workspace_bytes.argtypes = [ctypes.POINTER(LayerArgs)]
+_lib.aweq_layer_pass_fuses_ranges.restype = ctypes.c_int
+_lib.aweq_layer_pass_fuses_ranges.argtypes = [ctypes.POINTER(LayerArgs)]
 _lib.aweq_layer_pass.argtypes = [ctypes.POINTER(LayerArgs), _vp, _sz, _vp, _vp]
 _lib.aweq_plan_query.argtypes = [_i, _ll, _ll, ctypes.POINTER(_ll * 8)]
 _lib.aweq_plan_query.restype = _i
@@ -326,6 +328,9 @@ class LayerPass:
         a.act_bits, a.flags = act_bits, flags
         self.args = a
         self.ws_bytes = int(_lib.aweq_layer_pass_workspace_bytes(ctypes.byref(a)))
+        # steps 1 and 2 in one launch (the hooks around step 1 then cover the weight ranges too)
+        self.fused_ranges = bool(_lib.aweq_layer_pass_fuses_ranges(ctypes.byref(a)))
+        self.weight_bytes = sum(w.numel() * w.element_size() for w in Ws)
 
     def set_events(self, stats=None, act=None) -> None:
         """Profiling hooks: pairs of recorded-once ``torch.cuda.Event(enable_timing=True)``

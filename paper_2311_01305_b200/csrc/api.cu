@@ -275,7 +275,8 @@ aweq_status aweq_quant_act(const void *X, aweq_dtype dt, long long N, long long 
 // workspace layout: [column-reduction scratch | scratch of step 4]
 static size_t layer_ws_parts(const aweq_layer_args *a, size_t *col_part)
 {
-    size_t col = colreduce_ws_bytes(a->N, a->C_in);
+    size_t col = stats_wrange_fusable(a->N, a->C_in, a->C_out, a->n_w) ? colreduce_fused_ws_bytes(a->N, a->C_in)
+                                                     : colreduce_ws_bytes(a->N, a->C_in);
     size_t eq = 0;
     for (int i = 0; i < a->n_w; ++i) {
         size_t c = colreduce_ws_bytes(a->C_out[i], a->C_in);
@@ -286,6 +287,11 @@ static size_t layer_ws_parts(const aweq_layer_args *a, size_t *col_part)
     col = round256(col);
     if (col_part) *col_part = col;
     return col + round256(eq);
+}
+
+int aweq_layer_pass_fuses_ranges(const aweq_layer_args *args)
+{
+    return args && args->C_out && stats_wrange_fusable(args->N, args->C_in, args->C_out, args->n_w) ? 1 : 0;
 }
 
 size_t aweq_layer_pass_workspace_bytes(const aweq_layer_args *args)
@@ -346,22 +352,34 @@ aweq_status aweq_layer_pass(const aweq_layer_args *a, void *ws, size_t ws_bytes,
     // steps 1-2
     if (phases & AWEQ_FLAG_PHASE_REDUCE) {
         if (a->ev_stats_begin) AWEQ_CUDA_OK(record_hook(a->ev_stats_begin, cs));
-        if (a->stat_negmin_max) {
-            // aweq_stats' checks, then the sweep that also leaves the exchange form of the statistics
-            if (!aligned(a->xmin, 16) || !aligned(a->xmax, 16) || !aligned(a->xmean, 4)) return AWEQ_ERR_ALIGN;
-            AWEQ_LOGF("aweq_stats N=%lld C_in=%lld (with exchange buffers) bytes=%lld\n", a->N, a->C_in, 2 * a->N * a->C_in);
-            rc = run_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col, st,
-                           cs, a->stat_negmin_max, a->stat_sum_count);
+        if (!aligned(a->xmin, 16) || !aligned(a->xmax, 16) || !aligned(a->xmean, 4)) return AWEQ_ERR_ALIGN;
+        if (stats_wrange_fusable(a->N, a->C_in, a->C_out, a->n_w)) {
+            // steps 1 and 2 in one launch: every CTA of the sweep also takes its share of the rows of the
+            // matrices this input feeds (they have the same columns), so step 2 has no launch, fill or
+            // drain of its own.  The hook interval then covers both steps.
+            AWEQ_LOGF("aweq_stats + aweq_wrange x%d N=%lld C_in=%lld bytes=%lld (one launch)\n", a->n_w, a->N, a->C_in,
+                      2 * a->N * a->C_in);
+            rc = run_stats_wrange(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, a->W, a->C_out, a->ldw,
+                                  a->n_w, a->wmin, a->wmax, ws_col, st, cs, a->stat_negmin_max, a->stat_sum_count);
+            if (rc != AWEQ_OK) return rc;
+            if (a->ev_stats_end) AWEQ_CUDA_OK(record_hook(a->ev_stats_end, cs));
         } else {
-            rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
-                            col_part, st, stream);
+            if (a->stat_negmin_max) {
+                // the sweep that also leaves the exchange form of the statistics
+                AWEQ_LOGF("aweq_stats N=%lld C_in=%lld (with exchange buffers) bytes=%lld\n", a->N, a->C_in, 2 * a->N * a->C_in);
+                rc = run_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
+                               st, cs, a->stat_negmin_max, a->stat_sum_count);
+            } else {
+                rc = aweq_stats(a->X, a->dt, a->N, a->C_in, a->ldx, a->xmin, a->xmax, a->xmean, nullptr, nullptr, 0, ws_col,
+                                col_part, st, stream);
+            }
+            if (rc != AWEQ_OK) return rc;
+            if (a->ev_stats_end) AWEQ_CUDA_OK(record_hook(a->ev_stats_end, cs));
+            // step 2: the matrices share the input, hence one range per input channel over all of them
+            AWEQ_LOGF("aweq_wrange x%d C_in=%lld\n", a->n_w, a->C_in);
+            rc = run_wrange_multi(a->W, a->C_out, a->ldw, a->n_w, a->dt, a->C_in, a->wmin, a->wmax, 0, ws_col, st, cs);
+            if (rc != AWEQ_OK) return rc;
         }
-        if (rc != AWEQ_OK) return rc;
-        if (a->ev_stats_end) AWEQ_CUDA_OK(record_hook(a->ev_stats_end, cs));
-        // step 2: the matrices share the input, hence one range per input channel over all of them
-        AWEQ_LOGF("aweq_wrange x%d C_in=%lld\n", a->n_w, a->C_in);
-        rc = run_wrange_multi(a->W, a->C_out, a->ldw, a->n_w, a->dt, a->C_in, a->wmin, a->wmax, 0, ws_col, st, cs);
-        if (rc != AWEQ_OK) return rc;
     }
     const bool eq = !(a->flags & AWEQ_FLAG_NO_EQUALIZE);
     // without equalisation the layer sees x itself, so E[x^] = E[x]

@@ -196,7 +196,8 @@ template <class D, bool WITH_SUM>
 __global__ void __launch_bounds__(kColThreads + 32, kColCtasPerSm)
 colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int slab_w,
                  int phases, int stage_rows, long long rows_per_split, long long cols, float *__restrict__ pmin,
-                 float *__restrict__ pmax, double *__restrict__ psum, aweq_dev_status *st)
+                 float *__restrict__ pmax, double *__restrict__ psum, aweq_dev_status *st, long long rows_a,
+                 long long rows_per_split_b, float *__restrict__ pmin_b, float *__restrict__ pmax_b)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     ColSmem *sm = reinterpret_cast<ColSmem *>(smem_raw);
@@ -206,8 +207,15 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
     const int split = blockIdx.x / nslab;
     const int v0 = slab * slab_w;
     const int w = min(slab_w, nvec - v0);                 // vectors in this slab (> 0)
-    const long long r0 = (long long)split * rows_per_split;
-    const long long r1 = min(nrows, r0 + rows_per_split);
+    // Two jobs share the launch and the ring: job A is the first rows_a rows of the stack (all of it
+    // in an ordinary call), job B the rest -- the weight matrices fed by the input whose statistics
+    // job A takes -- reduced to extremes of their own.  Every CTA takes its share of both, one after
+    // the other, so the second job costs neither a launch nor a fill and drain of the ring.
+    const long long job_r0[2] = {min(rows_a, (long long)split * rows_per_split),
+                                 min(nrows, rows_a + (long long)split * rows_per_split_b)};
+    const long long job_r1[2] = {min(rows_a, job_r0[0] + rows_per_split),
+                                 min(nrows, job_r0[1] + rows_per_split_b)};
+    const int njobs = rows_per_split_b > 0 ? 2 : 1;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // phase p of the consumer threads takes rows [p, p + 1) * stage_rows / phases of every stage;
     // a phase is a whole number of warps
@@ -229,8 +237,11 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
     if (warp == kColThreads / 32) {
         // ---------------- producer warp
         bool ok = true;
-        long long cur = r0;
-        for (int t = 0; cur < r1 && ok; ++t) {
+        int t = 0;
+        for (int job = 0; job < njobs && ok; ++job) {
+        long long cur = job_r0[job];
+        const long long r1 = job_r1[job];
+        for (; cur < r1 && ok; ++t) {
             const int s = t % kColStages;
             const uint32_t use = t / kColStages;
             if (use > 0) {
@@ -257,6 +268,7 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
             }
             cur += rows;
         }
+        }
         if (!ok && lane == 0) {
             atomicExch(&sm->abort_flag, 1);
             if (st) atomicAdd(&st->wait_timeout, 1ull);
@@ -267,6 +279,9 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
         const int t_col = threadIdx.x - phase * wpad;
         const bool mine = t_col < w;
         const int rows_per_phase = stage_rows / phases;          // a multiple of kFlushRows
+        bool ok = true;
+        int t = 0;
+        for (int job = 0; job < njobs && ok; ++job) {
         typename D::T2 mn[4], mx[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -276,9 +291,9 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
         float sum_hi[8], sum_lo[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) sum_hi[k] = sum_lo[k] = 0.0f;
-        bool ok = true;
-        long long cur = r0;
-        for (int t = 0; cur < r1; ++t) {
+        long long cur = job_r0[job];
+        const long long r1 = job_r1[job];
+        for (; cur < r1; ++t) {
             const int s = t % kColStages;
             const uint32_t use = t / kColStages;
             ok = mbar_wait(&sm->full[s], use & 1);
@@ -317,11 +332,9 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm->empty[s]);
         }
-        if (!ok && lane == 0) {
-            atomicExch(&sm->abort_flag, 1);
-            if (st) atomicAdd(&st->wait_timeout, 1ull);
-        }
+        if (!ok) break;
         if (mine) {
+            // this CTA's partial of the job (neutral values when its share of the job is empty)
             const size_t o = ((size_t)split * phases + phase) * (size_t)cols + (size_t)(v0 + t_col) * 8;
             float lo[8], hi[8];
 #pragma unroll
@@ -330,18 +343,24 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
                 lo[2 * k] = a.x; lo[2 * k + 1] = a.y;
                 hi[2 * k] = b.x; hi[2 * k + 1] = b.y;
             }
-            float4 *qlo = reinterpret_cast<float4 *>(pmin + o), *qhi = reinterpret_cast<float4 *>(pmax + o);
+            float4 *qlo = reinterpret_cast<float4 *>((job == 0 ? pmin : pmin_b) + o);
+            float4 *qhi = reinterpret_cast<float4 *>((job == 0 ? pmax : pmax_b) + o);
             qlo[0] = make_float4(lo[0], lo[1], lo[2], lo[3]);
             qlo[1] = make_float4(lo[4], lo[5], lo[6], lo[7]);
             qhi[0] = make_float4(hi[0], hi[1], hi[2], hi[3]);
             qhi[1] = make_float4(hi[4], hi[5], hi[6], hi[7]);
-            if (WITH_SUM) {
+            if (WITH_SUM && job == 0) {
                 double2 *qs = reinterpret_cast<double2 *>(psum + o);
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
                     qs[k] = make_double2((double)sum_hi[2 * k] + (double)sum_lo[2 * k],
                                          (double)sum_hi[2 * k + 1] + (double)sum_lo[2 * k + 1]);
             }
+        }
+        }
+        if (!ok && lane == 0) {
+            atomicExch(&sm->abort_flag, 1);
+            if (st) atomicAdd(&st->wait_timeout, 1ull);
         }
     }
     // Every copy that was issued has been waited for by the consumers unless a
@@ -428,20 +447,39 @@ static size_t colreduce_smem_bytes(int slab_w, int stage_rows)
     return 128 + (size_t)kColStages * stage_rows * slab_w * 16;
 }
 
+// Scratch of a fused statistics + weight-range launch: the partials of both jobs.
+size_t colreduce_fused_ws_bytes(long long rows, long long cols)
+{
+    const size_t one = colreduce_ws_bytes(rows, cols) - 256;          // 16 bytes per (split, column)
+    return one + one / 2 + 256;                                       // + 8 for the second job's extremes
+}
+
+// rows_a: rows of job A (the first segments); segments beyond them are job B, reduced to omin_b / omax_b
+// (no sums).  rows_a < 0: a single job over all segments.
 template <class D, bool WITH_SUM>
 static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *omin,
                                     float *omax, float *omean, double *osum, long long *count, int accumulate,
                                     void *ws, aweq_dev_status *st, cudaStream_t stream, float *negmin_max = nullptr,
-                                    double *count_f64 = nullptr)
+                                    double *count_f64 = nullptr, long long rows_a = -1, float *omin_b = nullptr,
+                                    float *omax_b = nullptr)
 {
-    long long rows = 0;
-    for (int k = 0; k < segs.n; ++k) rows += segs.rows[k];
+    long long rows_all = 0;
+    for (int k = 0; k < segs.n; ++k) rows_all += segs.rows[k];
+    const long long rows = rows_a < 0 ? rows_all : rows_a;
+    const long long rows_b = rows_all - rows;
     ColPlan p = plan_colreduce(rows, cols);
     char *base = reinterpret_cast<char *>(ws);
     float *pmin = reinterpret_cast<float *>(base);
     const size_t nparts = (size_t)p.nsplit * p.phases;
     float *pmax = pmin + nparts * cols;
     double *psum = reinterpret_cast<double *>(base + nparts * cols * 8);
+    float *pmin_b = reinterpret_cast<float *>(base + nparts * cols * 16);
+    float *pmax_b = pmin_b + nparts * cols;
+    long long rps_b = 0;
+    if (rows_b > 0) {
+        rps_b = (rows_b + p.nsplit - 1) / p.nsplit;
+        rps_b = (rps_b + 7) / 8 * 8;
+    }
     const size_t smem = colreduce_smem_bytes(p.slab_w, p.stage_rows);
     auto kern = colreduce_kernel<D, WITH_SUM>;
     // set on every launch: the attribute belongs to the current device, which may change between calls
@@ -450,13 +488,19 @@ static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *
     int nsplit_eff = rows > 0 ? (int)nparts : 0;
     if (rows > 0) {
         AWEQ_LAUNCH(kern, dim3(p.nslab * p.nsplit), dim3(kColThreads + 32), smem, stream,
-                    segs, rows, p.nvec, p.nslab, p.slab_w, p.phases, p.stage_rows, p.rows_per_split, cols, pmin, pmax,
-                    psum, st);
+                    segs, rows_all, p.nvec, p.nslab, p.slab_w, p.phases, p.stage_rows, p.rows_per_split, cols, pmin, pmax,
+                    psum, st, rows, rps_b, pmin_b, pmax_b);
     }
     AWEQ_LAUNCH(colreduce_finalize_kernel<WITH_SUM>, dim3((unsigned)((cols + kFinCols - 1) / kFinCols)),
                 dim3(kFinCols * kFinLanes), 0, stream, (const float *)pmin, (const float *)pmax, (const double *)psum,
                 nsplit_eff, cols, rows, omin, omax, omean, osum, (const long long *)count, accumulate, st, negmin_max,
                 count_f64);
+    if (rows_b > 0) {
+        AWEQ_LAUNCH(colreduce_finalize_kernel<false>, dim3((unsigned)((cols + kFinCols - 1) / kFinCols)),
+                    dim3(kFinCols * kFinLanes), 0, stream, (const float *)pmin_b, (const float *)pmax_b,
+                    (const double *)nullptr, nsplit_eff, cols, rows_b, omin_b, omax_b, (float *)nullptr, (double *)nullptr,
+                    (const long long *)nullptr, 0, st, (float *)nullptr, (double *)nullptr);
+    }
     if (WITH_SUM && count) {
         AWEQ_LAUNCH(bump_count_kernel, dim3(1), dim3(1), 0, stream, count, rows, accumulate);
     }
@@ -520,6 +564,43 @@ aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, lo
                                            negmin_max, count_f64);
     return launch_colreduce<BF16, true>(segs, C, xmin, xmax, xmean, xsum, count, accumulate, ws, st, stream, negmin_max,
                                         count_f64);
+}
+
+// Steps 1 and 2 of one input in a single launch: the statistics of X and the common ranges of the (at
+// most three) weight matrices it feeds, which have the same number of columns.
+// Worth it while the matrices are small enough for a launch of their own to be dominated by the fill and
+// drain of its ring (measured: the passes of the LLaMA-7B, LLaMA-13B and OPT-125M shapes gain 0.5-1.2 %;
+// two 680 MB matrices reduce at 6.7 TB/s on their own and lose 0.5 % when folded into the sweep).
+bool stats_wrange_fusable(long long N, long long C_in, const long long *C_out, int n_w)
+{
+    if (N <= 0 || n_w < 1 || n_w > kColMaxSegs - 1) return false;
+    long long rows = 0;
+    for (int k = 0; k < n_w; ++k) rows += C_out[k];
+    return 2 * rows * C_in <= 400000000ll;
+}
+
+aweq_status run_stats_wrange(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin,
+                             float *xmax, float *xmean, const void *const *W, const long long *C_out,
+                             const long long *ldw, int n_w, float *wmin, float *wmax, void *ws, aweq_dev_status *st,
+                             cudaStream_t stream, float *negmin_max, double *sum_count)
+{
+    double *xsum = (negmin_max && sum_count) ? sum_count : nullptr;
+    double *count_f64 = (negmin_max && sum_count) ? sum_count + C : nullptr;
+    ColSegs segs = {};
+    segs.base[0] = reinterpret_cast<const uint16_t *>(X);
+    segs.rows[0] = N;
+    segs.ld[0] = ld;
+    for (int k = 0; k < n_w; ++k) {
+        segs.base[1 + k] = reinterpret_cast<const uint16_t *>(W[k]);
+        segs.rows[1 + k] = C_out[k];
+        segs.ld[1 + k] = ldw[k];
+    }
+    segs.n = 1 + n_w;
+    if (dt == AWEQ_F16)
+        return launch_colreduce<F16, true>(segs, C, xmin, xmax, xmean, xsum, nullptr, 0, ws, st, stream, negmin_max,
+                                           count_f64, N, wmin, wmax);
+    return launch_colreduce<BF16, true>(segs, C, xmin, xmax, xmean, xsum, nullptr, 0, ws, st, stream, negmin_max,
+                                        count_f64, N, wmin, wmax);
 }
 
 aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld, float *wmin,

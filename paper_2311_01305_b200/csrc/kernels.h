@@ -15,6 +15,13 @@ bool rowquant_describe(long long rows, long long cols, bool weights, long long p
 aweq_status run_stats(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin, float *xmax,
                       float *xmean, double *xsum, long long *count, int accumulate, void *ws, aweq_dev_status *st,
                       cudaStream_t stream, float *negmin_max = nullptr, double *sum_count = nullptr);
+// steps 1 and 2 of one input in one launch (n_w <= 3 matrices); ws: colreduce_fused_ws_bytes
+size_t colreduce_fused_ws_bytes(long long rows, long long cols);
+bool stats_wrange_fusable(long long N, long long C_in, const long long *C_out, int n_w);
+aweq_status run_stats_wrange(const void *X, aweq_dtype dt, long long N, long long C, long long ld, float *xmin,
+                             float *xmax, float *xmean, const void *const *W, const long long *C_out,
+                             const long long *ldw, int n_w, float *wmin, float *wmax, void *ws, aweq_dev_status *st,
+                             cudaStream_t stream, float *negmin_max = nullptr, double *sum_count = nullptr);
 aweq_status run_stats_from_exchange(const float *negmin_max, const double *sum_count, long long C, float *xmin,
                                     float *xmax, float *xmean, cudaStream_t stream);
 aweq_status run_wrange(const void *W, aweq_dtype dt, long long C_out, long long C_in, long long ld, float *wmin,

@@ -96,6 +96,20 @@ def test_decoder_layer_shapes_with_shared_inputs_few_tokens(name, bits):
     compare_layer(wl, bits, Xc, Wc, None)
 
 
+@pytest.mark.parametrize("n_w,c_in,tokens", [(5, 1032, 300), (3, 776, 37), (1, 4096, 3000), (4, 264, 1000)])
+def test_matrices_sharing_one_input_fused_and_separate_ranges(n_w, c_in, tokens):
+    """Up to three matrices on one input have their ranges taken inside the statistics sweep (one
+    launch, the matrices as further segments of the row stack); four or more go through launches of
+    their own in stacks of four.  Odd sizes: rows that are no multiple of eight, a ragged last slab."""
+    from paper_2311_01305_b200 import aweq
+    inputs = (synth.ActSpec("x", tokens, c_in, "normal", 0, 3, 30.0),)
+    linears = tuple(synth.LinearSpec("w%d" % k, 40 + 27 * k, c_in, "x", 0.02) for k in range(n_w))
+    wl = synth.Workload("custom", "bf16", 11, inputs, linears, (8,), "row", 0, True)
+    Xc, Wc = make_workload_tensors(wl, offset=0.5)
+    cal = compare_layer(wl, 8, Xc, Wc, None)
+    assert cal.passes[0].fused_ranges == (n_w <= 3)
+
+
 def test_ablation_switches():
     from paper_2311_01305_b200 import aweq
     wl = synth.workloads(n_tokens_scale=1.0 / 8)["opt125m_linear_w8a8"]

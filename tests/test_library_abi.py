@@ -83,7 +83,8 @@ def test_binding_imports_and_names_match_header():
     from paper_2311_01305_b200 import aweq
     for name in declared_functions():
         if name in ("aweq_strerror", "aweq_last_cuda_error", "aweq_version", "aweq_launch_count",
-                    "aweq_workspace_bytes", "aweq_layer_pass_workspace_bytes", "aweq_forward_check_workspace_bytes",
+                    "aweq_workspace_bytes", "aweq_layer_pass_workspace_bytes", "aweq_layer_pass_fuses_ranges",
+                    "aweq_forward_check_workspace_bytes",
                     "aweq_forward_check_weights_workspace_bytes"):
             continue
         assert hasattr(aweq, name), name
