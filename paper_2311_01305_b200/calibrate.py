@@ -63,9 +63,9 @@ class LayerCalibrator:
                  overlap: bool = False, exchange_buffers: bool = False, order: Optional[List[str]] = None):
         """``overlap``: split every pass into its parts (``FLAG_PHASE_*``) and issue the
         shared-memory-staged, HBM-bound kernels (the column reductions of steps 1-2 and step 6) on
-        one CUDA stream and the short, issue-bound kernels that need no shared memory (factors,
-        weight quantiser: steps 3-5) on another, each with its own scratch and ordered by events,
-        so that the weight kernels of one input run beside the statistics sweep of the next;
+        one CUDA stream and the short kernels of steps 3-5 (factors, weight quantiser) on others,
+        each with its own scratch and ordered by events, so that the weight kernels of one input
+        fill the tails of the following sweeps;
         ``run()`` forks from and joins back into the current stream.
         ``exchange_buffers``: give every pass the exchange form of its statistics (one flat
         ``float32`` buffer {-xmin, xmax} and one flat ``float64`` buffer {sums, count} over all
@@ -140,8 +140,13 @@ class LayerCalibrator:
         self.status = aweq.new_status(dev)
         self.overlap = bool(overlap) and len(self.passes) > 1 and dev.type == "cuda"
         if self.overlap:
-            self._streams = (torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev))
-            self._ws2 = (self.ws, aweq.workspace(ws_bytes, dev))
+            # One stream for the sweeps; for the weight kernels one stream per input when there is no
+            # step 6 (whatever is left when the last sweep ends -- the weight kernels only run in the tails
+            # of the sweeps -- then runs side by side: LLaMA-7B pass 1.986 -> 1.969 ms), else a single one
+            # (W8A8 passes gained nothing or lost 1 %).  Every stream has scratch of its own.
+            nsmall = 1 if wl.act_quant else len(self.passes)
+            self._streams = (torch.cuda.Stream(device=dev), [torch.cuda.Stream(device=dev) for _ in range(nsmall)])
+            self._ws2 = (self.ws, [aweq.workspace(ws_bytes, dev) for _ in range(nsmall)])
             self._fork = torch.cuda.Event()
             self._ev_stats = [torch.cuda.Event() for _ in self.passes]
             self._ev_weights = [torch.cuda.Event() for _ in self.passes]
@@ -167,11 +172,12 @@ class LayerCalibrator:
                     lp(self.ws, self.status)
             return
         cur = torch.cuda.current_stream()
-        big, small = self._streams
-        ws_big, ws_small = self._ws2
+        big, smalls = self._streams
+        ws_big, ws_smalls = self._ws2
         self._fork.record(cur)
         big.wait_event(self._fork)
-        small.wait_event(self._fork)
+        for small in smalls:
+            small.wait_event(self._fork)
         n = len(self.passes)
 
         def stats(i):
@@ -181,6 +187,7 @@ class LayerCalibrator:
 
         stats(0)
         for i, lp in enumerate(self.passes):
+            small, ws_small = smalls[i % len(smalls)], ws_smalls[i % len(smalls)]
             with torch.cuda.stream(small):
                 small.wait_event(self._ev_stats[i])
                 self._exchange(i)                  # sharded: beside the next input's sweep
@@ -193,7 +200,8 @@ class LayerCalibrator:
                     big.wait_event(self._ev_weights[i])
                     lp(ws_big, self.status, aweq.FLAG_PHASE_ACT)
         cur.wait_stream(big)
-        cur.wait_stream(small)
+        for small in smalls:
+            cur.wait_stream(small)
 
     def capture(self, events=None) -> "torch.cuda.CUDAGraph":
         """Record one ``run()`` (both streams and their events when ``overlap`` is on) into a CUDA
