@@ -104,7 +104,9 @@ unsigned long long aweq_launch_count(void);
  *                      row splits, row phases, rows per stage}
  *   row quantisers:   {CTAs, threads, shared bytes, threads per row, vectors per thread,
  *                      rows per stage, stages, kernel: 0 staged, 1 staged for wide rows, 2 plain
- *                      loads without stages (rows per stage and stages are 0 then)}
+ *                      loads without stages (rows per stage and stages are 0 then), 3 staged
+ *                      with every row shared by a cluster of two CTAs (threads per row = twice
+ *                      the threads of a CTA, shared bytes for half-rows)}
  * Returns AWEQ_ERR_SHAPE when the shape is not supported, AWEQ_ERR_UNSUPPORTED for other ops. */
 aweq_status aweq_plan_query(int op, long long rows, long long cols, long long plan[8]);
 

@@ -81,10 +81,11 @@ bool rowquant_describe(long long rows, long long cols, bool weights, long long p
         plan[4] = dv; plan[5] = 0; plan[6] = 0; plan[7] = 2;
         return true;
     }
-    const bool wide = !weights && plan_rowquant_wide(rows, cols, &pl);
-    if (!wide && !plan_rowquant(rows, cols, &pl)) return false;
+    const bool pair = !weights && plan_rowquant_cluster(rows, cols, &pl);
+    const bool wide = !pair && !weights && plan_rowquant_wide(rows, cols, &pl);
+    if (!pair && !wide && !plan_rowquant(rows, cols, &pl)) return false;
     plan[0] = pl.grid; plan[1] = pl.NT; plan[2] = (long long)pl.smem; plan[3] = pl.team; plan[4] = pl.V;
-    plan[5] = pl.rows_per_stage; plan[6] = pl.stages; plan[7] = wide ? 1 : 0;
+    plan[5] = pl.rows_per_stage; plan[6] = pl.stages; plan[7] = pair ? 3 : wide ? 1 : 0;
     return true;
 }
 
@@ -97,8 +98,9 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     RowQuantPlan pl = {};
     int tw = 0, dv = 0;
     const bool direct = plan_rowdirect(cols, weights, &tw, &dv);
-    const bool wide = !direct && !weights && plan_rowquant_wide(nrows, cols, &pl);
-    if (!direct && !wide && !plan_rowquant(nrows, cols, &pl)) return AWEQ_ERR_SHAPE;
+    const bool pair = !direct && !weights && plan_rowquant_cluster(nrows, cols, &pl);
+    const bool wide = !direct && !pair && !weights && plan_rowquant_wide(nrows, cols, &pl);
+    if (!direct && !pair && !wide && !plan_rowquant(nrows, cols, &pl)) return AWEQ_ERR_SHAPE;
     RowQuantParams p;
     p.X = reinterpret_cast<const uint16_t *>(X);
     p.nrows = nrows; p.ld = ld; p.nvec = (int)(cols / 8);
@@ -109,6 +111,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     p.st = st;
     const int mode = !weights ? 0 : ((mu && epsmu) ? 1 : 2);
     if (direct) return run_rowdirect(p, tw, dv, mode, dt, stream);
+    if (pair) return run_rowquant_cluster(p, pl, dt, stream);
     if (wide) return run_rowquant_wide(p, pl, dt, stream);
     return dt == AWEQ_F16 ? rq_launch_f16(p, pl, mode, stream) : rq_launch_bf16(p, pl, mode, stream);
 }

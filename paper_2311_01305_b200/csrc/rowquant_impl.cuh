@@ -436,6 +436,9 @@ static aweq_status rq_launch(const RowQuantParams &p, const RowQuantPlan &pl, in
 }
 
 aweq_status run_rowquant_wide(const RowQuantParams &p, const RowQuantPlan &pl, aweq_dtype dt, cudaStream_t stream);
+// rows of step 6 beyond 24576 channels, each shared by a cluster of two CTAs (rowquant_cluster.cu)
+bool plan_rowquant_cluster(long long nrows, long long cols, RowQuantPlan *out);
+aweq_status run_rowquant_cluster(const RowQuantParams &p, const RowQuantPlan &pl, aweq_dtype dt, cudaStream_t stream);
 aweq_status rq_launch_f16(const RowQuantParams &p, const RowQuantPlan &pl, int mode, cudaStream_t stream);
 aweq_status rq_launch_bf16(const RowQuantParams &p, const RowQuantPlan &pl, int mode, cudaStream_t stream);
 

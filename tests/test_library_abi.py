@@ -129,7 +129,7 @@ def test_row_quantiser_plans_fit_the_hardware(lib):
                 assert rc == 0, (op, rows, cols)
                 nvec = cols // 8
                 assert 1 <= ctas <= 444 and threads in (256, 512, 768, 1024) and smem <= SMEM_LIMIT
-                assert team % 32 == 0 and threads % team == 0 and team * V >= nvec      # the row is covered
+                assert team % 32 == 0 and (threads % team == 0 or team == 2 * threads) and team * V >= nvec      # the row is covered
                 if wide == 2:                                   # plain loads: no stages, a row per team
                     assert (threads == 256 and team <= 256 and V <= 10) or (threads == team == 1024 and V <= 5)
                     assert V >= 1 and team * (V - 1) < nvec
@@ -138,6 +138,11 @@ def test_row_quantiser_plans_fit_the_hardware(lib):
                     assert ctas <= max(1, -(-rows // (threads // team)))
                     continue
                 assert S >= 2 and R >= 1 and ctas <= 296
+                if wide == 3:                                   # a row per cluster of two CTAs, half a row each
+                    half = (nvec + 1) // 2
+                    assert op == 6 and cols > 24576 and threads == 512 and team == 1024 and V <= 5 and R <= 4
+                    assert ctas % 2 == 0 and ctas <= 148 and 512 * V >= half and smem == 4096 + S * R * half * 16
+                    continue
                 if wide:
                     assert op == 6 and cols > 10240 and V <= 5 and team == threads and R <= 4
                     assert smem >= 4096 + S * R * nvec * 16
