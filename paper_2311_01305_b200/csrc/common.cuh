@@ -233,19 +233,23 @@ __device__ __forceinline__ void cluster_mbar_arrive(uint32_t remote_bar)
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
 }
 // bounded wait on a local mbarrier that CTAs of the cluster arrive on
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity)
 {
+    if (mbar_try_wait_cluster(bar, parity)) return true;      // the clock is read only when the wait is a real one
     const unsigned long long t0 = global_ns();
     for (;;) {
-        for (int i = 0; i < 64; ++i) {
-            uint32_t ok;
-            asm volatile(
-                "{\n\t.reg .pred p;\n\t"
-                "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-                "selp.u32 %0, 1, 0, p;\n\t}"
-                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-            if (ok) return true;
-        }
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
         if (global_ns() - t0 > kWaitLimitNs) return false;
     }
 }

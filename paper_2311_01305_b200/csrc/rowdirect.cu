@@ -5,15 +5,28 @@
 
 namespace aweq {
 
-// The smallest team (1, 2, 4 or 8 warps) whose threads hold the row in at most ten vectors each;
-// beyond 20480 columns a whole CTA of 32 warps with at most five vectors per thread.  Weight
-// matrices always take this kernel; the per-token quantiser of step 6 only for rows of up to
-// 3072 columns, where it measured faster than the staged kernel (a long run over hundreds of
-// thousands of rows keeps the staged ring full, a matrix of a few thousand rows does not).
+// Weight matrices always take this kernel: the smallest team (1, 2, 4 or 8 warps) whose threads
+// hold the row in at most ten vectors each; beyond 20480 columns a whole CTA of 32 warps with at
+// most five vectors per thread.  The per-token quantiser of step 6 takes it for rows of up to
+// 12288 columns, with at most six vectors per thread because a team has the loads of its next
+// row in flight while it reduces and quantises the current one; with that it measured faster
+// than the staged kernels at every width up to there (wider rows would need 16 warps per row,
+// one CTA per SM, and lose to the wide-row kernel).
 bool plan_rowdirect(long long cols, bool weights, int *team_warps, int *V)
 {
     const int nvec = (int)(cols / 8);
-    if (!weights && nvec > 384) return false;
+    if (!weights) {
+        // step 6: the smallest team that holds the row with at most six vectors per thread
+        for (int tw = 1; tw <= 8; tw *= 2) {
+            const int v = (nvec + tw * 32 - 1) / (tw * 32);
+            if (v <= kRdActMaxV) {
+                *team_warps = tw;
+                *V = v;
+                return true;
+            }
+        }
+        return false;
+    }
     for (int tw = 1; tw <= 8; tw *= 2) {
         const int v = (nvec + tw * 32 - 1) / (tw * 32);
         if (v <= kRqMaxV) {

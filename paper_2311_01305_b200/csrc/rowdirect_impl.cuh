@@ -9,7 +9,11 @@
 // served by the L2, was measured at 2.3 TB/s and is not kept.)
 // Latency is hidden by the number of resident teams rather than by a staging pipeline, which
 // suits matrices of a few thousand rows (the weight matrices of step 4), where a persistent
-// ring spends most of its time filling and draining.  Shared memory: 512 bytes.
+// ring spends most of its time filling and draining.  On the long runs of rows of step 6 the
+// resident teams alone leave the kernel waiting for loads (24 warps x 1.5 KB in flight per SM at
+// 768 columns): there a team issues the loads of its next row as soon as the current row has
+// been unpacked, before the reduction, Step / Z and the codes (768 columns 5.45 -> 5.89 TB/s,
+// 3072 5.53 -> 6.36, 5120 5.92 -> 6.07, 9216 5.46 -> 5.85).  Shared memory: 768 bytes.
 //
 // The arithmetic is that of the staged kernel (rowquant_impl.cuh): binary32, no FMA
 // contraction across the two multiplies, ties to even, the literal path when a clamp could
@@ -22,6 +26,9 @@ namespace aweq {
 constexpr int kRdThreads = 256;
 // threads of a CTA: 256 (several teams), or the team itself when it has more than 8 warps
 __host__ __device__ constexpr int rd_threads(int TW) { return TW > 8 ? TW * 32 : kRdThreads; }
+// CTAs per SM the kernel is compiled for: three while the registers allow it (the next row's
+// raw vectors count when they are loaded early), else two; one for a team of a whole CTA
+__host__ __device__ constexpr int rd_ctas_per_sm(int TW, int V, bool PF) { return TW > 8 ? 1 : V <= (PF ? 3 : 4) ? 3 : 2; }
 
 struct RdSmem {
     float2 red[2][32];
@@ -92,9 +99,10 @@ __device__ __forceinline__ void rd_codes(const float2 (&x)[4], const QParams &q,
     }
 }
 
-// V: vectors per thread; TW: warps per team
-template <class D, int V, int TW, bool MU, bool BYTES_OUT>
-__global__ void __launch_bounds__(rd_threads(TW), TW > 8 ? 1 : V <= 4 ? 3 : 2)
+// V: vectors per thread; TW: warps per team; PF: the loads of the team's next row are issued
+// before the current row is reduced and quantised (two rows in flight per team)
+template <class D, int V, int TW, bool MU, bool BYTES_OUT, bool PF = false>
+__global__ void __launch_bounds__(rd_threads(TW), rd_ctas_per_sm(TW, V, PF))
 rowdirect_kernel(const RowQuantParams p)
 {
     __shared__ RdSmem sm;
@@ -125,19 +133,23 @@ rowdirect_kernel(const RowQuantParams p)
     }
 
     const long long nteams = (long long)gridDim.x * teams;
-    for (long long row = (long long)blockIdx.x * teams + tm; row < p.nrows; row += nteams) {
+    uint4 raw[V];
+    auto load_row = [&](long long row) {
         const uint16_t *xrow = p.X + row * p.ld;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const int idx = tt + v * T;
+            raw[v] = make_uint4(0, 0, 0, 0);
+            if (v < V - 1 || idx < p.nvec) raw[v] = ldg_stream(xrow + (size_t)idx * 8);
+        }
+    };
+    if (PF && (long long)blockIdx.x * teams + tm < p.nrows) load_row((long long)blockIdx.x * teams + tm);
+    for (long long row = (long long)blockIdx.x * teams + tm; row < p.nrows; row += nteams) {
         unsigned char *orow = p.out + row * p.out_pitch;
         float lo = INFINITY, hi = -INFINITY;
         float2 xh[V][4];
         {
-            uint4 raw[V];
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int idx = tt + v * T;
-                raw[v] = make_uint4(0, 0, 0, 0);
-                if (v < V - 1 || idx < p.nvec) raw[v] = ldg_stream(xrow + (size_t)idx * 8);
-            }
+            if (!PF) load_row(row);
 #pragma unroll
             for (int v = 0; v < V; ++v) {
                 const int idx = tt + v * T;
@@ -150,6 +162,7 @@ rowdirect_kernel(const RowQuantParams p)
                     }
                 }
             }
+            if (PF && row + nteams < p.nrows) load_row(row + nteams);
         }
         lo = redux_min(lo, 0xffffffffu);
         hi = redux_max(hi, 0xffffffffu);
@@ -193,32 +206,45 @@ rowdirect_kernel(const RowQuantParams p)
     }
 }
 
-template <class D, int V, int TW, bool MU, bool BYTES_OUT>
+template <class D, int V, int TW, bool MU, bool BYTES_OUT, bool PF = false>
 static aweq_status rd_launch_one(const RowQuantParams &p, cudaStream_t stream)
 {
     constexpr int teams = rd_threads(TW) / (TW * 32);
-    constexpr int per_sm = TW > 8 ? 1 : V <= 4 ? 3 : 2;
+    constexpr int per_sm = rd_ctas_per_sm(TW, V, PF);
     long long grid = (p.nrows + teams - 1) / teams;
     if (grid > (long long)kSmCount * per_sm) grid = (long long)kSmCount * per_sm;
     if (grid < 1) grid = 1;
-    AWEQ_LAUNCH((rowdirect_kernel<D, V, TW, MU, BYTES_OUT>), dim3((unsigned)grid), dim3(rd_threads(TW)), 0, stream, p);
+    AWEQ_LAUNCH((rowdirect_kernel<D, V, TW, MU, BYTES_OUT, PF>), dim3((unsigned)grid), dim3(rd_threads(TW)), 0, stream, p);
     return AWEQ_OK;
 }
 
-// mode: 0 = activations (one byte per code), 1 = weights with eps.mu sums, 2 = weights without
+// Largest V of the step-6 shapes: two rows of a team are in flight there, which the registers
+// hold up to six vectors per thread.
+constexpr int kRdActMaxV = 6;
+
+// mode: 0 = activations (one byte per code, next row's loads issued early), 1 = weights with eps.mu
+// sums, 2 = weights without
 template <class D, int V, int TW>
-static aweq_status rd_launch_mode(const RowQuantParams &p, int mode, cudaStream_t stream)
+static aweq_status rd_launch_weights(const RowQuantParams &p, int mode, cudaStream_t stream)
 {
     if (mode == 1) return rd_launch_one<D, V, TW, true, false>(p, stream);
-    if (mode == 2) return rd_launch_one<D, V, TW, false, false>(p, stream);
-    if constexpr (TW <= 2) return rd_launch_one<D, V, TW, false, true>(p, stream);
-    return AWEQ_ERR_UNSUPPORTED;
+    return rd_launch_one<D, V, TW, false, false>(p, stream);
 }
 
 template <class D>
 static aweq_status rd_launch(const RowQuantParams &p, int team_warps, int V, int mode, cudaStream_t stream)
 {
-#define AWEQ_RD_CASE(tw, v) if (team_warps == tw && V == v) return rd_launch_mode<D, v, tw>(p, mode, stream);
+    if (mode == 0) {
+        // the shapes plan_rowdirect gives step 6: one warp with 1-6 vectors, larger teams with 4-6
+#define AWEQ_RD_ACT(tw, v) if (team_warps == tw && V == v) return rd_launch_one<D, v, tw, false, true, true>(p, stream);
+        AWEQ_RD_ACT(1, 1) AWEQ_RD_ACT(1, 2) AWEQ_RD_ACT(1, 3) AWEQ_RD_ACT(1, 4) AWEQ_RD_ACT(1, 5) AWEQ_RD_ACT(1, 6)
+        AWEQ_RD_ACT(2, 4) AWEQ_RD_ACT(2, 5) AWEQ_RD_ACT(2, 6)
+        AWEQ_RD_ACT(4, 4) AWEQ_RD_ACT(4, 5) AWEQ_RD_ACT(4, 6)
+        AWEQ_RD_ACT(8, 4) AWEQ_RD_ACT(8, 5) AWEQ_RD_ACT(8, 6)
+#undef AWEQ_RD_ACT
+        return AWEQ_ERR_UNSUPPORTED;
+    }
+#define AWEQ_RD_CASE(tw, v) if (team_warps == tw && V == v) return rd_launch_weights<D, v, tw>(p, mode, stream);
     AWEQ_RD_CASE(1, 1) AWEQ_RD_CASE(1, 2) AWEQ_RD_CASE(1, 3) AWEQ_RD_CASE(1, 4) AWEQ_RD_CASE(1, 5)
     AWEQ_RD_CASE(1, 6) AWEQ_RD_CASE(1, 7) AWEQ_RD_CASE(1, 8) AWEQ_RD_CASE(1, 9) AWEQ_RD_CASE(1, 10)
     AWEQ_RD_CASE(2, 6) AWEQ_RD_CASE(2, 7) AWEQ_RD_CASE(2, 8) AWEQ_RD_CASE(2, 9) AWEQ_RD_CASE(2, 10)

@@ -74,7 +74,7 @@ bool rowquant_describe(long long rows, long long cols, bool weights, long long p
     int tw = 0, dv = 0;
     if (plan_rowdirect(cols, weights, &tw, &dv)) {
         // the plain-load kernel: no stages; teams take rows one by one
-        const int teams = rd_threads(tw) / (tw * 32), per_sm = tw > 8 ? 1 : dv <= 4 ? 3 : 2;
+        const int teams = rd_threads(tw) / (tw * 32), per_sm = rd_ctas_per_sm(tw, dv, !weights);
         long long grid = (rows + teams - 1) / teams;
         if (grid > (long long)kSmCount * per_sm) grid = (long long)kSmCount * per_sm;
         plan[0] = grid < 1 ? 1 : grid; plan[1] = rd_threads(tw); plan[2] = (long long)sizeof(RdSmem); plan[3] = tw * 32;

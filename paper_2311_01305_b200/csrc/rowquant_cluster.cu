@@ -20,6 +20,7 @@
 // says so; its peer then runs into the limit of its own wait.  Both reach the cluster-wide
 // barrier at the end of the kernel, which keeps a CTA's shared memory alive while the peer may
 // still write to it.
+#include <mutex>
 #include "rowquant_impl.cuh"
 
 namespace aweq {
@@ -167,7 +168,14 @@ __global__ void __launch_bounds__(kRcThreads, 1) rowquant_cluster_kernel(const R
                 cluster_mbar_arrive(cluster_map(&sm->xbar[par], peer));
             }
         }
-        if (!mbar_wait_cluster(&sm->xbar[par], (uint32_t)(k >> 1) & 1)) ok = false;
+        {
+            // one lane per warp polls; the warp barrier hands what it acquired to the other lanes
+            int got = 1;
+            if (lane == 0) got = mbar_wait_cluster(&sm->xbar[par], (uint32_t)(k >> 1) & 1) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            __syncwarp();
+            if (!got) ok = false;
+        }
 
         // ---- pass 2: Step, 1/Step, Z of the whole row from the two halves' extremes; codes of my half
         if (ok) {
@@ -269,7 +277,31 @@ static aweq_status rc_launch_one(const RowQuantParams &p, const RowQuantPlan &pl
 {
     auto kern = rowquant_cluster_kernel<D, V>;
     AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-    cudaError_t e = launch_pdl_cluster(kern, dim3(pl.grid), dim3(kRcThreads), pl.smem, stream, 2u, p);
+    // A persistent grid must be resident as a whole (a cluster that starts after the others doubles
+    // the run time): ask once how many clusters of this shape the device holds at the same time.
+    static std::mutex lock;
+    static size_t asked_smem = 0;
+    static int asked_resident = 0;
+    int resident;
+    {
+        std::lock_guard<std::mutex> hold(lock);
+        if (asked_smem != pl.smem) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(pl.grid); cfg.blockDim = dim3(kRcThreads); cfg.dynamicSmemBytes = pl.smem;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            int nc = 0;
+            AWEQ_CUDA_OK(cudaOccupancyMaxActiveClusters(&nc, kern, &cfg));
+            asked_resident = nc;
+            asked_smem = pl.smem;
+        }
+        resident = asked_resident;
+    }
+    int grid = pl.grid;
+    if (resident > 0 && grid > 2 * resident) grid = 2 * resident;
+    cudaError_t e = launch_pdl_cluster(kern, dim3(grid), dim3(kRcThreads), pl.smem, stream, 2u, p);
     note_launch();
     if (e != cudaSuccess) return cuda_failed(e);
     return AWEQ_OK;

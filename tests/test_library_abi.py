@@ -134,7 +134,10 @@ def test_row_quantiser_plans_fit_the_hardware(lib):
                     assert (threads == 256 and team <= 256 and V <= 10) or (threads == team == 1024 and V <= 5)
                     assert V >= 1 and team * (V - 1) < nvec
                     assert R == 0 and S == 0 and smem <= 1024
-                    assert op == 4 or cols <= 3072
+                    # step 6 has two rows of a team in flight: at most six vectors per thread, 12288 columns
+                    assert op == 4 or (cols <= 12288 and V <= 6 and threads == 256)
+                    # three CTAs per SM while the registers allow it, else two
+                    assert ctas <= 148 * (1 if team > 256 else 3 if V <= (3 if op == 6 else 4) else 2)
                     assert ctas <= max(1, -(-rows // (threads // team)))
                     continue
                 assert S >= 2 and R >= 1 and ctas <= 296
@@ -144,7 +147,7 @@ def test_row_quantiser_plans_fit_the_hardware(lib):
                     assert ctas % 2 == 0 and ctas <= 148 and 512 * V >= half and smem == 4096 + S * R * half * 16
                     continue
                 if wide:
-                    assert op == 6 and cols > 10240 and V <= 5 and team == threads and R <= 4
+                    assert op == 6 and cols > 12288 and V <= 5 and team == threads and R <= 4
                     assert smem >= 4096 + S * R * nvec * 16
                 else:
                     assert V <= 10 and smem == 512 + S * R * nvec * 16
