@@ -403,7 +403,7 @@ def time_layer_pass(wl, bits, X, W, steps, warmup, *, rank=0, world=1, local=0, 
     if wl.act_quant:
         act_ms = [sum(ea[0].elapsed_time(ea[1]) for _, ea in hk) for hk in hooks.values()]
         act_bytes = sum(3 * i.n_tokens * i.c_in + 8 * i.n_tokens for i in wl.inputs)
-        dom = {"kernel": "per-token quantiser: rowquant_kernel / rowquant_wide_kernel / rowquant_cluster_kernel by row width (aweq_quant_act)", "bytes": act_bytes,
+        dom = {"kernel": "per-token quantiser: rowdirect_kernel / rowquant_wide_kernel / rowquant_cluster_kernel by row width (aweq_quant_act)", "bytes": act_bytes,
                "ms": statistics.mean(act_ms), "launches_per_step": len(cal.passes),
                "stats_gbs": stats_bytes / statistics.mean(stats_ms) / 1e6}
     peak, peak_kind = measured_peaks()

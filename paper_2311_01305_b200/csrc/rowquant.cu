@@ -1,71 +1,15 @@
-// Host side of the row quantiser: how a row is split over threads, how many rows
-// form a stage, and the dispatch to the fp16 / bf16 instantiations.
+// Host side of the row quantisers: which kernel takes a row width (plain loads, the wide-row
+// ring, the cluster pair) and what the plan query reports for it.
 #include "rowdirect_impl.cuh"
 
 namespace aweq {
 
-// Everything that happens once per row (exchange of the extremes, Step, 1/Step, Z) is
-// repeated by every warp of the row's team, and a thread's last vector may be padding, so
-// the cost of a row is about (T / 32) * (V * c_vec + c_row) issue slots.  Pick the team
-// size that minimises it with V <= kRqMaxV.
-static void pick_team(int nvec, int *T_out, int *V_out)
-{
-    double best = 1e30;
-    int bestT = 0, bestV = 0;
-    for (int T = 32; T <= 512; T *= 2) {
-        const int V = (nvec + T - 1) / T;
-        if (V > kRqMaxV) continue;
-        const double c_vec = V <= kRqScaleRegsMaxV ? 55.0 : 59.0;
-        const double cost = (T / 32) * (V * c_vec + 90.0);
-        if (cost < best) { best = cost; bestT = T; bestV = V; }
-    }
-    *T_out = bestT;
-    *V_out = bestV;
-}
-
-bool plan_rowquant(long long nrows, long long cols, RowQuantPlan *out)
-{
-    const int nvec = (int)(cols / 8);
-    int T = 0, V = 0;
-    pick_team(nvec, &T, &V);
-    if (T == 0) return false;
-    RowQuantPlan p;
-    p.team = T;
-    p.V = V;
-    p.NT = T == 512 ? 512 : 256;
-    const int teams = p.NT / T;
-    const size_t row_bytes = (size_t)nvec * 16;
-    const size_t budget = (p.NT == 512 ? 200 * 1024 : 100 * 1024) - kRqHeader;
-    // rows per stage: about 32 KB, a multiple of the number of teams
-    int R = (int)(32768 / row_bytes);
-    R = R / teams * teams;
-    if (R < teams) R = teams;
-    if ((long long)R > nrows) R = (int)((nrows + teams - 1) / teams * teams);
-    if (R < 1) R = 1;
-    int S = (int)(budget / ((size_t)R * row_bytes));
-    while (S < 2 && R > 1) {
-        R = (R + 1) / 2;
-        S = (int)(budget / ((size_t)R * row_bytes));
-    }
-    if (S < 2) return false;          // the ring needs two stages
-    if (S > kRqStagesMax) S = kRqStagesMax;
-    p.rows_per_stage = R;
-    p.stages = S;
-    p.smem = kRqHeader + (size_t)S * R * row_bytes;
-    p.ntiles = (nrows + R - 1) / R;
-    const int per_sm = p.NT == 512 ? 1 : 2;
-    long long g = (long long)kSmCount * per_sm;
-    if (g > p.ntiles) g = p.ntiles;
-    if (g < 1) g = 1;
-    p.grid = (int)g;
-    *out = p;
-    return true;
-}
+// widest row any of the row quantisers takes
+constexpr long long kRowQuantMaxCols = 40960;
 
 bool rowquant_supported(long long nrows, long long cols)
 {
-    RowQuantPlan pl;
-    return plan_rowquant(nrows, cols, &pl);
+    return nrows >= 1 && cols >= 8 && cols <= kRowQuantMaxCols;
 }
 
 bool rowquant_describe(long long rows, long long cols, bool weights, long long plan[8])
@@ -83,9 +27,9 @@ bool rowquant_describe(long long rows, long long cols, bool weights, long long p
     }
     const bool pair = !weights && plan_rowquant_cluster(rows, cols, &pl);
     const bool wide = !pair && !weights && plan_rowquant_wide(rows, cols, &pl);
-    if (!pair && !wide && !plan_rowquant(rows, cols, &pl)) return false;
+    if (!pair && !wide) return false;
     plan[0] = pl.grid; plan[1] = pl.NT; plan[2] = (long long)pl.smem; plan[3] = pl.team; plan[4] = pl.V;
-    plan[5] = pl.rows_per_stage; plan[6] = pl.stages; plan[7] = pair ? 3 : wide ? 1 : 0;
+    plan[5] = pl.rows_per_stage; plan[6] = pl.stages; plan[7] = pair ? 3 : 1;
     return true;
 }
 
@@ -100,7 +44,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     const bool direct = plan_rowdirect(cols, weights, &tw, &dv);
     const bool pair = !direct && !weights && plan_rowquant_cluster(nrows, cols, &pl);
     const bool wide = !direct && !pair && !weights && plan_rowquant_wide(nrows, cols, &pl);
-    if (!direct && !pair && !wide && !plan_rowquant(nrows, cols, &pl)) return AWEQ_ERR_SHAPE;
+    if (!direct && !pair && !wide) return AWEQ_ERR_SHAPE;
     RowQuantParams p;
     p.X = reinterpret_cast<const uint16_t *>(X);
     p.nrows = nrows; p.ld = ld; p.nvec = (int)(cols / 8);
@@ -112,8 +56,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     const int mode = !weights ? 0 : ((mu && epsmu) ? 1 : 2);
     if (direct) return run_rowdirect(p, tw, dv, mode, dt, stream);
     if (pair) return run_rowquant_cluster(p, pl, dt, stream);
-    if (wide) return run_rowquant_wide(p, pl, dt, stream);
-    return dt == AWEQ_F16 ? rq_launch_f16(p, pl, mode, stream) : rq_launch_bf16(p, pl, mode, stream);
+    return run_rowquant_wide(p, pl, dt, stream);
 }
 
 }  // namespace aweq

@@ -1,20 +1,17 @@
-// Per-token quantiser of step 6 for wide rows (more than 10240 channels).
+// Per-token quantiser of step 6 for wide rows (12288 to 24576 channels; narrower rows go through
+// the plain-load kernel, wider ones through the cluster pair of rowquant_cluster.cu).
 //
-// The register-resident row quantiser needs a whole team of warps per row once a row no
-// longer fits the registers of a few warps, and then every row costs a team-wide exchange
-// and, worse, a second read of the per-channel factors from L1 / L2 (a 36864-channel factor
-// vector is 147 KB: larger than what L1 keeps beside the staging buffers).  Here the whole
-// CTA (512 or 1024 threads) works on a tile of R rows at a time; a thread owns the same V <= 5
-// column vectors in every row, so their factors stay on chip for the whole kernel (in
-// registers; with 1024 threads, where a thread has 64 registers, those of the fourth and
-// fifth vector sit in shared memory), and the rows are read twice from shared memory instead
-// of being kept in registers:
+// A row that no longer fits the registers of a few warps needs a whole team of warps, and then
+// every row costs a team-wide exchange.  Here the whole CTA (512 or 768 threads) works on a
+// tile of R rows at a time; a thread owns the same V <= 5 column vectors in every row, so their
+// factors stay in registers for the whole kernel, and the rows are read twice from shared
+// memory instead of being kept in registers:
 //   pass 1  x^ = x * (1/s), running min / max of each of the R rows     (no global loads)
 //   reduce  warp redux -> shared -> warp r finishes row r: Step, 1/Step, Z (Eq. 2)
 //   pass 2  x^ again, codes (Eq. 1), 8-byte coalesced stores
-// with two CTA-wide barriers per tile of R rows rather than per row.  Tiles arrive through
-// the same ring of bulk-copy (TMA) stages as in the register-resident kernel; warp 0 issues
-// the next tile at the top of each iteration.  Every wait is bounded.
+// with two CTA-wide barriers per tile of R rows rather than per row.  Tiles arrive through a
+// ring of bulk-copy (TMA) stages; warp 0 issues the next tile at the top of each iteration.
+// Every wait is bounded.
 #include "rowquant_impl.cuh"
 
 namespace aweq {
@@ -29,18 +26,12 @@ struct RwSmem {
 };
 static_assert(sizeof(RwSmem) <= kRwHeader, "header");
 
-// vectors per thread whose factors live in registers; the rest (1024-thread shape only) in shared memory
-__host__ __device__ constexpr int rw_reg_vectors(int V, int NT) { return NT == 1024 && V > 3 ? 3 : V; }
-__host__ __device__ constexpr size_t rw_scale_smem(int V, int NT) { return (size_t)(V - rw_reg_vectors(V, NT)) * NT * 32; }
-
 template <class D, int V, int NT>
 __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantParams p)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     RwSmem *sm = reinterpret_cast<RwSmem *>(smem_raw);
-    constexpr int VR = rw_reg_vectors(V, NT);
-    float4 *ssc = reinterpret_cast<float4 *>(smem_raw + kRwHeader);       // [(v - VR) * 2 + half][thread]
-    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw + kRwHeader + rw_scale_smem(V, NT));
+    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw + kRwHeader);
     constexpr int NW = NT / 32;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int R = p.rows_per_stage, S = p.stages;
@@ -65,7 +56,7 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
             rq_issue_tile(p, &sm->ring, stage_base, next_issue, S, R, stage_vecs, lane);
 
     // the factors of this thread's columns (no equalisation = ones, which is exact)
-    float2 sc[VR][4];
+    float2 sc[V][4];
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         const int idx = threadIdx.x + v * NT;
@@ -74,25 +65,10 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
             s0 = ldg_f4(p.scale + (size_t)idx * 8);
             s1 = ldg_f4(p.scale + (size_t)idx * 8 + 4);
         }
-        if (v < VR) {
-            sc[v][0] = make_float2(s0.x, s0.y); sc[v][1] = make_float2(s0.z, s0.w);
-            sc[v][2] = make_float2(s1.x, s1.y); sc[v][3] = make_float2(s1.z, s1.w);
-        } else {                                   // only this thread reads these back
-            ssc[((v - VR) * 2 + 0) * NT + threadIdx.x] = s0;
-            ssc[((v - VR) * 2 + 1) * NT + threadIdx.x] = s1;
-        }
+        sc[v][0] = make_float2(s0.x, s0.y); sc[v][1] = make_float2(s0.z, s0.w);
+        sc[v][2] = make_float2(s1.x, s1.y); sc[v][3] = make_float2(s1.z, s1.w);
     }
-#define AWEQ_RW_SCALES(v, f)                                                           \
-    float2 f[4];                                                                       \
-    if (v < VR) {                                                                      \
-        f[0] = sc[v < VR ? v : 0][0]; f[1] = sc[v < VR ? v : 0][1];                    \
-        f[2] = sc[v < VR ? v : 0][2]; f[3] = sc[v < VR ? v : 0][3];                    \
-    } else {                                                                           \
-        const float4 a = ssc[((v - VR) * 2 + 0) * NT + threadIdx.x];                   \
-        const float4 b = ssc[((v - VR) * 2 + 1) * NT + threadIdx.x];                   \
-        f[0] = make_float2(a.x, a.y); f[1] = make_float2(a.z, a.w);                    \
-        f[2] = make_float2(b.x, b.y); f[3] = make_float2(b.z, b.w);                    \
-    }
+#define AWEQ_RW_SCALES(v, f) const float2 (&f)[4] = sc[v];
 
     bool ok = true;
     for (long long k = 0; k < my_tiles; ++k) {
@@ -224,16 +200,15 @@ __global__ void __launch_bounds__(NT, 1) rowquant_wide_kernel(const RowQuantPara
 bool plan_rowquant_wide(long long nrows, long long cols, RowQuantPlan *out)
 {
     const int nvec = (int)(cols / 8);
-    if (nvec <= 1280 || nvec > 5 * 1024) return false;
+    if (nvec <= 1536 || nvec > 4 * 768) return false;
     RowQuantPlan p;
-    // 20481 .. 24576 columns: 768 threads with four vectors each keep two rows per stage (5.9 against
-    // 5.3 TB/s with 1024 threads); wider rows fill a stage alone and ran no faster with 768 threads
-    p.NT = nvec <= 5 * 512 ? 512 : nvec <= 4 * 768 ? 768 : 1024;
+    // up to 20480 columns 512 threads with four or five vectors each; 20481 .. 24576 columns 768 threads
+    // with four vectors each, which keeps two rows per stage
+    p.NT = nvec <= 5 * 512 ? 512 : 768;
     p.team = p.NT;
     p.V = (nvec + p.NT - 1) / p.NT;
     const size_t row_bytes = (size_t)nvec * 16;
-    const size_t scale_smem = rw_scale_smem(p.V, p.NT);
-    const size_t budget = 226 * 1024 - kRwHeader - scale_smem;
+    const size_t budget = 226 * 1024 - kRwHeader;
     int S = 2;
     int R = (int)(budget / (2 * row_bytes));
     if (R > kRwMaxR) R = kRwMaxR;
@@ -248,7 +223,7 @@ bool plan_rowquant_wide(long long nrows, long long cols, RowQuantPlan *out)
     if ((long long)R > nrows) R = (int)nrows;
     p.rows_per_stage = R;
     p.stages = S;
-    p.smem = kRwHeader + scale_smem + (size_t)S * R * row_bytes;
+    p.smem = kRwHeader + (size_t)S * R * row_bytes;
     p.ntiles = (nrows + R - 1) / R;
     long long g = kSmCount;
     if (g > p.ntiles) g = p.ntiles;
@@ -269,12 +244,9 @@ static aweq_status rw_launch_one(const RowQuantParams &p, const RowQuantPlan &pl
 template <class D>
 static aweq_status rw_launch(const RowQuantParams &p, const RowQuantPlan &pl, cudaStream_t stream)
 {
-#define AWEQ_RW_CASE(v)                                                              \
-    case v:                                                                          \
-        return pl.NT == 1024 ? rw_launch_one<D, v, 1024>(p, pl, stream) : rw_launch_one<D, v, 512>(p, pl, stream);
-    if (pl.NT == 768) return pl.V == 4 ? rw_launch_one<D, 4, 768>(p, pl, stream) : AWEQ_ERR_UNSUPPORTED;
-    switch (pl.V) { AWEQ_RW_CASE(1) AWEQ_RW_CASE(2) AWEQ_RW_CASE(3) AWEQ_RW_CASE(4) AWEQ_RW_CASE(5) }
-#undef AWEQ_RW_CASE
+    if (pl.NT == 768 && pl.V == 4) return rw_launch_one<D, 4, 768>(p, pl, stream);
+    if (pl.NT == 512 && pl.V == 4) return rw_launch_one<D, 4, 512>(p, pl, stream);
+    if (pl.NT == 512 && pl.V == 5) return rw_launch_one<D, 5, 512>(p, pl, stream);
     return AWEQ_ERR_UNSUPPORTED;
 }
 

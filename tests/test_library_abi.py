@@ -146,12 +146,9 @@ def test_row_quantiser_plans_fit_the_hardware(lib):
                     assert op == 6 and cols > 24576 and threads == 512 and team == 1024 and V <= 5 and R <= 4
                     assert ctas % 2 == 0 and ctas <= 148 and 512 * V >= half and smem == 4096 + S * R * half * 16
                     continue
-                if wide:
-                    assert op == 6 and cols > 12288 and V <= 5 and team == threads and R <= 4
-                    assert smem >= 4096 + S * R * nvec * 16
-                else:
-                    assert V <= 10 and smem == 512 + S * R * nvec * 16
-                    assert R % (threads // team) == 0 or R >= rows              # whole rounds of teams per stage
+                assert wide == 1                                # a tile of whole rows per CTA
+                assert op == 6 and cols > 12288 and V <= 5 and team == threads and R <= 4
+                assert smem >= 4096 + S * R * nvec * 16
     # beyond the supported width the query says so instead of planning something that cannot launch
     assert _plan(lib, 6, 100, 40968)[0] == 2 and _plan(lib, 4, 100, 81920)[0] == 2
     assert _plan(lib, 6, 100, 36)[0] == 2 and _plan(lib, 5, 100, 64)[0] == 9
