@@ -103,12 +103,11 @@ unsigned long long aweq_launch_count(void);
  *   column reduction: {CTAs, threads, shared bytes, column slabs, slab width in 16-byte vectors,
  *                      row splits, row phases, rows per stage}
  *   row quantisers:   {CTAs, threads, shared bytes, threads per row, vectors per thread,
- *                      rows per stage, stages, kernel: 1 shared-memory stages, a tile of rows per
- *                      CTA (step 6, 12296 to 24576 columns), 2 plain loads without stages (rows
- *                      per stage and stages are 0 then; step 4 at every width, step 6 up to 12288
- *                      columns), 3 staged with every row shared by a cluster of two CTAs (step 6
- *                      beyond 24576 columns; threads per row = twice the threads of a CTA,
- *                      shared bytes for half-rows)}
+ *                      rows per stage, stages, kernel: 2 plain loads without stages (rows per stage
+ *                      and stages are 0 then; step 4 at every width, step 6 up to 36864 columns),
+ *                      3 shared-memory stages with every row shared by a cluster of two CTAs (step 6
+ *                      beyond 36864 columns; threads per row = twice the threads of a CTA, shared
+ *                      bytes for half-rows)}
  * Returns AWEQ_ERR_SHAPE when the shape is not supported, AWEQ_ERR_UNSUPPORTED for other ops. */
 aweq_status aweq_plan_query(int op, long long rows, long long cols, long long plan[8]);
 

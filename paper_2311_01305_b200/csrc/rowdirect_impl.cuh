@@ -218,9 +218,11 @@ static aweq_status rd_launch_one(const RowQuantParams &p, cudaStream_t stream)
     return AWEQ_OK;
 }
 
-// Largest V of the step-6 shapes: two rows of a team are in flight there, which the registers
-// hold up to six vectors per thread.
-constexpr int kRdActMaxV = 6;
+// Largest V of the step-6 shapes: two rows of a team are in flight there, which 128 registers hold
+// up to nine vectors per thread (nine spills a few words in the small teams and still measured 5-8 %
+// faster than a larger team with five; ten spills over a hundred bytes and loses a quarter).
+constexpr int kRdActMaxV = 9;
+constexpr int kRdActMaxTeamWarps = 16;
 
 // mode: 0 = activations (one byte per code, next row's loads issued early), 1 = weights with eps.mu
 // sums, 2 = weights without
@@ -235,12 +237,14 @@ template <class D>
 static aweq_status rd_launch(const RowQuantParams &p, int team_warps, int V, int mode, cudaStream_t stream)
 {
     if (mode == 0) {
-        // the shapes plan_rowdirect gives step 6: one warp with 1-6 vectors, larger teams with 4-6
+        // the shapes plan_rowdirect gives step 6: one warp with 1-9 vectors, larger teams with 5-9
 #define AWEQ_RD_ACT(tw, v) if (team_warps == tw && V == v) return rd_launch_one<D, v, tw, false, true, true>(p, stream);
         AWEQ_RD_ACT(1, 1) AWEQ_RD_ACT(1, 2) AWEQ_RD_ACT(1, 3) AWEQ_RD_ACT(1, 4) AWEQ_RD_ACT(1, 5) AWEQ_RD_ACT(1, 6)
-        AWEQ_RD_ACT(2, 4) AWEQ_RD_ACT(2, 5) AWEQ_RD_ACT(2, 6)
-        AWEQ_RD_ACT(4, 4) AWEQ_RD_ACT(4, 5) AWEQ_RD_ACT(4, 6)
-        AWEQ_RD_ACT(8, 4) AWEQ_RD_ACT(8, 5) AWEQ_RD_ACT(8, 6)
+        AWEQ_RD_ACT(1, 7) AWEQ_RD_ACT(1, 8) AWEQ_RD_ACT(1, 9)
+        AWEQ_RD_ACT(2, 5) AWEQ_RD_ACT(2, 6) AWEQ_RD_ACT(2, 7) AWEQ_RD_ACT(2, 8) AWEQ_RD_ACT(2, 9)
+        AWEQ_RD_ACT(4, 5) AWEQ_RD_ACT(4, 6) AWEQ_RD_ACT(4, 7) AWEQ_RD_ACT(4, 8) AWEQ_RD_ACT(4, 9)
+        AWEQ_RD_ACT(8, 5) AWEQ_RD_ACT(8, 6) AWEQ_RD_ACT(8, 7) AWEQ_RD_ACT(8, 8) AWEQ_RD_ACT(8, 9)
+        AWEQ_RD_ACT(16, 5) AWEQ_RD_ACT(16, 6) AWEQ_RD_ACT(16, 7) AWEQ_RD_ACT(16, 8) AWEQ_RD_ACT(16, 9)
 #undef AWEQ_RD_ACT
         return AWEQ_ERR_UNSUPPORTED;
     }

@@ -1,5 +1,5 @@
-// Host side of the row quantisers: which kernel takes a row width (plain loads, the wide-row
-// ring, the cluster pair) and what the plan query reports for it.
+// Host side of the row quantisers: which kernel takes a row width (plain loads; for step 6 beyond
+// 36864 channels the cluster pair) and what the plan query reports for it.
 #include "rowdirect_impl.cuh"
 
 namespace aweq {
@@ -25,11 +25,9 @@ bool rowquant_describe(long long rows, long long cols, bool weights, long long p
         plan[4] = dv; plan[5] = 0; plan[6] = 0; plan[7] = 2;
         return true;
     }
-    const bool pair = !weights && plan_rowquant_cluster(rows, cols, &pl);
-    const bool wide = !pair && !weights && plan_rowquant_wide(rows, cols, &pl);
-    if (!pair && !wide) return false;
+    if (weights || !plan_rowquant_cluster(rows, cols, &pl)) return false;
     plan[0] = pl.grid; plan[1] = pl.NT; plan[2] = (long long)pl.smem; plan[3] = pl.team; plan[4] = pl.V;
-    plan[5] = pl.rows_per_stage; plan[6] = pl.stages; plan[7] = pair ? 3 : 1;
+    plan[5] = pl.rows_per_stage; plan[6] = pl.stages; plan[7] = 3;
     return true;
 }
 
@@ -43,8 +41,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     int tw = 0, dv = 0;
     const bool direct = plan_rowdirect(cols, weights, &tw, &dv);
     const bool pair = !direct && !weights && plan_rowquant_cluster(nrows, cols, &pl);
-    const bool wide = !direct && !pair && !weights && plan_rowquant_wide(nrows, cols, &pl);
-    if (!direct && !pair && !wide) return AWEQ_ERR_SHAPE;
+    if (!direct && !pair) return AWEQ_ERR_SHAPE;
     RowQuantParams p;
     p.X = reinterpret_cast<const uint16_t *>(X);
     p.nrows = nrows; p.ld = ld; p.nvec = (int)(cols / 8);
@@ -55,8 +52,7 @@ aweq_status run_rowquant(const void *X, aweq_dtype dt, long long nrows, long lon
     p.st = st;
     const int mode = !weights ? 0 : ((mu && epsmu) ? 1 : 2);
     if (direct) return run_rowdirect(p, tw, dv, mode, dt, stream);
-    if (pair) return run_rowquant_cluster(p, pl, dt, stream);
-    return run_rowquant_wide(p, pl, dt, stream);
+    return run_rowquant_cluster(p, pl, dt, stream);
 }
 
 }  // namespace aweq

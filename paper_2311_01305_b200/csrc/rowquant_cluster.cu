@@ -1,17 +1,18 @@
-// Per-token quantiser of step 6 for the widest rows (more than 24576 channels): a row is shared by
-// the two CTAs of a thread-block cluster.
+// Per-token quantiser of step 6 for the widest rows (more than 36864 channels, where the plain-load
+// kernel would need ten vectors per thread and spills): a row is shared by the two CTAs of a
+// thread-block cluster.
 //
-// A row of 36864 fp16 channels is 72 KB.  With one CTA per row only one row fits a stage of the
+// A row of 40960 fp16 channels is 80 KB.  With one CTA per row only one row fits a stage of a
 // bulk-copy ring, the CTA needs 1024 threads, and the factors of its columns do not all fit
-// in registers: two CTA-wide barriers per row, 4.9 TB/s.  Here the two CTAs of a cluster (two SMs)
-// each take half of the columns of the same rows, which makes each of them the well-behaved
-// case of the wide-row kernel -- 512 threads, at most five 16-byte vectors per thread, every
-// factor in registers, tiles of several half-rows per stage.  What the two halves must share is
+// in registers.  Here the two CTAs of a cluster (two SMs) each take half of the columns of the
+// same rows: 512 threads, five 16-byte vectors per thread, every factor in registers, tiles of
+// two half-rows per stage, which the whole CTA reads twice from shared memory (extremes, then
+// codes) with two CTA-wide barriers per tile.  What the two halves must share is
 // the pair of extremes of every row (Eq. 2 needs max and min over the whole row): after the first
 // pass a warp per row writes the CTA's (lo, hi) into its own and, through distributed shared
-// memory, into the peer's exchange slot and arrives on both CTAs' exchange barrier; every thread
-// then waits (bounded) for the eight arrivals of the tile, forms Step, 1/Step and Z from the two
-// halves' extremes itself, and runs the second pass on its half.  The CTAs of a pair run the same
+// memory, into the peer's exchange slot and arrives on both CTAs' exchange barrier; one lane of every
+// warp waits (bounded) for the eight arrivals of the tile, and every thread forms Step, 1/Step and Z from
+// the two halves' extremes itself and runs the second pass on its half.  The CTAs of a pair run the same
 // tiles in the same order, so the exchange needs no further hand-shake: a slot of parity k & 1 is
 // rewritten for tile k + 2 only after its owner has sent its extremes of tile k + 1, which it
 // does after reading the slot for tile k.
@@ -247,7 +248,7 @@ __global__ void __launch_bounds__(kRcThreads, 1) rowquant_cluster_kernel(const R
 bool plan_rowquant_cluster(long long nrows, long long cols, RowQuantPlan *out)
 {
     const int nvec = (int)(cols / 8);
-    if (nvec <= 3072 || nvec > 5120) return false;
+    if (nvec <= 4608 || nvec > 5120) return false;
     const int half0 = (nvec + 1) / 2;
     RowQuantPlan p;
     p.NT = kRcThreads;
@@ -311,7 +312,6 @@ template <class D>
 static aweq_status rc_launch(const RowQuantParams &p, const RowQuantPlan &pl, cudaStream_t stream)
 {
     switch (pl.V) {
-    case 4: return rc_launch_one<D, 4>(p, pl, stream);
     case 5: return rc_launch_one<D, 5>(p, pl, stream);
     }
     return AWEQ_ERR_UNSUPPORTED;

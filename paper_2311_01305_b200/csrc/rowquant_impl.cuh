@@ -1,5 +1,5 @@
 // What the row-wise Eq. 1-2 quantisers share: the kernel parameters and launch plans, the
-// shared-memory ring of the staged kernels (rowquant_wide.cu, rowquant_cluster.cu: persistent
+// barriers of the shared-memory ring of the staged kernel (rowquant_cluster.cu: persistent
 // CTAs pull tiles of rows through stages filled by 1-D bulk copies, completion on mbarriers,
 // warp 0 issues the copies between its own work) and the code packing.
 //
@@ -44,8 +44,6 @@ struct RowQuantPlan {
     long long ntiles;
 };
 
-// wide rows of step 6 (rowquant_wide.cu): a plan exists for 12288 < cols <= 24576
-bool plan_rowquant_wide(long long nrows, long long cols, RowQuantPlan *out);
 
 struct RqSmem {
     uint64_t full[kRqStagesMax];
@@ -107,32 +105,7 @@ __device__ __forceinline__ bool rq_stage_free(RqSmem *sm, long long t, int S, bo
     return ready;
 }
 
-// warp 0: start the copy of tile `t` of this CTA into its (free) stage.
-__device__ __forceinline__ void rq_issue_tile(const RowQuantParams &p, RqSmem *sm, uint4 *stage_base, long long t,
-                                              int S, int R, size_t stage_vecs, int lane)
-{
-    const int s = (int)(t % S);
-    const long long row0 = (blockIdx.x + t * gridDim.x) * (long long)R;
-    const int rows = (int)min((long long)R, p.nrows - row0);
-    const uint32_t row_bytes = (uint32_t)p.nvec * 16u;
-    uint4 *dst = stage_base + (size_t)s * stage_vecs;
-    if (lane == 0) mbar_arrive_expect_tx(&sm->full[s], (uint32_t)rows * row_bytes);
-    __syncwarp();
-    if (p.ld == (long long)p.nvec * 8) {
-        // the tile is one contiguous range: a copy per 32 KB chunk
-        const uint32_t total = (uint32_t)rows * row_bytes;
-        const uint32_t chunk = 32768u;
-        const char *src = reinterpret_cast<const char *>(p.X + row0 * p.ld);
-        for (uint32_t off = lane * chunk; off < total; off += 32u * chunk)
-            bulk_g2s(reinterpret_cast<char *>(dst) + off, src + off, min(chunk, total - off), &sm->full[s]);
-    } else {
-        for (int r = lane; r < rows; r += 32)
-            bulk_g2s(dst + (size_t)r * p.nvec, p.X + (row0 + r) * p.ld, row_bytes, &sm->full[s]);
-    }
-}
-
-aweq_status run_rowquant_wide(const RowQuantParams &p, const RowQuantPlan &pl, aweq_dtype dt, cudaStream_t stream);
-// rows of step 6 beyond 24576 channels, each shared by a cluster of two CTAs (rowquant_cluster.cu)
+// rows of step 6 beyond 36864 channels, each shared by a cluster of two CTAs (rowquant_cluster.cu)
 bool plan_rowquant_cluster(long long nrows, long long cols, RowQuantPlan *out);
 aweq_status run_rowquant_cluster(const RowQuantParams &p, const RowQuantPlan &pl, aweq_dtype dt, cudaStream_t stream);
 

@@ -128,27 +128,25 @@ def test_row_quantiser_plans_fit_the_hardware(lib):
                 rc, (ctas, threads, smem, team, V, R, S, wide) = _plan(lib, op, rows, cols)
                 assert rc == 0, (op, rows, cols)
                 nvec = cols // 8
-                assert 1 <= ctas <= 444 and threads in (256, 512, 768, 1024) and smem <= SMEM_LIMIT
+                assert 1 <= ctas <= 444 and threads in (256, 512, 1024) and smem <= SMEM_LIMIT
                 assert team % 32 == 0 and (threads % team == 0 or team == 2 * threads) and team * V >= nvec      # the row is covered
                 if wide == 2:                                   # plain loads: no stages, a row per team
-                    assert (threads == 256 and team <= 256 and V <= 10) or (threads == team == 1024 and V <= 5)
                     assert V >= 1 and team * (V - 1) < nvec
                     assert R == 0 and S == 0 and smem <= 1024
-                    # step 6 has two rows of a team in flight: at most six vectors per thread, 12288 columns
-                    assert op == 4 or (cols <= 12288 and V <= 6 and threads == 256)
-                    # three CTAs per SM while the registers allow it, else two
+                    if op == 4:
+                        assert (threads == 256 and team <= 256 and V <= 10) or (threads == team == 1024 and V <= 5)
+                    else:
+                        # step 6 has two rows of a team in flight: at most nine vectors per thread, teams of up to 16 warps
+                        assert cols <= 36864 and V <= 9 and ((threads == 256 and team <= 256) or threads == team == 512)
+                    # three CTAs per SM while the registers allow it, else two; one when the team is a whole large CTA
                     assert ctas <= 148 * (1 if team > 256 else 3 if V <= (3 if op == 6 else 4) else 2)
                     assert ctas <= max(1, -(-rows // (threads // team)))
                     continue
-                assert S >= 2 and R >= 1 and ctas <= 296
-                if wide == 3:                                   # a row per cluster of two CTAs, half a row each
-                    half = (nvec + 1) // 2
-                    assert op == 6 and cols > 24576 and threads == 512 and team == 1024 and V <= 5 and R <= 4
-                    assert ctas % 2 == 0 and ctas <= 148 and 512 * V >= half and smem == 4096 + S * R * half * 16
-                    continue
-                assert wide == 1                                # a tile of whole rows per CTA
-                assert op == 6 and cols > 12288 and V <= 5 and team == threads and R <= 4
-                assert smem >= 4096 + S * R * nvec * 16
+                # a row per cluster of two CTAs, half a row each, in shared-memory stages
+                half = (nvec + 1) // 2
+                assert wide == 3 and op == 6 and cols > 36864 and threads == 512 and team == 1024 and V == 5 and R <= 4
+                assert S >= 2 and R >= 1
+                assert ctas % 2 == 0 and ctas <= 148 and 512 * V >= half and smem == 4096 + S * R * half * 16
     # beyond the supported width the query says so instead of planning something that cannot launch
     assert _plan(lib, 6, 100, 40968)[0] == 2 and _plan(lib, 4, 100, 81920)[0] == 2
     assert _plan(lib, 6, 100, 36)[0] == 2 and _plan(lib, 5, 100, 64)[0] == 9
