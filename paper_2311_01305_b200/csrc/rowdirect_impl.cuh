@@ -12,10 +12,11 @@
 // ring spends most of its time filling and draining.  On the long runs of rows of step 6 the
 // resident teams alone leave the kernel waiting for loads (24 warps x 1.5 KB in flight per SM at
 // 768 columns): there a team issues the loads of its next row as soon as the current row has
-// been unpacked, before the reduction, Step / Z and the codes (768 columns 5.45 -> 5.89 TB/s,
-// 3072 5.53 -> 6.36, 5120 5.92 -> 6.07, 9216 5.46 -> 5.85).  Shared memory: 768 bytes.
+// been unpacked, before the reduction, Step / Z and the codes, and holds as many vectors per thread
+// as the registers allow (768 columns 5.45 -> 5.90 TB/s, 3072 5.53 -> 6.39, 5120 5.92 -> 6.07,
+// 9216 5.46 -> 6.27, 13824 6.05 -> 6.35, 36864 5.23 -> 6.14).  Shared memory: 768 bytes.
 //
-// The arithmetic is that of the staged kernel (rowquant_impl.cuh): binary32, no FMA
+// The arithmetic (see rowquant_impl.cuh): binary32, no FMA
 // contraction across the two multiplies, ties to even, the literal path when a clamp could
 // fire or the zero-point is too large for the add-constant rounding.
 #pragma once

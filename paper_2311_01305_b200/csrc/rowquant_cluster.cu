@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(kRcThreads, 1) rowquant_cluster_kernel(const R
         if (warp == 0 && next_issue < my_tiles) {
             // tile k + S - 1 goes into the stage that tile k - 1 released
             bool timed_out = false;
-            if (rq_stage_free(&sm->ring, next_issue, S, true, &timed_out)) {
+            if (rq_stage_free(&sm->ring, next_issue, S, &timed_out)) {
                 issue(next_issue);
                 ++next_issue;
             }

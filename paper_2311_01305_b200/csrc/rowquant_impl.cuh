@@ -87,21 +87,16 @@ __device__ __forceinline__ void store_codes(unsigned char *dst, const uint32_t (
     }
 }
 
-// warp 0: is the stage of tile `t` free again (released by every warp after its previous
-// use)?  Blocking (bounded) or a single test.  *timed_out is set when a blocking wait gave up.
-__device__ __forceinline__ bool rq_stage_free(RqSmem *sm, long long t, int S, bool block, bool *timed_out)
+// warp 0: wait (bounded) until the stage of tile `t` is free again, i.e. released by every warp
+// after its previous use.  *timed_out is set when the wait gave up.
+__device__ __forceinline__ bool rq_stage_free(RqSmem *sm, long long t, int S, bool *timed_out)
 {
     const int s = (int)(t % S);
     const uint32_t use = (uint32_t)(t / S);
     if (use == 0) return true;
-    bool ready;
-    if (block) {
-        ready = mbar_wait(&sm->empty[s], (use - 1) & 1);
-        ready = __all_sync(0xffffffffu, ready);
-        if (!ready) *timed_out = true;
-    } else {
-        ready = __all_sync(0xffffffffu, mbar_test(&sm->empty[s], (use - 1) & 1));
-    }
+    bool ready = mbar_wait(&sm->empty[s], (use - 1) & 1);
+    ready = __all_sync(0xffffffffu, ready);
+    if (!ready) *timed_out = true;
     return ready;
 }
 
