@@ -434,7 +434,7 @@ def time_layer_pass(wl, bits, X, W, steps, warmup, *, rank=0, world=1, local=0, 
            "launch": ("CUDA graph replay; every fourth step eager, with the event hooks" if mixed
                       else "one CUDA graph replay per step" if graph is not None else "eager"),
            "launch_trial": trial,
-           "schedule": ("two streams: column reductions and step 6 on one, factors and weight quantiser on the other"
+           "schedule": ("column reductions and step 6 on one stream, factors and weight quantisers on others (one per input for weight-only workloads, one in all for W8A8)"
                         if getattr(cal, "overlap", False) else "one stream")}
     return cal, res
 
