@@ -380,18 +380,18 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
 constexpr int kFinCols = 32, kFinLanes = 32;
 
 template <bool WITH_SUM>
-__global__ void __launch_bounds__(kFinCols * kFinLanes)
-colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restrict__ pmax,
-                          const double *__restrict__ psum, int nsplit, long long cols, long long nrows, float *omin,
-                          float *omax, float *omean, double *osum, const long long *count, int accumulate,
-                          aweq_dev_status *st, float *negmin_max, double *count_f64)
+__device__ __forceinline__ void colreduce_finalize_block(unsigned block, const float *__restrict__ pmin,
+                                                         const float *__restrict__ pmax, const double *__restrict__ psum,
+                                                         int nsplit, long long cols, long long nrows, float *omin,
+                                                         float *omax, float *omean, double *osum, const long long *count,
+                                                         int accumulate, aweq_dev_status *st, float *negmin_max,
+                                                         double *count_f64)
 {
     __shared__ float slo[kFinLanes][kFinCols], shi[kFinLanes][kFinCols];
-    __shared__ double ssum[kFinLanes][kFinCols];
-    pdl_begin();
-    if (count_f64 && blockIdx.x == 0 && threadIdx.x == 0) *count_f64 = (double)nrows;
+    __shared__ double ssum[WITH_SUM ? kFinLanes : 1][kFinCols];
+    if (count_f64 && block == 0 && threadIdx.x == 0) *count_f64 = (double)nrows;
     const int c = threadIdx.x % kFinCols, k0 = threadIdx.x / kFinCols;
-    const long long j = (long long)blockIdx.x * kFinCols + c;
+    const long long j = (long long)block * kFinCols + c;
     float lo = INFINITY, hi = -INFINITY;
     double sum = 0.0;
     if (j < cols) {
@@ -434,6 +434,41 @@ colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restric
         bool bad = (nrows > 0 || accumulate) && !(isfinite(lo) && isfinite(hi) && isfinite(sum));
         if (bad) atomicAdd(&st->nonfinite, 1ull);
     }
+}
+
+template <bool WITH_SUM>
+__global__ void __launch_bounds__(kFinCols * kFinLanes)
+colreduce_finalize_kernel(const float *__restrict__ pmin, const float *__restrict__ pmax,
+                          const double *__restrict__ psum, int nsplit, long long cols, long long nrows, float *omin,
+                          float *omax, float *omean, double *osum, const long long *count, int accumulate,
+                          aweq_dev_status *st, float *negmin_max, double *count_f64)
+{
+    pdl_begin();
+    colreduce_finalize_block<WITH_SUM>(blockIdx.x, pmin, pmax, psum, nsplit, cols, nrows, omin, omax, omean, osum, count,
+                                       accumulate, st, negmin_max, count_f64);
+}
+
+// Both jobs of a fused statistics + weight-range launch in one finalize launch: the first `blocks_a`
+// blocks finish job A (with the sums), the others job B (extremes only).
+struct FinalizeB {
+    const float *pmin, *pmax;
+    long long nrows;
+    float *omin, *omax;
+};
+__global__ void __launch_bounds__(kFinCols * kFinLanes)
+colreduce_finalize_pair_kernel(const float *__restrict__ pmin, const float *__restrict__ pmax,
+                               const double *__restrict__ psum, int nsplit, long long cols, long long nrows, float *omin,
+                               float *omax, float *omean, double *osum, aweq_dev_status *st, float *negmin_max,
+                               double *count_f64, unsigned blocks_a, const FinalizeB b)
+{
+    pdl_begin();
+    if (blockIdx.x < blocks_a)
+        colreduce_finalize_block<true>(blockIdx.x, pmin, pmax, psum, nsplit, cols, nrows, omin, omax, omean, osum,
+                                       (const long long *)nullptr, 0, st, negmin_max, count_f64);
+    else
+        colreduce_finalize_block<false>(blockIdx.x - blocks_a, b.pmin, b.pmax, (const double *)nullptr, nsplit, cols, b.nrows,
+                                        b.omin, b.omax, (float *)nullptr, (double *)nullptr, (const long long *)nullptr, 0, st,
+                                        (float *)nullptr, (double *)nullptr);
 }
 
 __global__ void bump_count_kernel(long long *count, long long nrows, int accumulate)
@@ -491,7 +526,17 @@ static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *
                     segs, rows_all, p.nvec, p.nslab, p.slab_w, p.phases, p.stage_rows, p.rows_per_split, cols, pmin, pmax,
                     psum, st, rows, rps_b, pmin_b, pmax_b);
     }
-    AWEQ_LAUNCH(colreduce_finalize_kernel<WITH_SUM>, dim3((unsigned)((cols + kFinCols - 1) / kFinCols)),
+    const unsigned fin_blocks = (unsigned)((cols + kFinCols - 1) / kFinCols);
+    if constexpr (WITH_SUM) {
+        if (rows_b > 0 && !accumulate && !count) {
+            const FinalizeB fb = {pmin_b, pmax_b, rows_b, omin_b, omax_b};
+            AWEQ_LAUNCH(colreduce_finalize_pair_kernel, dim3(2 * fin_blocks), dim3(kFinCols * kFinLanes), 0, stream,
+                        (const float *)pmin, (const float *)pmax, (const double *)psum, nsplit_eff, cols, rows, omin, omax,
+                        omean, osum, st, negmin_max, count_f64, fin_blocks, fb);
+            return AWEQ_OK;
+        }
+    }
+    AWEQ_LAUNCH(colreduce_finalize_kernel<WITH_SUM>, dim3(fin_blocks),
                 dim3(kFinCols * kFinLanes), 0, stream, (const float *)pmin, (const float *)pmax, (const double *)psum,
                 nsplit_eff, cols, rows, omin, omax, omean, osum, (const long long *)count, accumulate, st, negmin_max,
                 count_f64);
