@@ -483,6 +483,37 @@ def test_quant_act_degenerate_rows():
         util.assert_same_values(a, b)
 
 
+@pytest.mark.parametrize("C", [2304, 5120, 13824, 36864, 40960])
+def test_quant_act_wide_degenerate_rows_and_pitch(C):
+    """The degenerate rows of the narrow test at the widths of the larger teams (one warp with nine
+    vectors, four, eight and sixteen warps, the cluster pair), inside a wider allocation (row pitch
+    C + 64), with a factor vector: constant and zero rows, one-sided rows, a row whose top rounds past
+    2^b - 1 (the literal path), the largest finite values, and rows with Inf."""
+    g = torch.Generator().manual_seed(17)
+    X = torch.randn((11, C + 64), generator=g)
+    X[0] = 3.0
+    X[1] = 0.0
+    X[2] = X[2].abs() + 5
+    X[3] = -X[3].abs() - 5
+    X[4, :C // 2] = 2000.0
+    X[4, C // 2:] = 2001.0
+    X[5] = 65504.0
+    X[5, 1::2] = -65504.0
+    X[6, C - 1] = 300.0                       # the extreme sits in the last vector of the row
+    X[7, 0] = -300.0                          # ... and in the first
+    X[8, C // 2 + 3] = float("inf")
+    X[9, 5] = float("-inf")
+    big = X.to(torch.float16).to(DEV)
+    Xv = big[:, :C]
+    assert Xv.stride(0) == C + 64
+    rinv = (torch.rand(C, generator=g) + 0.5).numpy()
+    o = orc.quant_act(util.bits(Xv), orc.F16, rinv, orc.PER_ROW)
+    d = dev_quant_act(Xv, rinv, 8, aweq.PER_ROW)
+    util.assert_same_values(d[2], o[2], "zero-points")
+    util.assert_same_values(d[1], o[1], "Step")
+    util.assert_same_values(d[0], o[0], "codes")
+
+
 def test_quant_act_int32_saturation_and_nonfinite():
     """Step 6 on the hand-worked saturation cases (ones times 1/s values that carry the data)
     and on rows with Inf / NaN elements: the oracle's numbers, element by element."""
