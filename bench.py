@@ -335,16 +335,7 @@ def time_layer_pass(wl, bits, X, W, steps, warmup, *, rank=0, world=1, local=0, 
     # quantiser): a short trial of both launch modes before the timed region picks the one that is timed.
     trial = None
     if graph is not None and not graph_only:
-        def trial_ms(step_fn, n=3):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            a.record()
-            for _ in range(n):
-                step_fn()
-            b.record()
-            torch.cuda.synchronize()
-            return a.elapsed_time(b) / n
-        trial = {"eager_ms": trial_ms(cal.run), "graph_ms": trial_ms(graph.replay)}
+        trial = cal.launch_trial(graph, 3)
         if trial["eager_ms"] < 0.995 * trial["graph_ms"]:
             graph = None
     mixed = graph is not None and not graph_only

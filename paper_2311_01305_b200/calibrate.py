@@ -222,6 +222,23 @@ class LayerCalibrator:
             self.run()
         return graph
 
+    def launch_trial(self, graph, steps: int = 3) -> dict:
+        """Device time per pass of ``run()`` and of ``graph.replay()`` over ``steps`` passes each
+        (CUDA events, a synchronise around each measurement): ``{"eager_ms": .., "graph_ms": ..}``.
+        A graph removes the launch gaps, but it also orders the kernels of its branches in its own
+        way, so which of the two is faster depends on the workload; a caller that repeats the pass
+        (one call per decoder layer) times both once and keeps the faster."""
+        def ms(step_fn):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record()
+            for _ in range(steps):
+                step_fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / steps
+        return {"eager_ms": ms(self.run), "graph_ms": ms(graph.replay)}
+
     def forward_check(self, X, W, bias=None, corrected: bool = True):
         """The forward check of every linear after ``run()``: {linear name: (mean_err[C_out],
         sums[4])} as binary64 device tensors.  W8A8 workloads with row-wise 8-bit weights go

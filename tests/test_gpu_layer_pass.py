@@ -220,3 +220,9 @@ def test_graph_replay_equals_eager(overlap):
     for nm, outs in a.out.items():
         for k, v in outs.items():
             assert torch.equal(v.view(torch.uint8), b.out[nm][k].view(torch.uint8)), (nm, k)
+    # the trial of both launch modes times real passes and leaves the results as they were
+    trial = b.launch_trial(graph, steps=2)
+    assert 0.0 < trial["eager_ms"] < 50.0 and 0.0 < trial["graph_ms"] < 50.0
+    for nm, outs in a.out.items():
+        for k, v in outs.items():
+            assert torch.equal(v.view(torch.uint8), b.out[nm][k].view(torch.uint8)), (nm, k)
