@@ -7,14 +7,15 @@
 // and are bound by HBM bandwidth.
 //
 // Layout of the work: the columns are cut into slabs of at most 256 16-byte
-// vectors (2048 columns) and the rows into splits; one CTA per SM owns one
+// vectors (2048 columns; 320 or 384 vectors where that divides the row better)
+// and the rows into splits; one CTA per SM owns one
 // (slab, split) pair, so a thread owns one vector column for its whole life and
 // keeps that column's eight running minima, maxima and sums in registers.
 // A producer warp streams the CTA's rows through two shared-memory stages of
-// 24 rows each (up to 96 KB per stage) with 1-D bulk copies (TMA, completion on
-// mbarriers); eight consumer warps read the stages back conflict-free
+// 24 rows each (16 in the wider CTAs; up to 96 KB per stage) with 1-D bulk copies
+// (TMA, completion on mbarriers); the consumer warps read the stages back conflict-free
 // (consecutive lanes, consecutive 16-byte vectors).  Of the geometries timed
-// on B200 (2-6 stages of 8-24 rows, one or two CTAs per SM) this one was the
+// on B200 (2-6 stages of 8-24 rows, one or two CTAs per SM) the base one was the
 // fastest on both the 4096- and the 11008-column inputs.  min / max stay in packed 16-bit arithmetic (exact); sums
 // are binary32 over eight rows at a time (one mixed-precision add per element)
 // and are then added without rounding loss into a (hi, lo) pair of binary32
@@ -40,36 +41,63 @@ namespace aweq {
 #ifndef AWEQ_COL_CTAS_PER_SM
 #define AWEQ_COL_CTAS_PER_SM 1
 #endif
-constexpr int kColThreads = AWEQ_COL_THREADS;   // consumer threads = vectors per slab
-constexpr int kColRows = AWEQ_COL_ROWS;         // rows per stage
+constexpr int kColThreads = AWEQ_COL_THREADS;   // consumer threads = vectors per slab of the base geometry
+constexpr int kColRows = AWEQ_COL_ROWS;         // rows per stage of the base geometry
 constexpr int kColStages = AWEQ_COL_STAGES;
 constexpr int kColCtasPerSm = AWEQ_COL_CTAS_PER_SM;
 constexpr int kColTargetCtas = kColCtasPerSm * kSmCount;
 constexpr int kFlushRowsHost = 8;               // rows summed in binary32 before the error-free fold
+// Wider CTAs for the widths whose column count they divide better (a slab that fills the consumer
+// threads exactly, and larger bulk copies per row): 320 or 384 consumer threads with 16 rows per
+// stage.  Measured alone on 1 GiB inputs: 3072 columns (one contiguous slab of 384 vectors) 6.41 ->
+// 6.76 TB/s, 5120 (two slabs of 320) 6.74 -> 6.95, 9216 (three of 384) 6.85 -> 6.92; 4096, 11008,
+// 13824 and 36864 columns are best with 256.
+constexpr int kColWideRows = 16;
+constexpr int kColMaxThreads = 384;
 
 struct ColPlan {
     int nvec, nslab, slab_w, nsplit;
+    int threads;         // consumer threads of a CTA: 256, 320 or 384
     int phases;          // thread groups that share a slab's columns and split a stage's rows
     int stage_rows;      // rows per stage
     long long rows_per_split;
 };
 
-// Row phases and stage height.  A slab of w vectors keeps only w of the 256 consumer threads
+// Consumer threads for a row of nvec vectors: the candidate whose slabs leave the fewest threads
+// idle; ties go to the base geometry.  max_threads = 256 pins the base geometry (the built-in
+// scratch of aweq_stats_static is sized for it).
+static int pick_threads(int nvec, int max_threads)
+{
+    if (nvec <= kColThreads) return kColThreads;
+    const int cand[3] = {kColThreads, kColMaxThreads, 320};
+    int best = kColThreads;
+    double best_fill = 0.0;
+    for (int c : cand) {
+        if (c > max_threads) continue;
+        const int nslab = (nvec + c - 1) / c;
+        const double fill = (double)nvec / ((double)nslab * c);
+        if (fill > best_fill + 1e-9) { best_fill = fill; best = c; }
+    }
+    return best;
+}
+
+// Row phases and stage height.  A slab of w vectors keeps only w of the consumer threads
 // busy; when w <= 96 the idle threads take a second share of every stage's rows and write
 // partials of their own (more than two phases multiply the partials the finalize kernel has
 // to walk and were slower).  A stage holds as many rows as fit 96 KB (24 rows of a full slab):
 // narrow matrices get taller stages, so that one bulk copy still moves ~96 KB -- but a split
 // keeps at least a dozen stages, or filling and draining the two-stage ring shows.
 // (Narrower slabs with more phases were tried instead of idle threads and were slower.)
-static void pick_slabs(int nvec, long long rows_per_split, int *nslab_out, int *slab_w_out, int *phases_out,
+static void pick_slabs(int nvec, long long rows_per_split, int threads, int *nslab_out, int *slab_w_out, int *phases_out,
                        int *stage_rows_out)
 {
-    const int nslab = (nvec + kColThreads - 1) / kColThreads;
+    const int nslab = (nvec + threads - 1) / threads;
     const int w = (nvec + nslab - 1) / nslab;
     const int wpad = (w + 31) / 32 * 32;
     const int ph = wpad <= 96 ? 2 : 1;                         // from four warps per slab on, phases gained nothing
     const int unit = kFlushRowsHost * ph;                      // every phase gets whole eight-row groups
-    int rows = ph == 1 ? kColRows : (int)((size_t)kColRows * kColThreads / w) / unit * unit;
+    const int full_rows = threads == kColThreads ? kColRows : kColWideRows;
+    int rows = ph == 1 ? full_rows : (int)((size_t)kColRows * kColThreads / w) / unit * unit;
     if (rows > 256) rows = 256 / unit * unit;
     if (rows_per_split > 0 && rows > rows_per_split / 12) rows = (int)(rows_per_split / 12) / unit * unit;
     if (rows < unit) rows = unit;
@@ -79,11 +107,12 @@ static void pick_slabs(int nvec, long long rows_per_split, int *nslab_out, int *
     *stage_rows_out = rows;
 }
 
-ColPlan plan_colreduce(long long rows, long long cols)
+ColPlan plan_colreduce(long long rows, long long cols, int max_threads = kColMaxThreads)
 {
     ColPlan p;
     p.nvec = (int)(cols / 8);
-    pick_slabs(p.nvec, 0, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
+    p.threads = pick_threads(p.nvec, max_threads);
+    pick_slabs(p.nvec, 0, p.threads, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
     int nsplit = kColTargetCtas / p.nslab;
     if (nsplit < 1) nsplit = 1;
     long long max_split = (rows + 7) / 8;
@@ -93,28 +122,33 @@ ColPlan plan_colreduce(long long rows, long long cols)
     rps = (rps + 7) / 8 * 8;            // whole eight-row groups; the last stage of a split may be partial
     if (rps < 8) rps = 8;
     p.rows_per_split = rps;
-    pick_slabs(p.nvec, rps, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
+    pick_slabs(p.nvec, rps, p.threads, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
     p.nsplit = (int)((rows + rps - 1) / rps);
     if (p.nsplit < 1) p.nsplit = 1;
     return p;
 }
 
-size_t colreduce_ws_bytes(long long rows, long long cols)
+static size_t colreduce_ws_bytes_for(long long cols, int max_threads)
 {
     // pmin, pmax: float[nsplit * phases][cols]; psum: double[nsplit * phases][cols].  Sized for the
     // largest number of row splits any row count can get, so that a buffer sized
     // for N rows also serves every call with fewer rows (streamed chunks).
-    (void)rows;
     const int nvec = (int)(cols / 8);
     int nslab = 1, slab_w = 1, phases = 1, stage_rows = 8;
-    pick_slabs(nvec > 0 ? nvec : 1, 0, &nslab, &slab_w, &phases, &stage_rows);
+    pick_slabs(nvec > 0 ? nvec : 1, 0, pick_threads(nvec > 0 ? nvec : 1, max_threads), &nslab, &slab_w, &phases, &stage_rows);
     int max_split = kColTargetCtas / nslab;
     if (max_split < 1) max_split = 1;
     return (size_t)max_split * phases * (size_t)cols * 16 + 256;
 }
 
+size_t colreduce_ws_bytes(long long rows, long long cols)
+{
+    (void)rows;
+    return colreduce_ws_bytes_for(cols, kColMaxThreads);
+}
+
 constexpr int kFlushRows = kFlushRowsHost;
-static_assert(kColRows % kFlushRows == 0, "stage rows must be a multiple of the flush period");
+static_assert(kColRows % kFlushRows == 0 && kColWideRows % kFlushRows == 0, "stage rows must be a multiple of the flush period");
 
 // acc += widen(16-bit value): one mixed-precision add per element (exact widening,
 // one binary32 rounding), no separate conversion
@@ -192,8 +226,8 @@ struct ColSmem {
     int abort_flag;
 };
 
-template <class D, bool WITH_SUM>
-__global__ void __launch_bounds__(kColThreads + 32, kColCtasPerSm)
+template <class D, bool WITH_SUM, int NT>
+__global__ void __launch_bounds__(NT + 32, kColCtasPerSm)
 colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int slab_w,
                  int phases, int stage_rows, long long rows_per_split, long long cols, float *__restrict__ pmin,
                  float *__restrict__ pmax, double *__restrict__ psum, aweq_dev_status *st, long long rows_a,
@@ -234,7 +268,7 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
     pdl_begin();                 // everything above overlaps the tail of the previous kernel
     __syncthreads();
 
-    if (warp == kColThreads / 32) {
+    if (warp == NT / 32) {
         // ---------------- producer warp
         bool ok = true;
         int t = 0;
@@ -496,13 +530,13 @@ static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *
                                     float *omax, float *omean, double *osum, long long *count, int accumulate,
                                     void *ws, aweq_dev_status *st, cudaStream_t stream, float *negmin_max = nullptr,
                                     double *count_f64 = nullptr, long long rows_a = -1, float *omin_b = nullptr,
-                                    float *omax_b = nullptr)
+                                    float *omax_b = nullptr, int max_threads = kColMaxThreads)
 {
     long long rows_all = 0;
     for (int k = 0; k < segs.n; ++k) rows_all += segs.rows[k];
     const long long rows = rows_a < 0 ? rows_all : rows_a;
     const long long rows_b = rows_all - rows;
-    ColPlan p = plan_colreduce(rows, cols);
+    ColPlan p = plan_colreduce(rows, cols, max_threads);
     char *base = reinterpret_cast<char *>(ws);
     float *pmin = reinterpret_cast<float *>(base);
     const size_t nparts = (size_t)p.nsplit * p.phases;
@@ -516,13 +550,14 @@ static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *
         rps_b = (rps_b + 7) / 8 * 8;
     }
     const size_t smem = colreduce_smem_bytes(p.slab_w, p.stage_rows);
-    auto kern = colreduce_kernel<D, WITH_SUM>;
+    auto kern = p.threads == 384 ? colreduce_kernel<D, WITH_SUM, 384>
+              : p.threads == 320 ? colreduce_kernel<D, WITH_SUM, 320> : colreduce_kernel<D, WITH_SUM, kColThreads>;
     // set on every launch: the attribute belongs to the current device, which may change between calls
     AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)colreduce_smem_bytes(kColThreads, kColRows)));
     int nsplit_eff = rows > 0 ? (int)nparts : 0;
     if (rows > 0) {
-        AWEQ_LAUNCH(kern, dim3(p.nslab * p.nsplit), dim3(kColThreads + 32), smem, stream,
+        AWEQ_LAUNCH(kern, dim3(p.nslab * p.nsplit), dim3(p.threads + 32), smem, stream,
                     segs, rows_all, p.nvec, p.nslab, p.slab_w, p.phases, p.stage_rows, p.rows_per_split, cols, pmin, pmax,
                     psum, st, rows, rps_b, pmin_b, pmax_b);
     }
@@ -556,7 +591,7 @@ void colreduce_describe(long long rows, long long cols, long long plan[8])
 {
     const ColPlan p = plan_colreduce(rows, cols);
     plan[0] = (long long)p.nslab * p.nsplit;
-    plan[1] = kColThreads + 32;
+    plan[1] = p.threads + 32;
     plan[2] = (long long)colreduce_smem_bytes(p.slab_w, p.stage_rows);
     plan[3] = p.nslab;
     plan[4] = p.slab_w;
@@ -725,7 +760,7 @@ extern "C" aweq_status aweq_stats_static(const void *X, aweq_dtype dt, long long
     if (!X || !xmin || !xmax || !xmean) return AWEQ_ERR_NULL;
     if (dt != AWEQ_F16 && dt != AWEQ_BF16) return AWEQ_ERR_DTYPE;
     if (C_in <= 0 || (C_in % 8) != 0 || N <= 0 || N > (1ll << 40)) return AWEQ_ERR_SHAPE;
-    if (C_in > kStaticMaxCin || colreduce_ws_bytes(N, C_in) > kStaticScratchBytes) return AWEQ_ERR_LIMIT;
+    if (C_in > kStaticMaxCin || colreduce_ws_bytes_for(C_in, kColThreads) > kStaticScratchBytes) return AWEQ_ERR_LIMIT;
     if (ldx < C_in || (ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0) return AWEQ_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(xmin) & 15) != 0 || (reinterpret_cast<uintptr_t>(xmax) & 15) != 0)
         return AWEQ_ERR_ALIGN;
@@ -734,6 +769,17 @@ extern "C" aweq_status aweq_stats_static(const void *X, aweq_dtype dt, long long
     if (rc != AWEQ_OK) return rc;
     // every partial the reduction reads is written by this call first, so the
     // contents left by an earlier call need no clearing
-    return run_stats(X, dt, N, C_in, ldx, xmin, xmax, xmean, nullptr, nullptr, 0, scratch, st, (cudaStream_t)stream);
+    // (the base geometry: the array is sized for its number of partials)
+    ColSegs segs = {};
+    segs.base[0] = reinterpret_cast<const uint16_t *>(X);
+    segs.rows[0] = N;
+    segs.ld[0] = ldx;
+    segs.n = 1;
+    cudaStream_t cs = (cudaStream_t)stream;
+    if (dt == AWEQ_F16)
+        return launch_colreduce<F16, true>(segs, C_in, xmin, xmax, xmean, nullptr, nullptr, 0, scratch, st, cs, nullptr, nullptr,
+                                           -1, nullptr, nullptr, kColThreads);
+    return launch_colreduce<BF16, true>(segs, C_in, xmin, xmax, xmean, nullptr, nullptr, 0, scratch, st, cs, nullptr, nullptr, -1,
+                                        nullptr, nullptr, kColThreads);
 }
 

@@ -111,11 +111,16 @@ def test_column_reduction_plans_fit_the_hardware(lib):
             rc, (ctas, threads, smem, nslab, slab_w, nsplit, phases, stage_rows) = _plan(lib, 1, rows, cols)
             assert rc == 0
             nvec = cols // 8
-            assert 1 <= ctas <= 148 and ctas == nslab * nsplit and threads == 288
+            # 256, 320 or 384 consumer threads and the producer warp
+            assert 1 <= ctas <= 148 and ctas == nslab * nsplit and threads in (288, 352, 416)
+            consumers = threads - 32
             assert smem <= SMEM_LIMIT and smem == 128 + 2 * stage_rows * slab_w * 16
-            assert nslab * slab_w >= nvec and slab_w <= 256                 # every column has an owner
+            assert nslab * slab_w >= nvec and slab_w <= consumers           # every column has an owner
             assert phases in (1, 2) and stage_rows % (8 * phases) == 0      # whole eight-row groups per phase
-            assert phases * ((slab_w + 31) // 32 * 32) <= 256               # phases fit the consumer threads
+            assert phases * ((slab_w + 31) // 32 * 32) <= consumers         # phases fit the consumer threads
+            if consumers > 256:
+                # a wider CTA only where its slabs leave fewer threads idle than slabs of 256 would
+                assert nvec / (nslab * consumers) > nvec / (-(-nvec // 256) * 256) and phases == 1
             assert stage_rows * slab_w * 16 <= (1 << 20) - 1                # one mbarrier transaction count
             # the partials of the largest split count fit the advertised workspace
             assert nsplit * phases * cols * 16 + 256 <= lib.aweq_workspace_bytes(1, rows, cols, 0, 0, 0)
