@@ -100,7 +100,8 @@ unsigned long long aweq_launch_count(void);
  * only, no CUDA call; for diagnostics and tests).  op is AWEQ_OP_STATS / AWEQ_OP_WRANGE (the
  * column reduction), AWEQ_OP_EQUALIZE_QUANTIZE (row-wise weights) or AWEQ_OP_QUANT_ACT (per
  * token).  plan[8] receives
- *   column reduction: {CTAs, threads (256, 320 or 384 consumers and a producer warp), shared bytes,
+ *   column reduction: {CTAs, threads (256, 320 or 384 consumers and a producer warp), shared bytes
+ *                      (128 + stages x rows per stage x slab width x 16: two to four stages),
  *                      column slabs, slab width in 16-byte vectors, row splits, row phases, rows per stage}
  *   row quantisers:   {CTAs, threads, shared bytes, threads per row, vectors per thread,
  *                      rows per stage, stages, kernel: 2 plain loads without stages (rows per stage

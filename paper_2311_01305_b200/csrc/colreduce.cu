@@ -47,38 +47,39 @@ constexpr int kColStages = AWEQ_COL_STAGES;
 constexpr int kColCtasPerSm = AWEQ_COL_CTAS_PER_SM;
 constexpr int kColTargetCtas = kColCtasPerSm * kSmCount;
 constexpr int kFlushRowsHost = 8;               // rows summed in binary32 before the error-free fold
-// Wider CTAs for the widths whose column count they divide better (a slab that fills the consumer
-// threads exactly, and larger bulk copies per row): 320 or 384 consumer threads with 16 rows per
-// stage.  Measured alone on 1 GiB inputs: 3072 columns (one contiguous slab of 384 vectors) 6.41 ->
-// 6.76 TB/s, 5120 (two slabs of 320) 6.74 -> 6.95, 9216 (three of 384) 6.85 -> 6.92; 4096, 11008,
-// 13824 and 36864 columns are best with 256.
-constexpr int kColWideRows = 16;
+// Geometries (consumer threads x rows per stage x stages), from sweeps on 1 GiB inputs at eight widths:
+//   256 x 24 x 2   rows of one or two slabs (up to 4096 columns): few, tall stages      (4096: 7.04 TB/s)
+//   256 x 16 x 3   rows of three or more slabs: a third stage pays once a CTA's copies are short
+//                  (9216 columns 6.82 -> 7.11 TB/s, 11008 6.82 -> 7.09, 13824 6.96 -> 7.04, 36864 6.94 -> 6.91)
+//   320 x 8 x 4, 384 x 8 x 3   where the wider CTA brings a row into one or two slabs that 256 threads
+//                  cut into more (5120 columns = two slabs of 320: 6.72 -> 7.07; 3072 = one contiguous slab
+//                  of 384: 6.39 -> 6.92-7.03)
 constexpr int kColMaxThreads = 384;
+constexpr int kColMaxStages = 4;
 
 struct ColPlan {
     int nvec, nslab, slab_w, nsplit;
     int threads;         // consumer threads of a CTA: 256, 320 or 384
     int phases;          // thread groups that share a slab's columns and split a stage's rows
     int stage_rows;      // rows per stage
+    int stages;          // stages of the ring: 2, 3 or 4
     long long rows_per_split;
 };
 
-// Consumer threads for a row of nvec vectors: the candidate whose slabs leave the fewest threads
-// idle; ties go to the base geometry.  max_threads = 256 pins the base geometry (the built-in
-// scratch of aweq_stats_static is sized for it).
+// Consumer threads for a row of nvec vectors: 256, unless 320 or 384 threads bring the row into
+// one or two slabs where 256 need more (the narrower of the two that does).  max_threads = 256 pins
+// the base geometry (the built-in scratch of aweq_stats_static is sized for it).
 static int pick_threads(int nvec, int max_threads)
 {
-    if (nvec <= kColThreads) return kColThreads;
-    const int cand[3] = {kColThreads, kColMaxThreads, 320};
-    int best = kColThreads;
-    double best_fill = 0.0;
+    const int base_slabs = (nvec + kColThreads - 1) / kColThreads;
+    if (base_slabs <= 1) return kColThreads;
+    const int cand[2] = {320, kColMaxThreads};
     for (int c : cand) {
         if (c > max_threads) continue;
         const int nslab = (nvec + c - 1) / c;
-        const double fill = (double)nvec / ((double)nslab * c);
-        if (fill > best_fill + 1e-9) { best_fill = fill; best = c; }
+        if (nslab <= 2 && nslab < base_slabs) return c;
     }
-    return best;
+    return kColThreads;
 }
 
 // Row phases and stage height.  A slab of w vectors keeps only w of the consumer threads
@@ -89,14 +90,15 @@ static int pick_threads(int nvec, int max_threads)
 // keeps at least a dozen stages, or filling and draining the two-stage ring shows.
 // (Narrower slabs with more phases were tried instead of idle threads and were slower.)
 static void pick_slabs(int nvec, long long rows_per_split, int threads, int *nslab_out, int *slab_w_out, int *phases_out,
-                       int *stage_rows_out)
+                       int *stage_rows_out, int *stages_out)
 {
     const int nslab = (nvec + threads - 1) / threads;
     const int w = (nvec + nslab - 1) / nslab;
     const int wpad = (w + 31) / 32 * 32;
     const int ph = wpad <= 96 ? 2 : 1;                         // from four warps per slab on, phases gained nothing
     const int unit = kFlushRowsHost * ph;                      // every phase gets whole eight-row groups
-    const int full_rows = threads == kColThreads ? kColRows : kColWideRows;
+    const int stages = threads == 320 ? 4 : (threads == 384 || nslab >= 3) ? 3 : kColStages;
+    const int full_rows = threads > kColThreads ? 8 : stages == 3 ? 16 : kColRows;
     int rows = ph == 1 ? full_rows : (int)((size_t)kColRows * kColThreads / w) / unit * unit;
     if (rows > 256) rows = 256 / unit * unit;
     if (rows_per_split > 0 && rows > rows_per_split / 12) rows = (int)(rows_per_split / 12) / unit * unit;
@@ -105,6 +107,7 @@ static void pick_slabs(int nvec, long long rows_per_split, int threads, int *nsl
     *slab_w_out = w;
     *phases_out = ph;
     *stage_rows_out = rows;
+    *stages_out = stages;
 }
 
 ColPlan plan_colreduce(long long rows, long long cols, int max_threads = kColMaxThreads)
@@ -112,7 +115,7 @@ ColPlan plan_colreduce(long long rows, long long cols, int max_threads = kColMax
     ColPlan p;
     p.nvec = (int)(cols / 8);
     p.threads = pick_threads(p.nvec, max_threads);
-    pick_slabs(p.nvec, 0, p.threads, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
+    pick_slabs(p.nvec, 0, p.threads, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows, &p.stages);
     int nsplit = kColTargetCtas / p.nslab;
     if (nsplit < 1) nsplit = 1;
     long long max_split = (rows + 7) / 8;
@@ -122,7 +125,7 @@ ColPlan plan_colreduce(long long rows, long long cols, int max_threads = kColMax
     rps = (rps + 7) / 8 * 8;            // whole eight-row groups; the last stage of a split may be partial
     if (rps < 8) rps = 8;
     p.rows_per_split = rps;
-    pick_slabs(p.nvec, rps, p.threads, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows);
+    pick_slabs(p.nvec, rps, p.threads, &p.nslab, &p.slab_w, &p.phases, &p.stage_rows, &p.stages);
     p.nsplit = (int)((rows + rps - 1) / rps);
     if (p.nsplit < 1) p.nsplit = 1;
     return p;
@@ -134,8 +137,9 @@ static size_t colreduce_ws_bytes_for(long long cols, int max_threads)
     // largest number of row splits any row count can get, so that a buffer sized
     // for N rows also serves every call with fewer rows (streamed chunks).
     const int nvec = (int)(cols / 8);
-    int nslab = 1, slab_w = 1, phases = 1, stage_rows = 8;
-    pick_slabs(nvec > 0 ? nvec : 1, 0, pick_threads(nvec > 0 ? nvec : 1, max_threads), &nslab, &slab_w, &phases, &stage_rows);
+    int nslab = 1, slab_w = 1, phases = 1, stage_rows = 8, stages = 2;
+    pick_slabs(nvec > 0 ? nvec : 1, 0, pick_threads(nvec > 0 ? nvec : 1, max_threads), &nslab, &slab_w, &phases, &stage_rows,
+               &stages);
     int max_split = kColTargetCtas / nslab;
     if (max_split < 1) max_split = 1;
     return (size_t)max_split * phases * (size_t)cols * 16 + 256;
@@ -148,7 +152,7 @@ size_t colreduce_ws_bytes(long long rows, long long cols)
 }
 
 constexpr int kFlushRows = kFlushRowsHost;
-static_assert(kColRows % kFlushRows == 0 && kColWideRows % kFlushRows == 0, "stage rows must be a multiple of the flush period");
+static_assert(kColRows % kFlushRows == 0, "stage rows must be a multiple of the flush period");
 
 // acc += widen(16-bit value): one mixed-precision add per element (exact widening,
 // one binary32 rounding), no separate conversion
@@ -221,12 +225,12 @@ __device__ __forceinline__ void seg_locate(const ColSegs &sg, long long v, int &
 }
 
 struct ColSmem {
-    uint64_t full[kColStages];
-    uint64_t empty[kColStages];
+    uint64_t full[kColMaxStages];
+    uint64_t empty[kColMaxStages];
     int abort_flag;
 };
 
-template <class D, bool WITH_SUM, int NT>
+template <class D, bool WITH_SUM, int NT, int STAGES>
 __global__ void __launch_bounds__(NT + 32, kColCtasPerSm)
 colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int slab_w,
                  int phases, int stage_rows, long long rows_per_split, long long cols, float *__restrict__ pmin,
@@ -258,7 +262,7 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
     const size_t stage_vecs = (size_t)stage_rows * slab_w;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kColStages; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(&sm->full[s], 1);
             mbar_init(&sm->empty[s], active_warps);
         }
@@ -276,8 +280,8 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
         long long cur = job_r0[job];
         const long long r1 = job_r1[job];
         for (; cur < r1 && ok; ++t) {
-            const int s = t % kColStages;
-            const uint32_t use = t / kColStages;
+            const int s = t % STAGES;
+            const uint32_t use = t / STAGES;
             if (use > 0) {
                 ok = mbar_wait(&sm->empty[s], (use - 1) & 1);
                 ok = __all_sync(0xffffffffu, ok);
@@ -328,8 +332,8 @@ colreduce_kernel(const ColSegs segs, long long nrows, int nvec, int nslab, int s
         long long cur = job_r0[job];
         const long long r1 = job_r1[job];
         for (; cur < r1; ++t) {
-            const int s = t % kColStages;
-            const uint32_t use = t / kColStages;
+            const int s = t % STAGES;
+            const uint32_t use = t / STAGES;
             ok = mbar_wait(&sm->full[s], use & 1);
             if (!ok || *reinterpret_cast<volatile int *>(&sm->abort_flag)) { ok = false; break; }
             int m;
@@ -511,9 +515,9 @@ __global__ void bump_count_kernel(long long *count, long long nrows, int accumul
     count[0] = (accumulate ? count[0] : 0) + nrows;
 }
 
-static size_t colreduce_smem_bytes(int slab_w, int stage_rows)
+static size_t colreduce_smem_bytes(int slab_w, int stage_rows, int stages)
 {
-    return 128 + (size_t)kColStages * stage_rows * slab_w * 16;
+    return 128 + (size_t)stages * stage_rows * slab_w * 16;
 }
 
 // Scratch of a fused statistics + weight-range launch: the partials of both jobs.
@@ -549,12 +553,14 @@ static aweq_status launch_colreduce(const ColSegs &segs, long long cols, float *
         rps_b = (rows_b + p.nsplit - 1) / p.nsplit;
         rps_b = (rps_b + 7) / 8 * 8;
     }
-    const size_t smem = colreduce_smem_bytes(p.slab_w, p.stage_rows);
-    auto kern = p.threads == 384 ? colreduce_kernel<D, WITH_SUM, 384>
-              : p.threads == 320 ? colreduce_kernel<D, WITH_SUM, 320> : colreduce_kernel<D, WITH_SUM, kColThreads>;
+    const size_t smem = colreduce_smem_bytes(p.slab_w, p.stage_rows, p.stages);
+    auto kern = p.threads == 384   ? colreduce_kernel<D, WITH_SUM, 384, 3>
+                : p.threads == 320 ? colreduce_kernel<D, WITH_SUM, 320, 4>
+                : p.stages == 3    ? colreduce_kernel<D, WITH_SUM, kColThreads, 3>
+                                   : colreduce_kernel<D, WITH_SUM, kColThreads, kColStages>;
     // set on every launch: the attribute belongs to the current device, which may change between calls
     AWEQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)colreduce_smem_bytes(kColThreads, kColRows)));
+                                      (int)colreduce_smem_bytes(kColThreads, kColRows, kColStages)));
     int nsplit_eff = rows > 0 ? (int)nparts : 0;
     if (rows > 0) {
         AWEQ_LAUNCH(kern, dim3(p.nslab * p.nsplit), dim3(p.threads + 32), smem, stream,
@@ -592,7 +598,7 @@ void colreduce_describe(long long rows, long long cols, long long plan[8])
     const ColPlan p = plan_colreduce(rows, cols);
     plan[0] = (long long)p.nslab * p.nsplit;
     plan[1] = p.threads + 32;
-    plan[2] = (long long)colreduce_smem_bytes(p.slab_w, p.stage_rows);
+    plan[2] = (long long)colreduce_smem_bytes(p.slab_w, p.stage_rows, p.stages);
     plan[3] = p.nslab;
     plan[4] = p.slab_w;
     plan[5] = p.nsplit;

@@ -114,13 +114,17 @@ def test_column_reduction_plans_fit_the_hardware(lib):
             # 256, 320 or 384 consumer threads and the producer warp
             assert 1 <= ctas <= 148 and ctas == nslab * nsplit and threads in (288, 352, 416)
             consumers = threads - 32
-            assert smem <= SMEM_LIMIT and smem == 128 + 2 * stage_rows * slab_w * 16
+            stages, rem = divmod(smem - 128, stage_rows * slab_w * 16)        # the ring: two to four stages
+            assert smem <= SMEM_LIMIT and rem == 0 and stages in (2, 3, 4)
             assert nslab * slab_w >= nvec and slab_w <= consumers           # every column has an owner
             assert phases in (1, 2) and stage_rows % (8 * phases) == 0      # whole eight-row groups per phase
             assert phases * ((slab_w + 31) // 32 * 32) <= consumers         # phases fit the consumer threads
+            base_slabs = -(-nvec // 256)
             if consumers > 256:
-                # a wider CTA only where its slabs leave fewer threads idle than slabs of 256 would
-                assert nvec / (nslab * consumers) > nvec / (-(-nvec // 256) * 256) and phases == 1
+                # a wider CTA only where it brings the row into one or two slabs that 256 threads cut into more
+                assert nslab <= 2 and nslab < base_slabs and phases == 1 and stages == (4 if consumers == 320 else 3)
+            else:
+                assert stages == (3 if nslab >= 3 else 2)
             assert stage_rows * slab_w * 16 <= (1 << 20) - 1                # one mbarrier transaction count
             # the partials of the largest split count fit the advertised workspace
             assert nsplit * phases * cols * 16 + 256 <= lib.aweq_workspace_bytes(1, rows, cols, 0, 0, 0)
