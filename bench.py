@@ -274,18 +274,18 @@ def run_forward_check(args, wl, bits):
 # streams, eager), taken as a single profiler range (dram__bytes_read.sum, dram__bytes_write.sum):
 # {(workload, bits): (bytes read, bytes written)}.  Compared with the algorithmic bytes they say how
 # much of the pass the L2 served.  The kernels have not changed since the counters were taken.
-PASS_DRAM_BYTES = {("llama7b_layer_w4w3_g128", 4): (13012440320, 124258816),
-                   ("llama7b_layer_w4w3_g128", 3): (13011749888, 106911488),
-                   ("llama13b_layer_w8a8", 8): (31906331136, 7965332224),
-                   ("opt66b_ffn_w8a8", 8): (26884471808, 6710370304),
-                   ("opt125m_model_w8a8", 8): (5661844736, 1410405888)}
+PASS_DRAM_BYTES = {("llama7b_layer_w4w3_g128", 4): (13027861248, 108804096),
+                   ("llama7b_layer_w4w3_g128", 3): (13019588864, 86600960),
+                   ("llama13b_layer_w8a8", 8): (31903268608, 7977698304),
+                   ("opt66b_ffn_w8a8", 8): (26883141376, 6708150784),
+                   ("opt125m_model_w8a8", 8): (5662176768, 1417811968)}
 # Share of the second read of W (step 4, after step 2 has streamed the same matrices) that the L2 serves
 # instead of HBM.  "scheduled": from the range capture above (algorithmic read bytes minus DRAM read bytes,
 # over one read of W); a statistics sweep of the next input runs between the two reads and flushes the L2.
 # "one_stream": per-kernel DRAM read bytes of the step-4 kernels with every kernel of a pass serialised
 # (one stream, 1/32 of the tokens; weights are full size at any token count): what the L2 could serve.
-W_SECOND_READ_FROM_L2 = {("llama7b_layer_w4w3_g128", 4): {"scheduled": 0.027, "one_stream": 0.605},
-                         ("llama7b_layer_w4w3_g128", 3): {"scheduled": 0.029, "one_stream": 0.618}}
+W_SECOND_READ_FROM_L2 = {("llama7b_layer_w4w3_g128", 4): {"scheduled": 0.0, "one_stream": 0.605},
+                         ("llama7b_layer_w4w3_g128", 3): {"scheduled": 0.009, "one_stream": 0.618}}
 # DRAM traffic of the statistics sweep per launch, from a one-kernel capture at 1/8 of the tokens
 # (268.44 MB of X and 100.66 MB of W in one launch: 369.21 MB read): reads grow with the rows; the few MB written during the launch are
 # dirty lines of earlier kernels leaving the L2, not traffic of the sweep.
