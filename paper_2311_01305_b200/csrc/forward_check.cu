@@ -109,11 +109,11 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
             b[c] = bias ? (double)D::one(bias[o0 + c]) : 0.0;
             bq[c] = bias_q ? (double)bias_q[o0 + c] : b[c];      // no corrected bias: the layer keeps its own
         }
-#pragma unroll 4
+#pragma unroll 2
         for (long long n = r0 + warp; n < r1; n += 8) {
             const float4 y4 = __ldg(reinterpret_cast<const float4 *>(Y + n * C_out + o0));
             const float yv[4] = {y4.x, y4.y, y4.z, y4.w};
-            int sv[4] = {0, 0, 0, 0}, tv[4] = {0, 0, 0, 0};
+            double sv[4] = {0.0, 0.0, 0.0, 0.0};     // the integer contraction, exact in binary64
             float dv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             double zx = 0.0, u = 0.0, sx = 0.0;
             if (WO) {
@@ -121,10 +121,10 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
                 dv[0] = d4.x; dv[1] = d4.y; dv[2] = d4.z; dv[3] = d4.w;
             } else {
                 const int4 s4 = __ldg(reinterpret_cast<const int4 *>(S + n * C_out + o0));
-                sv[0] = s4.x; sv[1] = s4.y; sv[2] = s4.z; sv[3] = s4.w;
-                if (S2) {
+                sv[0] = (double)s4.x; sv[1] = (double)s4.y; sv[2] = (double)s4.z; sv[3] = (double)s4.w;
+                if (S2) {                     // a K above 32768 comes as two halves (the branch is uniform)
                     const int4 t4 = __ldg(reinterpret_cast<const int4 *>(S2 + n * C_out + o0));
-                    tv[0] = t4.x; tv[1] = t4.y; tv[2] = t4.z; tv[3] = t4.w;
+                    sv[0] += (double)t4.x; sv[1] += (double)t4.y; sv[2] += (double)t4.z; sv[3] += (double)t4.w;
                 }
                 zx = (double)act_zp[n];
                 u = (double)K * zx - (double)rx[n];
@@ -137,7 +137,7 @@ fc_compare_kernel(const int *__restrict__ S, const int *__restrict__ S2, const f
                 if (WO) {
                     d = (double)dv[c] + (bq[c] - b[c]);
                 } else {
-                    const double acc = ((double)sv[c] + (double)tv[c]) - zx * cwd[c] + zw[c] * u;
+                    const double acc = sv[c] - zx * cwd[c] + zw[c] * u;
                     d = (sx * sw[c] * acc + bq[c]) - y;
                 }
                 sd[c] += d;
