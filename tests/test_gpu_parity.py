@@ -44,7 +44,11 @@ def dev_stats(X, N=None):
 # ------------------------------------------------------------------ step 1
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
 @pytest.mark.parametrize("shape", [(1, 8), (7, 8), (257, 24), (1000, 768), (2048, 768), (4099, 2056),
-                                   (333, 11008), (9000, 4096), (70, 36864)])
+                                   (333, 11008), (9000, 4096), (70, 36864),
+                                   # the wider CTAs (320 / 384 consumer threads): exact fits and ragged slabs, and rows of
+                                   # three or more slabs (three stages)
+                                   (3001, 3072), (1777, 5120), (1500, 2824), (700, 4808), (900, 5608), (600, 9216),
+                                   (650, 13824)])
 def test_stats_matches_oracle(shape, dtype):
     Xc = util.rand16(shape, dtype, seed=shape[0] * 31 + shape[1], offset=2.0, outlier_cols=min(6, shape[1] // 4))
     o_min, o_max, o_mean, o_sum = orc.stats(util.bits(Xc), util.odt(Xc))
@@ -122,7 +126,7 @@ def test_stats_counts_nonfinite_channels():
 
 # ------------------------------------------------------------------ step 2
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
-@pytest.mark.parametrize("shape", [(768, 768), (3072, 768), (100, 4104), (4096, 11008)])
+@pytest.mark.parametrize("shape", [(768, 768), (3072, 768), (100, 4104), (4096, 11008), (5120, 5120), (64, 5608), (777, 3072)])
 def test_wrange_matches_oracle_and_merges(shape, dtype):
     Wc = util.rand16(shape, dtype, seed=shape[0] + 7 * shape[1], scale=0.02)
     W = Wc.to(DEV)
