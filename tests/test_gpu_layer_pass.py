@@ -96,7 +96,9 @@ def test_decoder_layer_shapes_with_shared_inputs_few_tokens(name, bits):
     compare_layer(wl, bits, Xc, Wc, None)
 
 
-@pytest.mark.parametrize("n_w,c_in,tokens", [(5, 1032, 300), (3, 776, 37), (1, 4096, 3000), (4, 264, 1000)])
+@pytest.mark.parametrize("n_w,c_in,tokens", [(5, 1032, 300), (3, 776, 37), (1, 4096, 3000), (4, 264, 1000),
+                                             # the 384- and 320-thread sweeps with ragged slabs, and a three-stage ring
+                                             (2, 2824, 1500), (3, 4808, 900), (2, 5608, 333), (1, 9224, 400)])
 def test_matrices_sharing_one_input_fused_and_separate_ranges(n_w, c_in, tokens):
     """Up to three matrices on one input have their ranges taken inside the statistics sweep (one
     launch, the matrices as further segments of the row stack); four or more go through launches of
