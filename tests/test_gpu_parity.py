@@ -425,7 +425,7 @@ def dev_quant_act(X, rinv, bits, gran, lo_hi=None):
                                     (130, 9216), (129, 11008), (65, 13824), (33, 36864), (20, 40960),
                                     (70, 10248), (41, 20488), (1, 13824), (23, 24576), (9, 24568), (7, 36872), (5, 24584), (14, 32768), (1, 36864),
                                     # plain-load teams with the next row in flight: every team size at its widest and just past it,
-                                    # a row count below the number of teams, the first width of the tile kernel
+                                    # a row count below the number of teams, a width just past the eight-warp teams
                                     (3000, 1536), (2500, 1544), (3, 768), (600, 3080), (400, 6144), (350, 6152),
                                     (200, 12288), (2, 12288), (100, 12296)])
 def test_quant_act_per_token(N, C_in, dtype):
